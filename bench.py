@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the GQLA decode hot path on B200.
+
+A step = one pass of the absorb path (absorb_q -> decode_absorb -> combine_splits -> up_proj)
+over the canonical workload (h_q=128, g=8, d_h=128, r_kv=512, d_r=64, B=64, T=4096, s_q=1,
+bf16 cache).  The GQA path (decode_gqa -> combine_splits on the expanded cache, s_q=2) is
+measured in the same run and reported under "paths".  One JSON line on stdout.
+
+    python bench.py --gpus 1 --steps 50 --warmup 5
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N   (independent replicas)
+    python bench.py --impl reference      (the fp64 CPU oracle on the host cores)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2605_15250_b200 import accounting as acct
+from paper_2605_15250_b200 import synth
+
+METRIC = "decode attn tokens/s (absorb path, canonical config, 1 B200)"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as fh:
+            d = json.load(fh)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.06)
+        self.proc.terminate()
+        out, _ = self.proc.communicate(timeout=10)
+        sm, mx, reasons = [], [], set()
+        for line in out.strip().splitlines():
+            f = [c.strip() for c in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def pick_splits(batch: int, ctas_per_seq: int, min_len: int, n_sm: int = 148) -> int:
+    """Smallest split count that gives every SM about two work units, with >= 512 rows per split."""
+    s = 1
+    while batch * ctas_per_seq * s < 2 * n_sm and (min_len // (2 * s)) >= 512:
+        s *= 2
+    return s
+
+
+# ---------------------------------------------------------------------------------- reference arm (oracle)
+
+
+def oracle_tokens_per_s(w: synth.Workload, x: dict, n_seqs: int, steps: int, warmup: int):
+    """Times the fp64 oracle's absorb path on the first n_seqs sequences of the workload."""
+    from threadpoolctl import threadpool_info
+
+    from oracle import gqla_oracle as O
+
+    od = O.Dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)
+    idx = list(range(n_seqs))
+    ss, sl = x["seq_start"].numpy()[idx], x["seqlens"].numpy()[idx]
+    n_rows = int(ss[-1] + sl[-1])
+
+    def step():
+        f_qc, f_qr = synth.to_f64(x["q_c"][idx]), synth.to_f64(x["q_r"][idx])
+        return O.absorb_path(od, f_qc, f_qr, synth.to_f64(x["w_uk"]), synth.to_f64(x["w_uv"]),
+                             x["cache"][:n_rows].to(torch.float64).numpy(), ss, sl, w.s_q, w.scale)
+
+    for _ in range(warmup):
+        step()
+    times = []
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        step()
+        times.append(time.perf_counter() - t0)
+    cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    per_step = sum(times) / len(times)
+    return n_seqs * w.s_q / per_step, per_step, cores
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = synth.WORKLOADS["C1"]
+    x = synth.make_inputs(w)
+    n_seqs = 16
+    val, per_step, cores = oracle_tokens_per_s(w, x, n_seqs, args.steps, min(args.warmup, 1))
+    sample = f"first {n_seqs} of {w.batch} sequences per step, all {w.h_q} heads, T={w.seqlen}"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "C1 canonical absorb path: h_q=128 g=8 d_h=128 r_kv=512 d_r=64 B=64 T=4096 s_q=1",
+                   "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------- our arm
+
+
+def time_region(fn, steps: int, dist_on: bool):
+    """Times `steps` calls of fn with CUDA events on the current stream; returns total ms (max over ranks)."""
+    import torch.distributed as dist
+
+    if dist_on:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    if dist_on:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    if dist_on:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
+def run_ours(args):
+    import torch.distributed as dist
+
+    from paper_2605_15250_b200 import binding as B
+    from paper_2605_15250_b200 import build as gbuild
+    from paper_2605_15250_b200.decoder import GqlaDecoder
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist_on = world > 1
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    if dist_on:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        gbuild.build()
+    if dist_on:
+        dist.barrier()
+    B.lib()
+    peaks, peak_kind = load_peaks()
+    steps, warmup = args.steps, max(args.warmup, 3)
+
+    # ---- workload: replicas only -- every rank owns an independent batch (no data-path collective)
+    w1 = synth.WORKLOADS["C1"].with_(seed=synth.WORKLOADS["C1"].seed + 0x100 * rank)
+    x = synth.make_inputs(w1)
+    dev = torch.device("cuda", local_rank)
+    dec = GqlaDecoder(w1.h_q, w1.g, w1.d_h, w1.r_kv, w1.d_r, x["w_uk"].to(dev), x["w_uv"].to(dev),
+                      x["cache"].to(dev), x["seq_start"].to(dev), x["seqlens"].to(dev), w1.scale)
+    q_c, q_r = x["q_c"].to(dev), x["q_r"].to(dev)
+    total_tokens = int(x["seqlens"].sum())
+    kern_a = B.kernel_for(dec.dims, torch.bfloat16, w1.s_q, "absorb")
+    S_a = args.splits if args.splits > 0 else pick_splits(w1.batch, 2 if kern_a == "tcgen05" else 1, w1.seqlen)
+
+    def absorb_step():
+        dec.absorb_step(q_c, q_r, S_a)
+
+    for _ in range(warmup):
+        absorb_step()
+    dec.check_status()
+
+    # dominant kernel alone, timed live with events around each launch inside the timed region
+    q_hat = dec._get("q_hat", (w1.batch, w1.s_q, w1.h_q, w1.d_abs), torch.bfloat16)
+    o_part = dec._get("o_part_a", (w1.batch, S_a, w1.s_q, w1.h_q, w1.r_kv), torch.float32)
+    lse_part = dec._get("lse_part_a", (w1.batch, S_a, w1.s_q, w1.h_q), torch.float32)
+    o_hat = dec._get("o_hat", (w1.batch, w1.s_q, w1.h_q, w1.r_kv), torch.bfloat16)
+    o_out = dec._get("o_a", (w1.batch, w1.s_q, w1.h_q, w1.d_h), torch.bfloat16)
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    it = {"i": 0}
+
+    def absorb_step_instrumented():
+        a, b = kev[it["i"]]
+        it["i"] += 1
+        B.gqla_absorb_q(dec.dims, q_c, q_r, dec.w_uk, q_hat)
+        a.record()
+        B.gqla_decode_absorb(dec.dims, q_hat, dec.cache, dec.seq_start, dec.seqlens, dec.scale, S_a, o_part, lse_part,
+                             dec.status)
+        b.record()
+        B.gqla_combine_splits(o_part, lse_part, o_hat, None)
+        B.gqla_up_proj(dec.dims, o_hat, dec.w_uv, o_out)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    total_ms = time_region(absorb_step_instrumented, steps, dist_on)
+    clocks = sampler.stop()
+    dec.check_status()
+    ms_per_step = total_ms / steps
+    kern_ms = statistics.mean(a.elapsed_time(b) for a, b in kev)
+    value = world * w1.batch * w1.s_q / (ms_per_step * 1e-3)
+
+    kbytes = acct.decode_kernel_bytes("absorb", h_q=w1.h_q, g=w1.g, d_h=w1.d_h, r_kv=w1.r_kv, d_r=w1.d_r,
+                                      s_q=w1.s_q, batch=w1.batch, total_tokens=total_tokens, num_splits=S_a)
+    kflops = acct.absorb_flops(w1.h_q, w1.r_kv, w1.d_r, w1.s_q, total_tokens)
+    t_mem = kbytes / (peaks["hbm_gbs"] * 1e9)
+    t_mma = kflops / (peaks["bf16_tflops"] * 1e12)
+    gbs = kbytes / (kern_ms * 1e-3) / 1e9
+    tfs = kflops / (kern_ms * 1e-3) / 1e12
+    if t_mem >= t_mma:
+        roof = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / peaks["hbm_gbs"]}
+    else:
+        roof = {"bound": "tensor", "achieved": tfs, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": tfs / peaks["bf16_tflops"]}
+    roof.update({"traffic": None, "kernel": f"gqla_decode_absorb[{kern_a}]", "kernel_us": kern_ms * 1e3,
+                 "peak_source": f"of {peak_kind}", "algorithmic_bytes": kbytes, "flops": kflops,
+                 "achieved_gbs": gbs, "achieved_tflops": tfs,
+                 "frac_of_roofline_time": max(t_mem, t_mma) / (kern_ms * 1e-3),
+                 "frac_of_nominal_roofline": acct.roofline_time(kflops, kbytes, 2.25e15, 8e12) / (kern_ms * 1e-3)})
+
+    # ---- end to end through the public API with host buffers: per step, the queries and the step's new
+    # cache rows go host -> device from pinned memory, and the attention output comes back.
+    h_qc, h_qr = x["q_c"].pin_memory(), x["q_r"].pin_memory()
+    T = w1.seqlen
+    cache3 = dec.cache.view(w1.batch, T, w1.d_abs)
+    h_new = x["cache"].view(w1.batch, T, w1.d_abs)[:, T - w1.s_q:, :].contiguous().pin_memory()
+    d_new = torch.empty_like(h_new, device=dev)
+    h_out = torch.empty((w1.batch, w1.s_q, w1.h_q, w1.d_h), dtype=torch.bfloat16).pin_memory()
+
+    def e2e_step():
+        q_c.copy_(h_qc, non_blocking=True)
+        q_r.copy_(h_qr, non_blocking=True)
+        d_new.copy_(h_new, non_blocking=True)
+        cache3[:, T - w1.s_q:, :].copy_(d_new)
+        o = dec.absorb_step(q_c, q_r, S_a)
+        h_out.copy_(o, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for _ in range(3):
+        e2e_step()
+    e2e_ms = time_region(e2e_step, steps, dist_on) / steps
+    e2e = {"value": world * w1.batch * w1.s_q / (e2e_ms * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": h_qc.numel() * 2 + h_qr.numel() * 2 + h_new.numel() * 2,
+           "d2h_bytes_per_step": h_out.numel() * 2, "ms_per_step": e2e_ms}
+
+    # ---- GQA path on the same weights and latent (config 2: expanded cache, s_q = 2)
+    w2 = synth.WORKLOADS["C2"].with_(seed=w1.seed)
+    x2 = synth.make_inputs(w2)
+    q2 = torch.cat([x2["q_c"], x2["q_r"]], -1).contiguous().to(dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    dec.expand_cache()
+    ev1.record()
+    torch.cuda.synchronize()
+    expand_ms = ev0.elapsed_time(ev1)
+    kern_g = B.kernel_for(dec.dims, torch.bfloat16, w2.s_q, "gqa")
+    S_g = args.splits if args.splits > 0 else pick_splits(w2.batch, w2.g, w2.seqlen)
+    og_part = dec._get("o_part_g", (w2.batch, S_g, w2.s_q, w2.h_q, w2.d_h), torch.float32)
+    lg_part = dec._get("lse_part_g", (w2.batch, S_g, w2.s_q, w2.h_q), torch.float32)
+    og = dec._get("o_g", (w2.batch, w2.s_q, w2.h_q, w2.d_h), torch.bfloat16)
+    gev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    it["i"] = 0
+
+    def gqa_step_instrumented():
+        a, b = gev[it["i"]]
+        it["i"] += 1
+        a.record()
+        B.gqla_decode_gqa(dec.dims, q2, dec.k_c, dec.v, dec.k_r, dec.seq_start, dec.seqlens, dec.scale, S_g, og_part,
+                          lg_part, dec.status)
+        b.record()
+        B.gqla_combine_splits(og_part, lg_part, og, None)
+
+    for _ in range(warmup):
+        dec.gqa_step(q2, S_g)
+    gqa_ms = time_region(gqa_step_instrumented, steps, dist_on) / steps
+    dec.check_status()
+    gk_ms = statistics.mean(a.elapsed_time(b) for a, b in gev)
+    gbytes = acct.decode_kernel_bytes("gqa", h_q=w2.h_q, g=w2.g, d_h=w2.d_h, r_kv=w2.r_kv, d_r=w2.d_r, s_q=w2.s_q,
+                                      batch=w2.batch, total_tokens=total_tokens, num_splits=S_g)
+    gflops = acct.gqa_flops(w2.h_q, w2.d_h, w2.d_r, w2.s_q, total_tokens)
+    g_gbs = gbytes / (gk_ms * 1e-3) / 1e9
+    paths = {
+        "absorb": {"workload": "C1", "s_q": w1.s_q, "num_splits": S_a, "kernel": kern_a, "ms_per_step": ms_per_step,
+                   "tokens_per_s": value, "decode_kernel_us": kern_ms * 1e3, "gbs": gbs, "tflops": tfs},
+        "gqa": {"workload": "C2", "s_q": w2.s_q, "num_splits": S_g, "kernel": kern_g, "ms_per_step": gqa_ms,
+                "tokens_per_s": world * w2.batch * w2.s_q / (gqa_ms * 1e-3), "decode_kernel_us": gk_ms * 1e3,
+                "gbs": g_gbs, "tflops": gflops / (gk_ms * 1e-3) / 1e12,
+                "roofline": {"bound": "hbm", "achieved": g_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                             "frac": g_gbs / peaks["hbm_gbs"], "frac_of_8tbs": g_gbs / 8000.0,
+                             "algorithmic_bytes": gbytes, "peak_source": f"of {peak_kind}"},
+                "expand_cache_ms_one_shot": expand_ms},
+    }
+
+    # ---- CPU baseline: the oracle as it stands, rank 0 at N=1 only
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_seqs = w1.batch
+        val, per_step, cores = oracle_tokens_per_s(w1, x, n_seqs, 5, 1)
+        cpu = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"first {n_seqs} of {w1.batch} sequences of C1, all heads, 5 timed passes "
+                         f"({per_step:.2f} s each)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "C1 canonical absorb path: h_q=128 g=8 d_h=128 r_kv=512 d_r=64 B=64 T=4096 s_q=1 "
+                                   "bf16 cache (576 elems/token)", "num_splits": S_a, "parallelism": "replicas only",
+                       "l2": "inputs larger than L2 (302 MB cache vs 126 MB L2); no flush"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * steps, "roofline": roof, "cpu_baseline": cpu,
+            "paths": paths,
+        }
+        print(json.dumps(line))
+    if dist_on:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--splits", type=int, default=0, help="force the split count (0 = automatic)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

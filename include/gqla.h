@@ -1,0 +1,145 @@
+/*
+ * gqla.h -- C ABI of the GQLA decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * GQLA (Group-Query Latent Attention) weights expose two algebraically
+ * equivalent decoding paths (paper Sec. 3.1, "Two equivalent decoding paths"):
+ *
+ *   MQA-absorb path, Eq. (mqa):  all h_q heads attend the shared latent
+ *       k_hat_s = [c_s^KV ; k_s^R]  (r_kv + d_r wide),  v_hat_s = c_s^KV,
+ *       with W^UK folded into the query and W^UV applied to the output.
+ *   GQA path, Eq. (mha):  head i attends its group's expanded cache
+ *       k_{s,i} = [k^C_{s,j(i)} ; k_s^R],  v_{s,i} = v^C_{s,j(i)},
+ *       j(i) = ceil(i / (h_q/g)).
+ *
+ * General conventions
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  The library
+ *     allocates nothing, frees nothing, and never synchronises; each call
+ *     enqueues its kernels on `stream` (a cudaStream_t passed as void*, NULL =
+ *     the legacy default stream) and returns.
+ *   - Tensors are row-major with the innermost dimension contiguous.  Base
+ *     pointers and row strides must be 16-byte aligned (GQLA_ERR_ALIGN).
+ *   - `dtype` is the storage type of q, cache and weights: GQLA_BF16 or
+ *     GQLA_F32.  Accumulation, softmax statistics, split partials and LSE are
+ *     always fp32.  With GQLA_BF16 the softmax probabilities are rounded to
+ *     bf16 before the P.V contraction on the tensor-core kernels.
+ *   - Weights W^UK, W^UV are stored [g, r_kv, d_h]: W[j][r][d] is entry (d, r)
+ *     of the paper's group-j slice W_j in R^{d_h x r_kv}.
+ *   - Sequence b owns cache rows seq_start[b] .. seq_start[b]+seqlens[b]-1.
+ *     seqlens[b] already counts the s_q tokens of this step (their rows are
+ *     appended before the call).  Query p (0 <= p < s_q) sits at position
+ *     seqlens[b]-s_q+p and attends rows [0, seqlens[b]-(s_q-1-p)): the causal
+ *     sum  sum_{s=1..t}  of Eqs. (mha)/(mqa).  A query with no visible row
+ *     yields o = 0 and lse = -inf.
+ *   - Split-KV: split k of S covers rows [k*chunk, min((k+1)*chunk, T)) with
+ *     chunk = ceil(ceil(T/S)/64)*64; a split may be empty (o = 0, lse = -inf).
+ *     Each partial is normalised within its split; lse is the natural-log
+ *     sum-exp of the scaled scores.
+ *   - Errors: argument violations return a code before anything is launched.
+ *     A launch failure returns GQLA_ERR_CUDA.  Device-side waits are bounded;
+ *     if one expires the kernel writes a non-zero code to *status_word (device
+ *     int32, may be NULL) and exits -- the call itself stays asynchronous.
+ */
+#ifndef GQLA_H_
+#define GQLA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* The (h_q, g, d_h, r_kv, d_h^R) tuple of Sec. 4.2; canonical (128, 8, 128, 512, 64).
+ * The value dimension equals d_h. */
+typedef struct {
+    int32_t h_q;  /* query heads                      */
+    int32_t g;    /* K/V groups, h_q % g == 0          */
+    int32_t d_h;  /* per-head dim                      */
+    int32_t r_kv; /* latent rank                       */
+    int32_t d_r;  /* decoupled-RoPE dim d_h^R          */
+} gqla_dims;
+
+typedef enum {
+    GQLA_OK = 0,
+    GQLA_ERR_NULL = 1,        /* a required pointer is NULL                     */
+    GQLA_ERR_SHAPE = 2,       /* a dimension / count is out of range            */
+    GQLA_ERR_ALIGN = 3,       /* pointer or stride not 16-byte aligned          */
+    GQLA_ERR_DTYPE = 4,       /* unknown dtype                                  */
+    GQLA_ERR_UNSUPPORTED = 5, /* valid but no kernel covers it                  */
+    GQLA_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed            */
+    GQLA_ERR_TIMEOUT = 7      /* value written to *status_word by a bounded wait */
+} gqla_status;
+
+typedef enum { GQLA_BF16 = 0, GQLA_F32 = 1 } gqla_dtype;
+
+/* Kernel policy (process-wide): AUTO picks the tensor-core (tcgen05) kernels
+ * when the shape is covered and the generic SIMT kernels otherwise; GENERIC
+ * forces the SIMT kernels (used by tests to cross-check the two). */
+typedef enum { GQLA_POLICY_AUTO = 0, GQLA_POLICY_GENERIC = 1 } gqla_policy;
+void gqla_set_policy(gqla_policy p);
+int32_t gqla_get_policy(void);
+
+/* Eq. (mqa), line 2:  q_hat_i = [ (W^UK_{j(i)})^T q_i^C ; q_i^R ].
+ *   q_c   [B, s_q, h_q, d_h]   q_r [B, s_q, h_q, d_r]   w_uk [g, r_kv, d_h]
+ *   q_hat [B, s_q, h_q, r_kv + d_r]  (out, same dtype) */
+gqla_status gqla_absorb_q(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q,
+                          const void* q_c, const void* q_r, const void* w_uk, void* q_hat, void* stream);
+
+/* Eq. (mqa), lines 3-5: split-KV attention of every head over the shared latent rows.
+ *   q_hat [B, s_q, h_q, r_kv+d_r];  cache [N, r_kv+d_r] with row stride
+ *   cache_row_stride (elements);  seq_start int64 [B], seqlens int32 [B] (device).
+ *   o_part   [B, S, s_q, h_q, r_kv] fp32 (out),  lse_part [B, S, s_q, h_q] fp32 (out).
+ *   S = num_splits >= 1.  Cache bytes are read once per step whatever s_q is (Sec. 4.2.1). */
+gqla_status gqla_decode_absorb(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                               int32_t num_splits, const void* q_hat, const void* cache,
+                               int64_t cache_row_stride, const int64_t* seq_start, const int32_t* seqlens,
+                               float* o_part, float* lse_part, int32_t* status_word, void* stream);
+
+/* Sec. 3.1: k^C = W^UK c^KV, v^C = W^UV c^KV per group, k^R carried over -- the one-shot
+ * cache expansion that switches from the absorb path to the GQA path.
+ *   cache [N, r_kv+d_r] (row stride cache_row_stride);  w_uk, w_uv [g, r_kv, d_h]
+ *   k_c [N, g, d_h], v [N, g, d_h], k_r [N, d_r]  (out, same dtype; 2 g d_h + d_r per token).
+ *   k_r may be NULL to skip the copy (the GQA path can read k^R from the latent cache's tail). */
+gqla_status gqla_expand_cache(const gqla_dims* dims, gqla_dtype dtype, int64_t N, const void* cache,
+                              int64_t cache_row_stride, const void* w_uk, const void* w_uv, void* k_c, void* v,
+                              void* k_r, void* stream);
+
+/* Eq. (mha): split-KV attention of each head over its group's K_C, V plus the shared k^R.
+ *   q [B, s_q, h_q, d_h+d_r] (= [q^C ; q^R]);  k_c, v [N, g, d_h];  k_r [N, .] with row stride
+ *   k_r_row_stride (elements; d_r for a dense plane, r_kv+d_r when aliasing the latent cache).
+ *   o_part [B, S, s_q, h_q, d_h] fp32 (out),  lse_part [B, S, s_q, h_q] fp32 (out). */
+gqla_status gqla_decode_gqa(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                            int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
+                            int64_t k_r_row_stride, const int64_t* seq_start, const int32_t* seqlens,
+                            float* o_part, float* lse_part, int32_t* status_word, void* stream);
+
+/* Log-sum-exp merge of split partials (split-KV is not in the paper; it is the flash-decoding
+ * reduction of the same softmax):  M = max_k lse_k, w_k = exp(lse_k - M),
+ *   out = sum_k w_k o_k / sum_k w_k,   lse = M + ln sum_k w_k;  all splits empty -> out = 0, lse = -inf.
+ *   o_part [B, S, rows_per_seq, d_out] fp32, lse_part [B, S, rows_per_seq] fp32 (rows_per_seq = s_q*h_q)
+ *   out [B, rows_per_seq, d_out] of out_dtype;  lse [B, rows_per_seq] fp32 or NULL. */
+gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_splits, int32_t d_out,
+                                gqla_dtype out_dtype, const float* o_part, const float* lse_part, void* out,
+                                float* lse, void* stream);
+
+/* Eq. (mqa), line 6:  o_i = W^UV_{j(i)} o_hat_i.
+ *   o_hat [B, s_q, h_q, r_kv]   w_uv [g, r_kv, d_h]   o [B, s_q, h_q, d_h] (out, same dtype) */
+gqla_status gqla_up_proj(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, const void* o_hat,
+                         const void* w_uv, void* o, void* stream);
+
+/* Integer bookkeeping, exported so it can be compared exactly with an independent statement.
+ * HOST pointers. */
+/* Split ranges of a sequence of `seqlen` rows: begin[k], end[k] for k < num_splits. */
+gqla_status gqla_split_plan(int32_t seqlen, int32_t num_splits, int32_t* begin, int32_t* end);
+/* Rows visible to query p of an s_q-token step: max(0, seqlen - (s_q-1-p)). */
+int32_t gqla_visible_limit(int32_t seqlen, int32_t s_q, int32_t p);
+/* 0-indexed group of 0-indexed head: the paper's j(i) = ceil(i/(h_q/g)); -1 on bad input. */
+int32_t gqla_group_of_head(const gqla_dims* dims, int32_t head);
+/* Name of the kernel family the current policy selects for a decode call
+ * ("tcgen05" or "generic"); path: 0 = absorb, 1 = GQA. */
+const char* gqla_kernel_for(const gqla_dims* dims, gqla_dtype dtype, int32_t s_q, int32_t path);
+const char* gqla_status_str(gqla_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GQLA_H_ */

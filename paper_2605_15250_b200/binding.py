@@ -1,0 +1,205 @@
+"""ctypes binding of libgqla.so: one Python function per C entry point, same names.
+
+Argument marshalling only -- every step of the decode path runs in the CUDA
+library.  torch supplies device memory and the current stream.  There is no
+fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_char_p, c_float, c_int32, c_int64, c_void_p
+
+import torch
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libgqla.so")
+
+GQLA_BF16, GQLA_F32 = 0, 1
+POLICY_AUTO, POLICY_GENERIC = 0, 1
+
+
+class GqlaDims(ctypes.Structure):
+    """(h_q, g, d_h, r_kv, d_h^R) of the paper's Sec. 4.2."""
+
+    _fields_ = [("h_q", c_int32), ("g", c_int32), ("d_h", c_int32), ("r_kv", c_int32), ("d_r", c_int32)]
+
+
+class GqlaError(RuntimeError):
+    pass
+
+
+_lib = None
+
+_PROTOTYPES = {
+    "gqla_set_policy": (None, [c_int32]),
+    "gqla_get_policy": (c_int32, []),
+    "gqla_absorb_q": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_decode_absorb": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
+                                     c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_expand_cache": (c_int32, [c_void_p, c_int32, c_int64, c_void_p, c_int64, c_void_p, c_void_p, c_void_p,
+                                    c_void_p, c_void_p, c_void_p]),
+    "gqla_decode_gqa": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
+                                  c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                  c_void_p]),
+    "gqla_combine_splits": (c_int32, [c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
+                                      c_void_p, c_void_p]),
+    "gqla_up_proj": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_split_plan": (c_int32, [c_int32, c_int32, c_void_p, c_void_p]),
+    "gqla_visible_limit": (c_int32, [c_int32, c_int32, c_int32]),
+    "gqla_group_of_head": (c_int32, [c_void_p, c_int32]),
+    "gqla_kernel_for": (c_char_p, [c_void_p, c_int32, c_int32, c_int32]),
+    "gqla_status_str": (c_char_p, [c_int32]),
+}
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libgqla.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise GqlaError(f"{LIB_PATH} not found: build it with `python -m paper_2605_15250_b200.build`")
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _PROTOTYPES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def exported_symbols() -> list[str]:
+    return sorted(_PROTOTYPES)
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        raise GqlaError(f"{what}: {lib().gqla_status_str(code).decode()} (status {code})")
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return GQLA_BF16
+    if t.dtype == torch.float32:
+        return GQLA_F32
+    raise GqlaError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t: torch.Tensor | None) -> int | None:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise GqlaError("expected a CUDA tensor")
+    return t.data_ptr()
+
+
+def _contig(*ts: torch.Tensor) -> None:
+    for t in ts:
+        if t is not None and not t.is_contiguous():
+            raise GqlaError("expected a contiguous tensor")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def make_dims(h_q: int, g: int, d_h: int, r_kv: int, d_r: int) -> GqlaDims:
+    return GqlaDims(h_q, g, d_h, r_kv, d_r)
+
+
+def set_policy(policy: int) -> None:
+    lib().gqla_set_policy(policy)
+
+
+def get_policy() -> int:
+    return lib().gqla_get_policy()
+
+
+def kernel_for(dims: GqlaDims, dtype: torch.dtype, s_q: int, path: str) -> str:
+    code = GQLA_BF16 if dtype == torch.bfloat16 else GQLA_F32
+    return lib().gqla_kernel_for(ctypes.byref(dims), code, s_q, 0 if path == "absorb" else 1).decode()
+
+
+# ------------------------------------------------------------------ the six calls
+
+
+def gqla_absorb_q(dims: GqlaDims, q_c: torch.Tensor, q_r: torch.Tensor, w_uk: torch.Tensor,
+                  q_hat: torch.Tensor) -> None:
+    """q_hat[B,s_q,h_q,r_kv+d_r] = [(W^UK_{j(i)})^T q_c ; q_r]  (Eq. (mqa), line 2)."""
+    _contig(q_c, q_r, w_uk, q_hat)
+    B, s_q = q_c.shape[0], q_c.shape[1]
+    _check(lib().gqla_absorb_q(ctypes.byref(dims), _dtype_code(q_c), B, s_q, _ptr(q_c), _ptr(q_r), _ptr(w_uk),
+                               _ptr(q_hat), _stream()), "gqla_absorb_q")
+
+
+def gqla_decode_absorb(dims: GqlaDims, q_hat: torch.Tensor, cache: torch.Tensor, seq_start: torch.Tensor,
+                       seqlens: torch.Tensor, scale: float, num_splits: int, o_part: torch.Tensor,
+                       lse_part: torch.Tensor, status_word: torch.Tensor | None = None) -> None:
+    """Split-KV absorb-path attention (Eq. (mqa), lines 3-5).  cache is [N, r_kv+d_r] (rows may be strided)."""
+    _contig(q_hat, seq_start, seqlens, o_part, lse_part)
+    assert cache.dim() == 2 and cache.stride(1) == 1
+    assert seq_start.dtype == torch.int64 and seqlens.dtype == torch.int32
+    assert o_part.dtype == torch.float32 and lse_part.dtype == torch.float32
+    B, s_q = q_hat.shape[0], q_hat.shape[1]
+    _check(lib().gqla_decode_absorb(ctypes.byref(dims), _dtype_code(q_hat), B, s_q, scale, num_splits, _ptr(q_hat),
+                                    _ptr(cache), cache.stride(0), _ptr(seq_start), _ptr(seqlens), _ptr(o_part),
+                                    _ptr(lse_part), _ptr(status_word), _stream()), "gqla_decode_absorb")
+
+
+def gqla_expand_cache(dims: GqlaDims, cache: torch.Tensor, w_uk: torch.Tensor, w_uv: torch.Tensor,
+                      k_c: torch.Tensor, v: torch.Tensor, k_r: torch.Tensor | None) -> None:
+    """K_C, V [N,g,d_h] = W^UK c, W^UV c per group; k_R [N,d_r] copied (Sec. 3.1)."""
+    _contig(w_uk, w_uv, k_c, v, k_r)
+    assert cache.dim() == 2 and cache.stride(1) == 1
+    _check(lib().gqla_expand_cache(ctypes.byref(dims), _dtype_code(cache), cache.shape[0], _ptr(cache),
+                                   cache.stride(0), _ptr(w_uk), _ptr(w_uv), _ptr(k_c), _ptr(v), _ptr(k_r),
+                                   _stream()), "gqla_expand_cache")
+
+
+def gqla_decode_gqa(dims: GqlaDims, q: torch.Tensor, k_c: torch.Tensor, v: torch.Tensor, k_r: torch.Tensor,
+                    seq_start: torch.Tensor, seqlens: torch.Tensor, scale: float, num_splits: int,
+                    o_part: torch.Tensor, lse_part: torch.Tensor, status_word: torch.Tensor | None = None) -> None:
+    """Split-KV GQA-path attention (Eq. (mha)).  k_r is [N, d_r] and may be a strided view."""
+    _contig(q, k_c, v, seq_start, seqlens, o_part, lse_part)
+    assert k_r.dim() == 2 and k_r.stride(1) == 1
+    assert seq_start.dtype == torch.int64 and seqlens.dtype == torch.int32
+    assert o_part.dtype == torch.float32 and lse_part.dtype == torch.float32
+    B, s_q = q.shape[0], q.shape[1]
+    _check(lib().gqla_decode_gqa(ctypes.byref(dims), _dtype_code(q), B, s_q, scale, num_splits, _ptr(q), _ptr(k_c),
+                                 _ptr(v), _ptr(k_r), k_r.stride(0), _ptr(seq_start), _ptr(seqlens), _ptr(o_part),
+                                 _ptr(lse_part), _ptr(status_word), _stream()), "gqla_decode_gqa")
+
+
+def gqla_combine_splits(o_part: torch.Tensor, lse_part: torch.Tensor, out: torch.Tensor,
+                        lse: torch.Tensor | None = None) -> None:
+    """LSE merge over the split axis: o_part [B,S,s_q,h_q,D], lse_part [B,S,s_q,h_q] -> out [B,s_q,h_q,D]."""
+    _contig(o_part, lse_part, out, lse)
+    B, S = o_part.shape[0], o_part.shape[1]
+    rows = o_part.shape[2] * o_part.shape[3]
+    _check(lib().gqla_combine_splits(B, rows, S, o_part.shape[-1], _dtype_code(out), _ptr(o_part), _ptr(lse_part),
+                                     _ptr(out), _ptr(lse), _stream()), "gqla_combine_splits")
+
+
+def gqla_up_proj(dims: GqlaDims, o_hat: torch.Tensor, w_uv: torch.Tensor, o: torch.Tensor) -> None:
+    """o[B,s_q,h_q,d_h] = W^UV_{j(i)} o_hat  (Eq. (mqa), line 6)."""
+    _contig(o_hat, w_uv, o)
+    B, s_q = o_hat.shape[0], o_hat.shape[1]
+    _check(lib().gqla_up_proj(ctypes.byref(dims), _dtype_code(o_hat), B, s_q, _ptr(o_hat), _ptr(w_uv), _ptr(o),
+                              _stream()), "gqla_up_proj")
+
+
+# ------------------------------------------------------------------ integer helpers (host)
+
+
+def gqla_split_plan(seqlen: int, num_splits: int) -> list[tuple[int, int]]:
+    begin = (c_int32 * num_splits)()
+    end = (c_int32 * num_splits)()
+    _check(lib().gqla_split_plan(seqlen, num_splits, begin, end), "gqla_split_plan")
+    return [(int(begin[k]), int(end[k])) for k in range(num_splits)]
+
+
+def gqla_visible_limit(seqlen: int, s_q: int, p: int) -> int:
+    return int(lib().gqla_visible_limit(seqlen, s_q, p))
+
+
+def gqla_group_of_head(dims: GqlaDims, head: int) -> int:
+    return int(lib().gqla_group_of_head(ctypes.byref(dims), head))

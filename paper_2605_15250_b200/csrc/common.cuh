@@ -1,0 +1,42 @@
+// Shared device/host helpers for the GQLA kernels (integer bookkeeping, type loads).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gqla {
+
+constexpr int kSplitGranule = 64;
+
+// Split-KV partition: chunk = ceil(ceil(T/S)/64)*64 rows per split.
+__host__ __device__ inline void split_range(int32_t T, int32_t S, int32_t k, int32_t* begin, int32_t* end) {
+    int64_t per = ((int64_t)T + S - 1) / S;
+    int64_t chunk = ((per + kSplitGranule - 1) / kSplitGranule) * kSplitGranule;
+    int64_t b = (int64_t)k * chunk, e = (int64_t)(k + 1) * chunk;
+    *begin = (int32_t)(b < T ? b : T);
+    *end = (int32_t)(e < T ? e : T);
+}
+
+// Rows visible to query p of an s_q-token step (causal sum over s = 1..t, Eqs. (mha)/(mqa)).
+__host__ __device__ inline int32_t visible_limit(int32_t T, int32_t s_q, int32_t p) {
+    int32_t lim = T - (s_q - 1 - p);
+    return lim > 0 ? lim : 0;
+}
+
+__device__ __forceinline__ float ldf(const float* p) { return *p; }
+__device__ __forceinline__ float ldf(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void stf(float* p, float v) { *p = v; }
+__device__ __forceinline__ void stf(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+}  // namespace gqla

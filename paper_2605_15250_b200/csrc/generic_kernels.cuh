@@ -1,0 +1,225 @@
+// Generic SIMT kernels: any (h_q, g, d_h, r_kv, d_r), bf16 or fp32 storage, any s_q.
+// They are the correctness floor for shapes the tensor-core kernels do not cover, and an
+// on-device cross-check for the ones they do.  fp32 arithmetic throughout.
+#pragma once
+#include "common.cuh"
+
+namespace gqla {
+
+struct DecodeArgs {
+    // score(s) = scale * ( q[0:dA] . kA[s] + q[dA:dA+dB] . kB[s] ),  value(s) = v[s][0:dv]
+    const void* q;       // [B, s_q, h_q, dA+dB]
+    const void* kA;      // first key part; row stride kA_stride, + group * kA_gstride
+    const void* kB;      // second key part (shared by all groups); may be null when dB == 0
+    const void* v;       // values; row stride v_stride, + group * v_gstride
+    int64_t kA_stride, kA_gstride, kB_stride, v_stride, v_gstride;
+    int32_t dA, dB, dv;
+    const int64_t* seq_start;
+    const int32_t* seqlens;
+    int32_t B, S, s_q, h_q, hpg;
+    float scale;
+    float* o_part;    // [B, S, s_q, h_q, dv]
+    float* lse_part;  // [B, S, s_q, h_q]
+};
+
+constexpr int kGenericMaxV = 16;  // value columns per lane: dv <= 512
+
+// One warp per (b, split, p, head) row.  Lanes stride over the feature dimension; the
+// online-softmax state (m, l) is warp-uniform; each lane owns dv/32 output columns.
+template <typename E>
+__global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nrows = (int64_t)a.B * a.S * a.s_q * a.h_q;
+    if (row >= nrows) return;
+    const int i = (int)(row % a.h_q);
+    const int p = (int)((row / a.h_q) % a.s_q);
+    const int k = (int)((row / ((int64_t)a.h_q * a.s_q)) % a.S);
+    const int b = (int)(row / ((int64_t)a.h_q * a.s_q * a.S));
+    const int j = i / a.hpg;  // 0-indexed form of j(i) = ceil(i/(h_q/g))
+
+    const int32_t T = a.seqlens[b];
+    int32_t begin, end;
+    split_range(T, a.S, k, &begin, &end);
+    const int32_t lim = visible_limit(T, a.s_q, p);
+    if (end > lim) end = lim;
+
+    const E* q = (const E*)a.q + ((int64_t)(b * a.s_q + p) * a.h_q + i) * (a.dA + a.dB);
+    const int64_t r0 = a.seq_start[b];
+    const E* kA = (const E*)a.kA + (int64_t)j * a.kA_gstride;
+    const E* kB = (const E*)a.kB;
+    const E* vv = (const E*)a.v + (int64_t)j * a.v_gstride;
+
+    float acc[kGenericMaxV];
+#pragma unroll
+    for (int c = 0; c < kGenericMaxV; ++c) acc[c] = 0.f;
+    float m = -INFINITY, l = 0.f;
+
+    for (int32_t s = begin; s < end; ++s) {
+        const E* ka = kA + (r0 + s) * a.kA_stride;
+        float dot = 0.f;
+        for (int d = lane; d < a.dA; d += 32) dot = fmaf(ldf(q + d), ldf(ka + d), dot);
+        if (a.dB > 0) {
+            const E* kb = kB + (r0 + s) * a.kB_stride;
+            for (int d = lane; d < a.dB; d += 32) dot = fmaf(ldf(q + a.dA + d), ldf(kb + d), dot);
+        }
+        const float x = warp_sum(dot) * a.scale;
+        const float m_new = fmaxf(m, x);
+        const float corr = expf(m - m_new);  // exp(-inf) = 0 on the first row
+        const float e = expf(x - m_new);
+        l = l * corr + e;
+        const E* vr = vv + (r0 + s) * a.v_stride;
+#pragma unroll
+        for (int c = 0; c < kGenericMaxV; ++c) {
+            const int d = lane + 32 * c;
+            if (d < a.dv) acc[c] = fmaf(e, ldf(vr + d), acc[c] * corr);
+        }
+        m = m_new;
+    }
+
+    float* o = a.o_part + row * a.dv;
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+    for (int c = 0; c < kGenericMaxV; ++c) {
+        const int d = lane + 32 * c;
+        if (d < a.dv) o[d] = acc[c] * inv;
+    }
+    if (lane == 0) a.lse_part[row] = l > 0.f ? m + logf(l) : -INFINITY;
+}
+
+// Log-sum-exp merge: one block per (b, row).  Weights staged in shared memory.
+template <typename TO>
+__global__ void __launch_bounds__(128) combine_generic_kernel(int32_t B, int32_t rows_per_seq, int32_t S, int32_t d_out,
+                                                              const float* __restrict__ o_part,
+                                                              const float* __restrict__ lse_part, TO* __restrict__ out,
+                                                              float* __restrict__ lse) {
+    extern __shared__ float w[];  // [S]
+    __shared__ float red[4];
+    const int64_t r = blockIdx.x;  // b * rows_per_seq + row
+    const int b = (int)(r / rows_per_seq);
+    const int rr = (int)(r % rows_per_seq);
+    const float* lp = lse_part + ((int64_t)b * S) * rows_per_seq + rr;
+    float mx = -INFINITY;
+    for (int k = threadIdx.x; k < S; k += blockDim.x) mx = fmaxf(mx, lp[(int64_t)k * rows_per_seq]);
+    mx = warp_max(mx);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    mx = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+    __syncthreads();
+    const bool dead = !(mx > -INFINITY);
+    float den = 0.f;
+    for (int k = threadIdx.x; k < S; k += blockDim.x) {
+        const float wk = dead ? 0.f : expf(lp[(int64_t)k * rows_per_seq] - mx);
+        w[k] = wk;
+        den += wk;
+    }
+    den = warp_sum(den);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = den;
+    __syncthreads();
+    den = red[0] + red[1] + red[2] + red[3];
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+    const float* op = o_part + (((int64_t)b * S) * rows_per_seq + rr) * d_out;
+    for (int d = threadIdx.x; d < d_out; d += blockDim.x) {
+        float acc = 0.f;
+        for (int k = 0; k < S; ++k) {
+            const float wk = w[k];
+            if (wk != 0.f) acc = fmaf(wk, op[(int64_t)k * rows_per_seq * d_out + d], acc);
+        }
+        stf(out + r * d_out + d, acc * inv);
+    }
+    if (lse != nullptr && threadIdx.x == 0) lse[r] = dead ? -INFINITY : mx + logf(den);
+}
+
+// q_hat[row, r] = sum_d W_UK[j][r][d] * q_c[row, d]  (r < r_kv);  q_hat[row, r_kv + d] = q_r[row, d].
+// One block per row (b, p, i); the q_c row is staged in shared memory.
+template <typename T>
+__global__ void __launch_bounds__(128) absorb_q_generic_kernel(int32_t h_q, int32_t hpg, int32_t d_h, int32_t r_kv,
+                                                               int32_t d_r, const T* __restrict__ q_c,
+                                                               const T* __restrict__ q_r, const T* __restrict__ w_uk,
+                                                               T* __restrict__ q_hat) {
+    extern __shared__ float qs[];  // [d_h]
+    const int64_t row = blockIdx.x;
+    const int i = (int)(row % h_q);
+    const int j = i / hpg;
+    for (int d = threadIdx.x; d < d_h; d += blockDim.x) qs[d] = ldf(q_c + row * d_h + d);
+    __syncthreads();
+    const T* W = w_uk + (int64_t)j * r_kv * d_h;
+    T* out = q_hat + row * (r_kv + d_r);
+    for (int r = threadIdx.x; r < r_kv; r += blockDim.x) {
+        const T* wr = W + (int64_t)r * d_h;
+        float acc = 0.f;
+        for (int d = 0; d < d_h; ++d) acc = fmaf(ldf(wr + d), qs[d], acc);
+        stf(out + r, acc);
+    }
+    for (int d = threadIdx.x; d < d_r; d += blockDim.x) out[r_kv + d] = q_r[row * d_r + d];
+}
+
+// o[row, d] = sum_r W_UV[j][r][d] * o_hat[row, r].  One block per row; o_hat row staged in smem.
+template <typename T>
+__global__ void __launch_bounds__(128) up_proj_generic_kernel(int32_t h_q, int32_t hpg, int32_t d_h, int32_t r_kv,
+                                                              const T* __restrict__ o_hat, const T* __restrict__ w_uv,
+                                                              T* __restrict__ o) {
+    extern __shared__ float os[];  // [r_kv]
+    const int64_t row = blockIdx.x;
+    const int i = (int)(row % h_q);
+    const int j = i / hpg;
+    for (int r = threadIdx.x; r < r_kv; r += blockDim.x) os[r] = ldf(o_hat + row * r_kv + r);
+    __syncthreads();
+    const T* W = w_uv + (int64_t)j * r_kv * d_h;
+    for (int d = threadIdx.x; d < d_h; d += blockDim.x) {
+        float acc = 0.f;
+        for (int r = 0; r < r_kv; ++r) acc = fmaf(ldf(W + (int64_t)r * d_h + d), os[r], acc);
+        stf(o + row * d_h + d, acc);
+    }
+}
+
+// K_C[n, j, d] = sum_r W_UK[j][r][d] c[n][r],  V likewise with W_UV,  k_R[n] = cache[n, r_kv:].
+// One block per kRows cache rows; the latent rows are staged in shared memory and every thread
+// owns one (j, d) output column of both planes for all staged rows.
+constexpr int kExpandRows = 8;
+template <typename T>
+__global__ void __launch_bounds__(256) expand_cache_generic_kernel(int64_t N, int32_t g, int32_t d_h, int32_t r_kv,
+                                                                   int32_t d_r, const T* __restrict__ cache,
+                                                                   int64_t cache_stride, const T* __restrict__ w_uk,
+                                                                   const T* __restrict__ w_uv, T* __restrict__ k_c,
+                                                                   T* __restrict__ v, T* __restrict__ k_r) {
+    extern __shared__ float cs[];  // [kExpandRows][r_kv]
+    const int64_t n0 = (int64_t)blockIdx.x * kExpandRows;
+    const int nr = (int)((N - n0) < kExpandRows ? (N - n0) : kExpandRows);
+    for (int t = threadIdx.x; t < nr * r_kv; t += blockDim.x) {
+        const int rr = t / r_kv, c = t % r_kv;
+        cs[rr * r_kv + c] = ldf(cache + (n0 + rr) * cache_stride + c);
+    }
+    __syncthreads();
+    const int cols = g * d_h;
+    for (int col = threadIdx.x; col < cols; col += blockDim.x) {
+        const int j = col / d_h, d = col % d_h;
+        const T* wk = w_uk + (int64_t)j * r_kv * d_h + d;
+        const T* wv = w_uv + (int64_t)j * r_kv * d_h + d;
+        float ak[kExpandRows], av[kExpandRows];
+#pragma unroll
+        for (int rr = 0; rr < kExpandRows; ++rr) ak[rr] = av[rr] = 0.f;
+        for (int r = 0; r < r_kv; ++r) {
+            const float a = ldf(wk + (int64_t)r * d_h), b = ldf(wv + (int64_t)r * d_h);
+#pragma unroll
+            for (int rr = 0; rr < kExpandRows; ++rr) {
+                const float c = cs[rr * r_kv + r];
+                ak[rr] = fmaf(a, c, ak[rr]);
+                av[rr] = fmaf(b, c, av[rr]);
+            }
+        }
+#pragma unroll
+        for (int rr = 0; rr < kExpandRows; ++rr)
+            if (rr < nr) {
+                stf(k_c + (n0 + rr) * cols + col, ak[rr]);
+                stf(v + (n0 + rr) * cols + col, av[rr]);
+            }
+    }
+    if (k_r != nullptr)
+        for (int t = threadIdx.x; t < nr * d_r; t += blockDim.x) {
+            const int rr = t / d_r, c = t % d_r;
+            k_r[(n0 + rr) * d_r + c] = cache[(n0 + rr) * cache_stride + r_kv + c];
+        }
+}
+
+}  // namespace gqla

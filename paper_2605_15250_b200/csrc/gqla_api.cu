@@ -1,0 +1,267 @@
+// C-ABI entry points of the GQLA decode library: argument validation, kernel selection, launch.
+#include "../../include/gqla.h"
+
+#include <atomic>
+
+#include "common.cuh"
+#include "generic_kernels.cuh"
+#include "tc_dispatch.cuh"
+
+using namespace gqla;
+
+namespace {
+
+std::atomic<int> g_policy{GQLA_POLICY_AUTO};
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t elem_size(gqla_dtype t) { return t == GQLA_BF16 ? 2 : 4; }
+
+gqla_status check_dims(const gqla_dims* d) {
+    if (d == nullptr) return GQLA_ERR_NULL;
+    if (d->h_q <= 0 || d->g <= 0 || d->d_h <= 0 || d->r_kv <= 0 || d->d_r < 0) return GQLA_ERR_SHAPE;
+    if (d->h_q % d->g != 0) return GQLA_ERR_SHAPE;
+    return GQLA_OK;
+}
+gqla_status check_dtype(gqla_dtype t) { return (t == GQLA_BF16 || t == GQLA_F32) ? GQLA_OK : GQLA_ERR_DTYPE; }
+
+gqla_status launch_status() { return cudaGetLastError() == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA; }
+
+gqla_status launch_decode_generic(gqla_dtype dtype, const DecodeArgs& a, cudaStream_t st) {
+    if (a.dv > 32 * kGenericMaxV) return GQLA_ERR_UNSUPPORTED;
+    const int64_t nrows = (int64_t)a.B * a.S * a.s_q * a.h_q;
+    if (nrows == 0) return GQLA_OK;
+    const int warps = 4;
+    const int64_t blocks = (nrows + warps - 1) / warps;
+    if (blocks > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    if (dtype == GQLA_BF16)
+        decode_generic_kernel<__nv_bfloat16><<<(unsigned)blocks, warps * 32, 0, st>>>(a);
+    else
+        decode_generic_kernel<float><<<(unsigned)blocks, warps * 32, 0, st>>>(a);
+    return launch_status();
+}
+
+}  // namespace
+
+extern "C" {
+
+void gqla_set_policy(gqla_policy p) { g_policy.store(p == GQLA_POLICY_GENERIC ? GQLA_POLICY_GENERIC : GQLA_POLICY_AUTO); }
+int32_t gqla_get_policy(void) { return g_policy.load(); }
+
+const char* gqla_status_str(gqla_status s) {
+    switch (s) {
+        case GQLA_OK: return "ok";
+        case GQLA_ERR_NULL: return "null pointer";
+        case GQLA_ERR_SHAPE: return "bad shape";
+        case GQLA_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
+        case GQLA_ERR_DTYPE: return "unknown dtype";
+        case GQLA_ERR_UNSUPPORTED: return "unsupported configuration";
+        case GQLA_ERR_CUDA: return "CUDA error";
+        case GQLA_ERR_TIMEOUT: return "device wait timed out";
+    }
+    return "unknown status";
+}
+
+gqla_status gqla_split_plan(int32_t seqlen, int32_t num_splits, int32_t* begin, int32_t* end) {
+    if (begin == nullptr || end == nullptr) return GQLA_ERR_NULL;
+    if (seqlen < 0 || num_splits < 1) return GQLA_ERR_SHAPE;
+    for (int32_t k = 0; k < num_splits; ++k) split_range(seqlen, num_splits, k, &begin[k], &end[k]);
+    return GQLA_OK;
+}
+
+int32_t gqla_visible_limit(int32_t seqlen, int32_t s_q, int32_t p) { return visible_limit(seqlen, s_q, p); }
+
+int32_t gqla_group_of_head(const gqla_dims* d, int32_t head) {
+    if (check_dims(d) != GQLA_OK || head < 0 || head >= d->h_q) return -1;
+    return head / (d->h_q / d->g);
+}
+
+const char* gqla_kernel_for(const gqla_dims* d, gqla_dtype dtype, int32_t s_q, int32_t path) {
+    if (check_dims(d) != GQLA_OK) return "invalid";
+    if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, path)) return "tcgen05";
+    return "generic";
+}
+
+gqla_status gqla_absorb_q(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, const void* q_c,
+                          const void* q_r, const void* w_uk, void* q_hat, void* stream) {
+    gqla_status s;
+    if ((s = check_dims(d)) != GQLA_OK) return s;
+    if ((s = check_dtype(dtype)) != GQLA_OK) return s;
+    if (B < 0 || s_q < 1) return GQLA_ERR_SHAPE;
+    if (q_c == nullptr || w_uk == nullptr || q_hat == nullptr || (d->d_r > 0 && q_r == nullptr)) return GQLA_ERR_NULL;
+    if (!aligned16(q_c) || !aligned16(q_r) || !aligned16(w_uk) || !aligned16(q_hat)) return GQLA_ERR_ALIGN;
+    const int64_t rows = (int64_t)B * s_q * d->h_q;
+    if (rows == 0) return GQLA_OK;
+    if (rows > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (g_policy.load() == GQLA_POLICY_AUTO) {
+        s = tc_absorb_q(*d, dtype, B, s_q, q_c, q_r, w_uk, q_hat, st);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
+    const int hpg = d->h_q / d->g;
+    const size_t smem = (size_t)d->d_h * sizeof(float);
+    if (smem > 48 * 1024) return GQLA_ERR_UNSUPPORTED;
+    if (dtype == GQLA_BF16)
+        absorb_q_generic_kernel<__nv_bfloat16><<<(unsigned)rows, 128, smem, st>>>(
+            d->h_q, hpg, d->d_h, d->r_kv, d->d_r, (const __nv_bfloat16*)q_c, (const __nv_bfloat16*)q_r,
+            (const __nv_bfloat16*)w_uk, (__nv_bfloat16*)q_hat);
+    else
+        absorb_q_generic_kernel<float><<<(unsigned)rows, 128, smem, st>>>(
+            d->h_q, hpg, d->d_h, d->r_kv, d->d_r, (const float*)q_c, (const float*)q_r, (const float*)w_uk,
+            (float*)q_hat);
+    return launch_status();
+}
+
+gqla_status gqla_up_proj(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, const void* o_hat,
+                         const void* w_uv, void* o, void* stream) {
+    gqla_status s;
+    if ((s = check_dims(d)) != GQLA_OK) return s;
+    if ((s = check_dtype(dtype)) != GQLA_OK) return s;
+    if (B < 0 || s_q < 1) return GQLA_ERR_SHAPE;
+    if (o_hat == nullptr || w_uv == nullptr || o == nullptr) return GQLA_ERR_NULL;
+    if (!aligned16(o_hat) || !aligned16(w_uv) || !aligned16(o)) return GQLA_ERR_ALIGN;
+    const int64_t rows = (int64_t)B * s_q * d->h_q;
+    if (rows == 0) return GQLA_OK;
+    if (rows > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (g_policy.load() == GQLA_POLICY_AUTO) {
+        s = tc_up_proj(*d, dtype, B, s_q, o_hat, w_uv, o, st);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
+    const int hpg = d->h_q / d->g;
+    const size_t smem = (size_t)d->r_kv * sizeof(float);
+    if (smem > 48 * 1024) return GQLA_ERR_UNSUPPORTED;
+    if (dtype == GQLA_BF16)
+        up_proj_generic_kernel<__nv_bfloat16><<<(unsigned)rows, 128, smem, st>>>(
+            d->h_q, hpg, d->d_h, d->r_kv, (const __nv_bfloat16*)o_hat, (const __nv_bfloat16*)w_uv, (__nv_bfloat16*)o);
+    else
+        up_proj_generic_kernel<float><<<(unsigned)rows, 128, smem, st>>>(d->h_q, hpg, d->d_h, d->r_kv,
+                                                                        (const float*)o_hat, (const float*)w_uv,
+                                                                        (float*)o);
+    return launch_status();
+}
+
+gqla_status gqla_expand_cache(const gqla_dims* d, gqla_dtype dtype, int64_t N, const void* cache,
+                              int64_t cache_row_stride, const void* w_uk, const void* w_uv, void* k_c, void* v,
+                              void* k_r, void* stream) {
+    gqla_status s;
+    if ((s = check_dims(d)) != GQLA_OK) return s;
+    if ((s = check_dtype(dtype)) != GQLA_OK) return s;
+    if (N < 0 || cache_row_stride < d->r_kv + d->d_r) return GQLA_ERR_SHAPE;
+    if (N == 0) return GQLA_OK;
+    if (cache == nullptr || w_uk == nullptr || w_uv == nullptr || k_c == nullptr || v == nullptr) return GQLA_ERR_NULL;
+    if (!aligned16(cache) || !aligned16(w_uk) || !aligned16(w_uv) || !aligned16(k_c) || !aligned16(v) ||
+        !aligned16(k_r))
+        return GQLA_ERR_ALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (g_policy.load() == GQLA_POLICY_AUTO) {
+        s = tc_expand_cache(*d, dtype, N, cache, cache_row_stride, w_uk, w_uv, k_c, v, k_r, st);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
+    const size_t smem = (size_t)kExpandRows * d->r_kv * sizeof(float);
+    if (smem > 48 * 1024) return GQLA_ERR_UNSUPPORTED;
+    const int64_t blocks = (N + kExpandRows - 1) / kExpandRows;
+    if (blocks > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    if (dtype == GQLA_BF16)
+        expand_cache_generic_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, smem, st>>>(
+            N, d->g, d->d_h, d->r_kv, d->d_r, (const __nv_bfloat16*)cache, cache_row_stride,
+            (const __nv_bfloat16*)w_uk, (const __nv_bfloat16*)w_uv, (__nv_bfloat16*)k_c, (__nv_bfloat16*)v,
+            (__nv_bfloat16*)k_r);
+    else
+        expand_cache_generic_kernel<float><<<(unsigned)blocks, 256, smem, st>>>(
+            N, d->g, d->d_h, d->r_kv, d->d_r, (const float*)cache, cache_row_stride, (const float*)w_uk,
+            (const float*)w_uv, (float*)k_c, (float*)v, (float*)k_r);
+    return launch_status();
+}
+
+static gqla_status check_decode_common(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, int32_t S,
+                                       const int64_t* seq_start, const int32_t* seqlens, const float* o_part,
+                                       const float* lse_part) {
+    gqla_status s;
+    if ((s = check_dims(d)) != GQLA_OK) return s;
+    if ((s = check_dtype(dtype)) != GQLA_OK) return s;
+    if (B < 0 || s_q < 1 || S < 1) return GQLA_ERR_SHAPE;
+    if (B == 0) return GQLA_OK;
+    if (seq_start == nullptr || seqlens == nullptr || o_part == nullptr || lse_part == nullptr) return GQLA_ERR_NULL;
+    if (!aligned16(o_part)) return GQLA_ERR_ALIGN;
+    return GQLA_OK;
+}
+
+gqla_status gqla_decode_absorb(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                               int32_t num_splits, const void* q_hat, const void* cache, int64_t cache_row_stride,
+                               const int64_t* seq_start, const int32_t* seqlens, float* o_part, float* lse_part,
+                               int32_t* status_word, void* stream) {
+    gqla_status s = check_decode_common(d, dtype, B, s_q, num_splits, seq_start, seqlens, o_part, lse_part);
+    if (s != GQLA_OK) return s;
+    if (B == 0) return GQLA_OK;
+    if (q_hat == nullptr || cache == nullptr) return GQLA_ERR_NULL;
+    if (!aligned16(q_hat) || !aligned16(cache)) return GQLA_ERR_ALIGN;
+    if (cache_row_stride < d->r_kv + d->d_r) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, 0)) {
+        s = tc_decode_absorb(*d, B, s_q, scale, num_splits, q_hat, cache, cache_row_stride, seq_start, seqlens,
+                             o_part, lse_part, status_word, st);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
+    DecodeArgs a{};
+    a.q = q_hat;
+    a.kA = cache; a.kA_stride = cache_row_stride; a.kA_gstride = 0; a.dA = d->r_kv + d->d_r;
+    a.kB = nullptr; a.kB_stride = 0; a.dB = 0;
+    a.v = cache; a.v_stride = cache_row_stride; a.v_gstride = 0; a.dv = d->r_kv;
+    a.seq_start = seq_start; a.seqlens = seqlens;
+    a.B = B; a.S = num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
+    a.scale = scale; a.o_part = o_part; a.lse_part = lse_part;
+    return launch_decode_generic(dtype, a, st);
+}
+
+gqla_status gqla_decode_gqa(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                            int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
+                            int64_t k_r_row_stride, const int64_t* seq_start, const int32_t* seqlens, float* o_part,
+                            float* lse_part, int32_t* status_word, void* stream) {
+    gqla_status s = check_decode_common(d, dtype, B, s_q, num_splits, seq_start, seqlens, o_part, lse_part);
+    if (s != GQLA_OK) return s;
+    if (B == 0) return GQLA_OK;
+    if (q == nullptr || k_c == nullptr || v == nullptr || (d->d_r > 0 && k_r == nullptr)) return GQLA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k_c) || !aligned16(v) || !aligned16(k_r)) return GQLA_ERR_ALIGN;
+    if (d->d_r > 0 && k_r_row_stride < d->d_r) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, 1)) {
+        s = tc_decode_gqa(*d, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, seq_start, seqlens, o_part,
+                          lse_part, status_word, st);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
+    DecodeArgs a{};
+    a.q = q;
+    a.kA = k_c; a.kA_stride = (int64_t)d->g * d->d_h; a.kA_gstride = d->d_h; a.dA = d->d_h;
+    a.kB = k_r; a.kB_stride = k_r_row_stride; a.dB = d->d_r;
+    a.v = v; a.v_stride = (int64_t)d->g * d->d_h; a.v_gstride = d->d_h; a.dv = d->d_h;
+    a.seq_start = seq_start; a.seqlens = seqlens;
+    a.B = B; a.S = num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
+    a.scale = scale; a.o_part = o_part; a.lse_part = lse_part;
+    return launch_decode_generic(dtype, a, st);
+}
+
+gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_splits, int32_t d_out,
+                                gqla_dtype out_dtype, const float* o_part, const float* lse_part, void* out,
+                                float* lse, void* stream) {
+    gqla_status s;
+    if ((s = check_dtype(out_dtype)) != GQLA_OK) return s;
+    if (B < 0 || rows_per_seq < 1 || num_splits < 1 || d_out < 1) return GQLA_ERR_SHAPE;
+    if (B == 0) return GQLA_OK;
+    if (o_part == nullptr || lse_part == nullptr || out == nullptr) return GQLA_ERR_NULL;
+    if (!aligned16(o_part) || !aligned16(out)) return GQLA_ERR_ALIGN;
+    const int64_t rows = (int64_t)B * rows_per_seq;
+    if (rows > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    const size_t smem = (size_t)num_splits * sizeof(float);
+    if (smem > 48 * 1024) return GQLA_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (out_dtype == GQLA_BF16)
+        combine_generic_kernel<__nv_bfloat16><<<(unsigned)rows, 128, smem, st>>>(B, rows_per_seq, num_splits, d_out,
+                                                                                 o_part, lse_part,
+                                                                                 (__nv_bfloat16*)out, lse);
+    else
+        combine_generic_kernel<float><<<(unsigned)rows, 128, smem, st>>>(B, rows_per_seq, num_splits, d_out, o_part,
+                                                                         lse_part, (float*)out, lse);
+    return launch_status();
+}
+
+}  // extern "C"

@@ -1,0 +1,89 @@
+"""Decode-step driver: owns the device buffers of one GQLA attention layer and chains
+the library calls of each path.  No arithmetic happens here -- torch only allocates."""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+class GqlaDecoder:
+    """One layer's decode attention over a resident KV cache, through either path.
+
+    Absorb path (Eq. (mqa)):  absorb_q -> decode_absorb -> combine_splits -> up_proj
+    GQA path    (Eq. (mha)):  decode_gqa -> combine_splits   (after a one-shot expand_cache)
+    """
+
+    def __init__(self, h_q: int, g: int, d_h: int, r_kv: int, d_r: int, w_uk: torch.Tensor, w_uv: torch.Tensor,
+                 cache: torch.Tensor, seq_start: torch.Tensor, seqlens: torch.Tensor, scale: float):
+        assert cache.is_cuda and w_uk.is_cuda and w_uv.is_cuda
+        self.dims = B.make_dims(h_q, g, d_h, r_kv, d_r)
+        self.h_q, self.g, self.d_h, self.r_kv, self.d_r = h_q, g, d_h, r_kv, d_r
+        self.w_uk, self.w_uv, self.cache = w_uk, w_uv, cache
+        self.seq_start, self.seqlens = seq_start, seqlens
+        self.scale = float(scale)
+        self.dtype = cache.dtype
+        self.device = cache.device
+        self.batch = int(seqlens.shape[0])
+        self.k_c = self.v = self.k_r = None
+        self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
+        self._buf = {}
+
+    def _get(self, name: str, shape, dtype) -> torch.Tensor:
+        key = (name, tuple(shape), dtype)
+        t = self._buf.get(key)
+        if t is None:
+            t = torch.empty(shape, dtype=dtype, device=self.device)
+            self._buf[key] = t
+        return t
+
+    # ---- one-shot cache expansion (Sec. 3.1) ----
+    def expand_cache(self, alias_k_r: bool = True) -> None:
+        """Builds K_C, V [N,g,d_h].  With alias_k_r the shared RoPE key is read in place from
+        the latent cache's last d_r columns (the paper's "no-op view"); otherwise it is copied."""
+        N = self.cache.shape[0]
+        self.k_c = torch.empty((N, self.g, self.d_h), dtype=self.dtype, device=self.device)
+        self.v = torch.empty((N, self.g, self.d_h), dtype=self.dtype, device=self.device)
+        if alias_k_r:
+            B.gqla_expand_cache(self.dims, self.cache, self.w_uk, self.w_uv, self.k_c, self.v, None)
+            self.k_r = self.cache[:, self.r_kv:]
+        else:
+            self.k_r = torch.empty((N, self.d_r), dtype=self.dtype, device=self.device)
+            B.gqla_expand_cache(self.dims, self.cache, self.w_uk, self.w_uv, self.k_c, self.v, self.k_r)
+
+    # ---- absorb path ----
+    def absorb_step(self, q_c: torch.Tensor, q_r: torch.Tensor, num_splits: int = 1, want_lse: bool = False):
+        Bn, s_q = q_c.shape[0], q_c.shape[1]
+        q_hat = self._get("q_hat", (Bn, s_q, self.h_q, self.r_kv + self.d_r), self.dtype)
+        o_part = self._get("o_part_a", (Bn, num_splits, s_q, self.h_q, self.r_kv), torch.float32)
+        lse_part = self._get("lse_part_a", (Bn, num_splits, s_q, self.h_q), torch.float32)
+        o_hat = self._get("o_hat", (Bn, s_q, self.h_q, self.r_kv), self.dtype)
+        lse = self._get("lse_a", (Bn, s_q, self.h_q), torch.float32) if want_lse else None
+        o = self._get("o_a", (Bn, s_q, self.h_q, self.d_h), self.dtype)
+        B.gqla_absorb_q(self.dims, q_c, q_r, self.w_uk, q_hat)
+        B.gqla_decode_absorb(self.dims, q_hat, self.cache, self.seq_start, self.seqlens, self.scale, num_splits,
+                             o_part, lse_part, self.status)
+        B.gqla_combine_splits(o_part, lse_part, o_hat, lse)
+        B.gqla_up_proj(self.dims, o_hat, self.w_uv, o)
+        return (o, lse) if want_lse else o
+
+    # ---- GQA path ----
+    def gqa_step(self, q: torch.Tensor, num_splits: int = 1, want_lse: bool = False):
+        """q is [B, s_q, h_q, d_h+d_r] = [q^C ; q^R]."""
+        if self.k_c is None:
+            raise B.GqlaError("expand_cache() must run before the GQA path")
+        Bn, s_q = q.shape[0], q.shape[1]
+        o_part = self._get("o_part_g", (Bn, num_splits, s_q, self.h_q, self.d_h), torch.float32)
+        lse_part = self._get("lse_part_g", (Bn, num_splits, s_q, self.h_q), torch.float32)
+        lse = self._get("lse_g", (Bn, s_q, self.h_q), torch.float32) if want_lse else None
+        o = self._get("o_g", (Bn, s_q, self.h_q, self.d_h), self.dtype)
+        B.gqla_decode_gqa(self.dims, q, self.k_c, self.v, self.k_r, self.seq_start, self.seqlens, self.scale,
+                          num_splits, o_part, lse_part, self.status)
+        B.gqla_combine_splits(o_part, lse_part, o, lse)
+        return (o, lse) if want_lse else o
+
+    def check_status(self) -> None:
+        """Synchronises and raises if a bounded device wait expired in any earlier call."""
+        code = int(self.status.item())
+        if code != 0:
+            raise B.GqlaError(f"device status word = {code} (a bounded wait expired)")

@@ -1,0 +1,176 @@
+"""GPU parity: every C-ABI call against the fp64 oracle on the same seeded inputs.
+
+Bar: bit-exact integer bookkeeping (checked on the host), and for floating point
+max|err| <= 1e-2 * max|ref| + 1e-3 (bf16 inputs, fp32 accumulation)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_15250_b200 import binding as B
+from paper_2605_15250_b200 import build as gbuild
+from paper_2605_15250_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    gbuild.build()
+    assert torch.cuda.is_available()
+    B.lib()
+    yield
+    B.set_policy(B.POLICY_AUTO)
+
+
+@pytest.fixture(params=["auto", "generic"])
+def policy(request):
+    B.set_policy(B.POLICY_AUTO if request.param == "auto" else B.POLICY_GENERIC)
+    yield request.param
+    B.set_policy(B.POLICY_AUTO)
+
+
+CANON = dict(h_q=128, g=8, d_h=128, r_kv=512, d_r=64)
+LLAMA = dict(h_q=32, g=8, d_h=128, r_kv=512, d_r=64)
+
+
+def _wl(name, batch, s_q, seed, dtype="bf16", **dims):
+    return synth.Workload(name, batch=batch, s_q=s_q, dtype=dtype, seed=seed, **dims)
+
+
+def test_c0_tiny_fp32(policy):
+    """BASELINE config 0: B=1, h_q=8, g=2, d_h=16, r_kv=32, d_r=8, T=64, fp32."""
+    from tests.parity_util import end_to_end, stagewise
+    w = synth.WORKLOADS["C0"]
+    errs = stagewise(w, None, 1)
+    errs.update(end_to_end(w, None, 1))
+    # fp32 storage: far inside the bf16 tolerance
+    assert max(errs.values()) < 1e-4
+    errs = stagewise(w.with_(dtype="bf16"), None, 2)
+
+
+@pytest.mark.parametrize("s_q", [1, 2, 3])
+@pytest.mark.parametrize("S", [1, 3])
+def test_odd_shapes_generic(s_q, S):
+    """Shapes no specialised kernel covers (h_q/g = 1 and 3, odd dims): generic kernels."""
+    from tests.parity_util import end_to_end, stagewise
+    B.set_policy(B.POLICY_AUTO)
+    w = _wl("odd", 5, s_q, 77, dtype="f32", h_q=6, g=2, d_h=20, r_kv=36, d_r=12)
+    seqlens = np.array([0, 1, 2, 65, 200], dtype=np.int32)
+    stagewise(w, seqlens, S)
+    end_to_end(w, seqlens, S)
+    w = _wl("odd2", 3, s_q, 78, dtype="bf16", h_q=4, g=4, d_h=24, r_kv=40, d_r=8)
+    stagewise(w, np.array([130, 64, 63], dtype=np.int32), S)
+
+
+@pytest.mark.parametrize("s_q", [1, 2])
+@pytest.mark.parametrize("S,q_gain", [(1, 1.0), (4, 4.0), (9, 4.0)])
+def test_canonical_dims_ragged_stagewise(policy, s_q, S, q_gain):
+    """Canonical dims, several tiles and ragged tails, empty sequences and T < s_q."""
+    from tests.parity_util import stagewise
+    w = _wl("canon", 8, s_q, 101, **CANON)
+    seqlens = np.array([1, 0, 63, 64, 65, 1000, 129, 2050], dtype=np.int32)
+    stagewise(w, seqlens, S, q_gain)
+
+
+@pytest.mark.parametrize("s_q", [1, 2])
+def test_llama_dims_ragged_stagewise(policy, s_q):
+    from tests.parity_util import stagewise
+    w = _wl("llama", 6, s_q, 102, **LLAMA)
+    seqlens = np.array([513, 2, 700, 64, 3000, 127], dtype=np.int32)
+    stagewise(w, seqlens, 5, 4.0)
+
+
+@pytest.mark.parametrize("dims", [CANON, LLAMA])
+@pytest.mark.parametrize("s_q,S", [(1, 1), (2, 4)])
+def test_end_to_end_mid(policy, dims, s_q, S):
+    from tests.parity_util import end_to_end
+    w = _wl("mid", 5, s_q, 103, **dims)
+    seqlens = np.array([777, 64, 1, 2049, 300], dtype=np.int32)
+    end_to_end(w, seqlens, S, q_gain=4.0)
+    end_to_end(w, seqlens, S, q_gain=1.0, alias_k_r=False)
+
+
+def test_two_gpu_paths_agree_with_each_other():
+    """Same weights, same latent: the two paths' GPU outputs differ by at most twice the
+    tolerance (each is within it of the same oracle value)."""
+    from tests.parity_util import ABS, REL
+    from paper_2605_15250_b200.decoder import GqlaDecoder
+    w = _wl("agree", 4, 2, 104, **CANON)
+    x = synth.make_inputs(w, seqlens=np.array([500, 1200, 64, 333], dtype=np.int32), q_gain=4.0)
+    dec = GqlaDecoder(w.h_q, w.g, w.d_h, w.r_kv, w.d_r, x["w_uk"].cuda(), x["w_uv"].cuda(), x["cache"].cuda(),
+                      x["seq_start"].cuda(), x["seqlens"].cuda(), w.scale)
+    a = dec.absorb_step(x["q_c"].cuda(), x["q_r"].cuda(), 2).float().cpu()
+    dec.expand_cache()
+    gq = dec.gqa_step(torch.cat([x["q_c"], x["q_r"]], -1).contiguous().cuda(), 2).float().cpu()
+    assert (a - gq).abs().max().item() <= 2 * (REL * a.abs().max().item() + ABS)
+
+
+def test_determinism_run_to_run():
+    from paper_2605_15250_b200.decoder import GqlaDecoder
+    w = _wl("det", 4, 2, 105, **CANON)
+    x = synth.make_inputs(w, seqlens=np.array([900, 4000, 65, 2048], dtype=np.int32))
+    dec = GqlaDecoder(w.h_q, w.g, w.d_h, w.r_kv, w.d_r, x["w_uk"].cuda(), x["w_uv"].cuda(), x["cache"].cuda(),
+                      x["seq_start"].cuda(), x["seqlens"].cuda(), w.scale)
+    qc, qr = x["q_c"].cuda(), x["q_r"].cuda()
+    a1 = dec.absorb_step(qc, qr, 4).clone()
+    a2 = dec.absorb_step(qc, qr, 4).clone()
+    assert torch.equal(a1, a2)
+
+
+# ------------------------------------------------------------------ BASELINE configs at full size
+
+
+def test_c1_full_absorb():
+    """Config 1: h_q=128, g=8, B=64, T=4096, s_q=1, absorb path (as the benchmark launches it)."""
+    from tests.parity_util import end_to_end
+    end_to_end(synth.WORKLOADS["C1"], None, 1, paths=("absorb",))
+
+
+def test_c2_full_gqa_mtp():
+    """Config 2: same weights and latent, expanded cache, s_q=2 causal.  The oracle runs a sample
+    of sequences (all heads, both draft positions)."""
+    from tests.parity_util import end_to_end
+    end_to_end(synth.WORKLOADS["C2"], None, 1, sample_seqs=(0, 17, 63), paths=("gqa",))
+    end_to_end(synth.WORKLOADS["C2"], None, 1, q_gain=4.0, sample_seqs=(5,), paths=("gqa", "absorb"))
+
+
+@pytest.mark.parametrize("s_q", [1, 2])
+def test_c3_full_ragged(s_q):
+    """Config 3: LLaMA-3-8B shape, B=128, seqlens uniform in [512, 32768]; both paths.
+    The oracle runs the shortest, the longest and two more sequences."""
+    from tests.parity_util import end_to_end
+    w = synth.WORKLOADS["C3"].with_(s_q=s_q)
+    sl = synth.make_seqlens(w)
+    assert sl.min() >= 512 and sl.max() <= 32768
+    sample = sorted({int(sl.argmin()), int(sl.argmax()), 3, 100})
+    end_to_end(w, None, 4, q_gain=4.0, sample_seqs=sample)
+
+
+@pytest.mark.parametrize("s_q", [1, 2])
+def test_c4_long_context_split_sweep(s_q):
+    """Config 4: B=4, T=131072, split count swept over {1, 8, 32, 128} with the LSE combine."""
+    from tests.parity_util import assert_close, dims_of
+    from oracle import gqla_oracle as O
+    from paper_2605_15250_b200.decoder import GqlaDecoder
+    w = synth.WORKLOADS["C4"].with_(s_q=s_q)
+    od, _ = dims_of(w)
+    x = synth.make_inputs(w, q_gain=4.0)
+    dec = GqlaDecoder(w.h_q, w.g, w.d_h, w.r_kv, w.d_r, x["w_uk"].cuda(), x["w_uv"].cuda(), x["cache"].cuda(),
+                      x["seq_start"].cuda(), x["seqlens"].cuda(), w.scale)
+    dec.expand_cache()
+    b = 2  # the oracle runs one of the four sequences
+    T = int(x["seqlens"][b])
+    s0 = int(x["seq_start"][b])
+    rows = synth.to_f64(x["cache"][s0:s0 + T])
+    args = (od, synth.to_f64(x["q_c"][b:b + 1]), synth.to_f64(x["q_r"][b:b + 1]), synth.to_f64(x["w_uk"]),
+            synth.to_f64(x["w_uv"]), rows, np.zeros(1, dtype=np.int64), np.array([T], dtype=np.int32), s_q, w.scale)
+    ref_a = O.absorb_path(*args)
+    ref_g = O.gqa_path(*args)
+    q = torch.cat([x["q_c"], x["q_r"]], -1).contiguous().cuda()
+    qc, qr = x["q_c"].cuda(), x["q_r"].cuda()
+    for S in (1, 8, 32, 128):
+        a = dec.absorb_step(qc, qr, S).float().cpu().numpy()[b:b + 1]
+        assert_close(a, ref_a, f"C4 absorb S={S}")
+        gq = dec.gqa_step(q, S).float().cpu().numpy()[b:b + 1]
+        assert_close(gq, ref_g, f"C4 gqa S={S}")
+    dec.check_status()
