@@ -4,8 +4,19 @@
 #pragma once
 #include "../../include/gqla.h"
 #include "common.cuh"
+#include "tc_gemm.cuh"
 
 namespace gqla {
+
+inline bool stride_ok(int64_t elems) { return (elems * 2) % 16 == 0; }
+
+// Shapes the grouped tcgen05 GEMMs cover: bf16, d_h = 128, r_kv a multiple of 256, d_r a multiple
+// of 8, heads-per-group dividing 128.
+inline bool tc_gemm_covers(const gqla_dims& d, gqla_dtype dtype) {
+    const int hpg = d.h_q / d.g;
+    return dtype == GQLA_BF16 && d.d_h == 128 && d.r_kv % 256 == 0 && d.r_kv <= 4096 && d.d_r % 8 == 0 &&
+           hpg <= 128 && 128 % hpg == 0;
+}
 
 // path: 0 = absorb, 1 = GQA
 inline bool tc_covers(const gqla_dims& d, gqla_dtype dtype, int32_t s_q, int32_t path) {
@@ -13,18 +24,97 @@ inline bool tc_covers(const gqla_dims& d, gqla_dtype dtype, int32_t s_q, int32_t
     return false;
 }
 
-inline gqla_status tc_absorb_q(const gqla_dims&, gqla_dtype, int32_t, int32_t, const void*, const void*, const void*,
-                               void*, cudaStream_t) {
-    return GQLA_ERR_UNSUPPORTED;
+inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t N, const void* cache,
+                                   int64_t cache_row_stride, const void* w_uk, const void* w_uv, void* k_c, void* v,
+                                   void* k_r, cudaStream_t st) {
+    if (!tc_gemm_covers(d, dtype) || !stride_ok(cache_row_stride)) return GQLA_ERR_UNSUPPORTED;
+    const int64_t m_tiles = (N + 127) / 128;
+    if (m_tiles * 2 * d.g > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
+    CUtensorMap tmA, tmK, tmV;
+    {
+        const uint64_t dims[2] = {(uint64_t)d.r_kv, (uint64_t)N};
+        const uint64_t str[1] = {(uint64_t)cache_row_stride * 2};
+        const uint32_t box[2] = {64, 128};
+        if (!tc::make_tmap_bf16(&tmA, cache, 2, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)d.d_h, (uint64_t)d.g * d.r_kv};
+        const uint64_t str[1] = {(uint64_t)d.d_h * 2};
+        const uint32_t box[2] = {64, 64};
+        if (!tc::make_tmap_bf16(&tmK, w_uk, 2, dims, str, box)) return GQLA_ERR_CUDA;
+        if (!tc::make_tmap_bf16(&tmV, w_uv, 2, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    tc::GemmParams p{};
+    p.k_blocks = d.r_kv / 64;
+    p.m_total = N;
+    p.h_q = d.h_q; p.g = d.g; p.hpg = d.h_q / d.g; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
+    p.out0 = k_c; p.out1 = v; p.aux_in = cache; p.aux_out = k_r; p.aux_stride = cache_row_stride;
+    p.status = nullptr;
+    cudaError_t e = tc::gemm_launch<tc::kGemmExpand, 128, true>(p, tmA, tmK, tmV, dim3((unsigned)(m_tiles * 2 * d.g)), st);
+    return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
 }
-inline gqla_status tc_up_proj(const gqla_dims&, gqla_dtype, int32_t, int32_t, const void*, const void*, void*,
-                              cudaStream_t) {
-    return GQLA_ERR_UNSUPPORTED;
+
+// 4-D view of a [B*s_q, h_q, feat] activation: (feat, head-in-group, group, position).
+inline bool make_grouped_act_map(CUtensorMap* m, const void* base, const gqla_dims& d, int feat, int64_t positions) {
+    const int hpg = d.h_q / d.g;
+    const uint64_t dims[4] = {(uint64_t)feat, (uint64_t)hpg, (uint64_t)d.g, (uint64_t)positions};
+    const uint64_t str[3] = {(uint64_t)feat * 2, (uint64_t)hpg * feat * 2, (uint64_t)d.h_q * feat * 2};
+    const uint32_t box[4] = {64, (uint32_t)hpg, 1, (uint32_t)(128 / hpg)};
+    return tc::make_tmap_bf16(m, base, 4, dims, str, box);
 }
-inline gqla_status tc_expand_cache(const gqla_dims&, gqla_dtype, int64_t, const void*, int64_t, const void*,
-                                   const void*, void*, void*, void*, cudaStream_t) {
-    return GQLA_ERR_UNSUPPORTED;
+
+inline gqla_status tc_absorb_q(const gqla_dims& d, gqla_dtype dtype, int32_t B, int32_t s_q, const void* q_c,
+                               const void* q_r, const void* w_uk, void* q_hat, cudaStream_t st) {
+    if (!tc_gemm_covers(d, dtype)) return GQLA_ERR_UNSUPPORTED;
+    const int hpg = d.h_q / d.g;
+    const int64_t positions = (int64_t)B * s_q;
+    const int64_t m_tiles = (positions + 128 / hpg - 1) / (128 / hpg);
+    if (m_tiles > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
+    CUtensorMap tmA, tmB;
+    if (!make_grouped_act_map(&tmA, q_c, d, d.d_h, positions)) return GQLA_ERR_CUDA;
+    {
+        // W_UK[j] as a K-major B operand: rows = (j, r), columns = d (contraction)
+        const uint64_t dims[2] = {(uint64_t)d.d_h, (uint64_t)d.g * d.r_kv};
+        const uint64_t str[1] = {(uint64_t)d.d_h * 2};
+        const uint32_t box[2] = {64, 256};
+        if (!tc::make_tmap_bf16(&tmB, w_uk, 2, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    tc::GemmParams p{};
+    p.k_blocks = d.d_h / 64;
+    p.m_total = positions;
+    p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
+    p.out0 = q_hat; p.aux_in = q_r;
+    cudaError_t e = tc::gemm_launch<tc::kGemmAbsorbQ, 256, false>(
+        p, tmA, tmB, tmB, dim3((unsigned)m_tiles, (unsigned)d.g, (unsigned)(d.r_kv / 256)), st);
+    return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
 }
+
+inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, int32_t s_q, const void* o_hat,
+                              const void* w_uv, void* o, cudaStream_t st) {
+    if (!tc_gemm_covers(d, dtype)) return GQLA_ERR_UNSUPPORTED;
+    const int hpg = d.h_q / d.g;
+    const int64_t positions = (int64_t)B * s_q;
+    const int64_t m_tiles = (positions + 128 / hpg - 1) / (128 / hpg);
+    if (m_tiles > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
+    CUtensorMap tmA, tmB;
+    if (!make_grouped_act_map(&tmA, o_hat, d, d.r_kv, positions)) return GQLA_ERR_CUDA;
+    {
+        // W_UV[j] as an MN-major B operand: rows = (j, r) (contraction), columns = d (output)
+        const uint64_t dims[2] = {(uint64_t)d.d_h, (uint64_t)d.g * d.r_kv};
+        const uint64_t str[1] = {(uint64_t)d.d_h * 2};
+        const uint32_t box[2] = {64, 64};
+        if (!tc::make_tmap_bf16(&tmB, w_uv, 2, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    tc::GemmParams p{};
+    p.k_blocks = d.r_kv / 64;
+    p.m_total = positions;
+    p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
+    p.out0 = o;
+    cudaError_t e =
+        tc::gemm_launch<tc::kGemmUpProj, 128, true>(p, tmA, tmB, tmB, dim3((unsigned)m_tiles, (unsigned)d.g, 1), st);
+    return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
+}
+
 inline gqla_status tc_decode_absorb(const gqla_dims&, int32_t, int32_t, float, int32_t, const void*, const void*,
                                     int64_t, const int64_t*, const int32_t*, float*, float*, int32_t*, cudaStream_t) {
     return GQLA_ERR_UNSUPPORTED;

@@ -1,0 +1,222 @@
+// tcgen05 GEMM kernels for the three plain contractions of the path:
+//   expand_cache :  K_C / V [n, j, :] = sum_r c[n, r] W[j][r][:]          (Sec. 3.1)
+//   absorb_q     :  q_hat[row, r]     = sum_d q_c[row, d] W_UK[j][r][d]   (Eq. (mqa), line 2)
+//   up_proj      :  o[row, d]         = sum_r o_hat[row, r] W_UV[j][r][d] (Eq. (mqa), line 6)
+// One CTA computes a 128 x BN output tile: warp 0 streams A/B tiles with TMA through a ring of
+// shared-memory stages, warp 1 issues tcgen05.mma into a TMEM accumulator, warps 2-5 read the
+// accumulator back (tcgen05.ld) and store bf16 rows.
+#pragma once
+#include "tc_common.cuh"
+
+namespace gqla {
+namespace tc {
+
+enum GemmMode { kGemmExpand = 0, kGemmAbsorbQ = 1, kGemmUpProj = 2 };
+
+struct GemmParams {
+    int32_t k_blocks;   // K / 64
+    int64_t m_total;    // expand: cache rows N;  others: B * s_q (query positions)
+    int32_t h_q, g, hpg, d_h, r_kv, d_r;
+    void* out0;         // expand: k_c;  absorb_q: q_hat;  up_proj: o
+    void* out1;         // expand: v
+    const void* aux_in; // absorb_q: q_r (copied into q_hat's tail);  expand: cache (for the k_R copy)
+    void* aux_out;      // expand: k_r plane or null
+    int64_t aux_stride; // expand: cache row stride (elements)
+    int32_t* status;
+};
+
+template <int BN, bool B_MN>
+struct GemmSmem {
+    static constexpr int kStages = 4;
+    static constexpr int kABytes = 128 * 128;  // 128 rows x 64 bf16
+    static constexpr int kBBytes = BN * 128;   // K-major: BN rows x 64 k;  MN-major: (BN/64) boxes of 64 k-rows x 64 n
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kTotal = kStages * kStageBytes + 1024 /*align slack*/ + 256 /*barriers*/;
+};
+
+template <int MODE, int BN, bool B_MN>
+__global__ void __launch_bounds__(192, 1)
+gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+               const __grid_constant__ CUtensorMap tmB1) {
+    using L = GemmSmem<BN, B_MN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + L::kStages * L::kStageBytes);
+    uint64_t* full = bars;
+    uint64_t* empty = bars + L::kStages;
+    uint64_t* acc_full = bars + 2 * L::kStages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * L::kStages + 1);
+    volatile int32_t* abort_flag = reinterpret_cast<volatile int32_t*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const Abort ab{abort_flag, p.status};
+
+    // tile coordinates
+    // expand: linear grid, (plane, group) fastest so that the CTAs sharing a tile of cache rows run together
+    const int m_tile = (MODE == kGemmExpand) ? (int)(blockIdx.x / (2 * p.g)) : (int)blockIdx.x;
+    const int grp = (MODE == kGemmExpand) ? (int)(blockIdx.x % (2 * p.g)) : (int)blockIdx.y;  // plane * g + j, or j
+    const int n_tile = (MODE == kGemmExpand) ? 0 : (int)blockIdx.z;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < L::kStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(acc_full, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, BN);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const CUtensorMap* tmB = (MODE == kGemmExpand && grp >= p.g) ? &tmB1 : &tmB0;
+    const int j = (MODE == kGemmExpand) ? grp % p.g : grp;
+
+    if (warp == 0) {
+        if (elect_one()) {
+            tma_prefetch_desc(&tmA);
+            tma_prefetch_desc(tmB);
+            for (int kb = 0; kb < p.k_blocks; ++kb) {
+                const int s = kb % L::kStages;
+                const uint32_t ph = (kb / L::kStages) & 1;
+                if (!mbar_wait(&empty[s], ph ^ 1, ab, 1)) break;
+                uint8_t* a_dst = tiles + s * L::kStageBytes;
+                uint8_t* b_dst = a_dst + L::kABytes;
+                mbar_expect_tx(&full[s], L::kStageBytes);
+                if (MODE == kGemmExpand) {
+                    tma_load_2d(a_dst, &tmA, kb * 64, m_tile * 128, &full[s]);
+                } else {
+                    // 4-D view (feature, head-in-group, group, query position): 128/hpg positions x hpg heads
+                    asm volatile(
+                        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], "
+                        "[%1, {%3, %4, %5, %6}], [%2];" ::"r"(smem_u32(a_dst)),
+                        "l"(reinterpret_cast<uint64_t>(&tmA)), "r"(smem_u32(&full[s])), "r"(kb * 64), "r"(0), "r"(j),
+                        "r"(m_tile * (128 / p.hpg))
+                        : "memory");
+                }
+                if (B_MN) {
+                    // rows = j * K + k, columns = output feature; one 64x64 box per 64 output columns
+#pragma unroll
+                    for (int nb = 0; nb < BN / 64; ++nb)
+                        tma_load_2d(b_dst + nb * 8192, tmB, n_tile * BN + nb * 64, j * p.k_blocks * 64 + kb * 64,
+                                    &full[s]);
+                } else {
+                    // rows = j * r_kv + output feature, columns = k
+                    tma_load_2d(b_dst, tmB, kb * 64, j * p.r_kv + n_tile * BN, &full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (elect_one()) {
+            constexpr uint32_t idesc = idesc_bf16(128, BN, 0, B_MN ? 1 : 0);
+            bool ok = true;
+            for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
+                const int s = kb % L::kStages;
+                const uint32_t ph = (kb / L::kStages) & 1;
+                ok = mbar_wait(&full[s], ph, ab, 2);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(tiles + s * L::kStageBytes);
+                const uint32_t b_addr = a_addr + L::kABytes;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t a_desc = desc_kmajor_sw128(a_addr + ks * 32);
+                    const uint64_t b_desc = B_MN ? desc_mnmajor_sw128(b_addr + ks * 2048, 8192)
+                                                 : desc_kmajor_sw128(b_addr + ks * 32);
+                    umma_ss(tmem_base, a_desc, b_desc, idesc, (kb | ks) != 0);
+                }
+                umma_commit(&empty[s]);
+            }
+            if (ok) umma_commit(acc_full);
+        }
+    } else {
+        // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32)
+        const int q = warp & 3;
+        const int row = q * 32 + lane;  // row of the tile == TMEM lane
+        const bool ok = mbar_wait(acc_full, 0, ab, 3);
+        tc_fence_after();
+        __nv_bfloat16* dst = nullptr;
+        if (MODE == kGemmExpand) {
+            const int64_t n = (int64_t)m_tile * 128 + row;
+            if (n < p.m_total) {
+                __nv_bfloat16* plane = reinterpret_cast<__nv_bfloat16*>(grp >= p.g ? p.out1 : p.out0);
+                dst = plane + n * ((int64_t)p.g * p.d_h) + (int64_t)j * p.d_h + n_tile * BN;
+                if (grp == 0 && n_tile == 0 && p.aux_out != nullptr) {
+                    const uint4* src = reinterpret_cast<const uint4*>(
+                        reinterpret_cast<const __nv_bfloat16*>(p.aux_in) + n * p.aux_stride + p.r_kv);
+                    uint4* kr = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.aux_out) + n * p.d_r);
+                    for (int c = 0; c < p.d_r / 8; ++c) kr[c] = src[c];
+                }
+            }
+        } else {
+            const int64_t bp = (int64_t)m_tile * (128 / p.hpg) + row / p.hpg;
+            const int i = j * p.hpg + row % p.hpg;
+            if (bp < p.m_total) {
+                const int64_t r = bp * p.h_q + i;
+                if (MODE == kGemmAbsorbQ) {
+                    __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out0) + r * (p.r_kv + p.d_r);
+                    dst = orow + n_tile * BN;
+                    if (n_tile == 0) {
+                        const uint4* src =
+                            reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.aux_in) + r * p.d_r);
+                        uint4* tail = reinterpret_cast<uint4*>(orow + p.r_kv);
+                        for (int c = 0; c < p.d_r / 8; ++c) tail[c] = src[c];
+                    }
+                } else {
+                    dst = reinterpret_cast<__nv_bfloat16*>(p.out0) + r * p.d_h + n_tile * BN;
+                }
+            }
+        }
+        if (ok) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem_addr(tmem_base, q * 32, c0), v);
+                tmem_wait_ld();
+                if (dst != nullptr) {
+                    uint4* d4 = reinterpret_cast<uint4*>(dst + c0);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        uint4 o;
+                        o.x = pack_bf16(__uint_as_float(v[8 * t + 0]), __uint_as_float(v[8 * t + 1]));
+                        o.y = pack_bf16(__uint_as_float(v[8 * t + 2]), __uint_as_float(v[8 * t + 3]));
+                        o.z = pack_bf16(__uint_as_float(v[8 * t + 4]), __uint_as_float(v[8 * t + 5]));
+                        o.w = pack_bf16(__uint_as_float(v[8 * t + 6]), __uint_as_float(v[8 * t + 7]));
+                        d4[t] = o;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, BN);
+}
+
+// ----------------------------------------------------------------------------- host launchers
+
+template <int MODE, int BN, bool B_MN>
+inline cudaError_t gemm_launch(const GemmParams& p, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
+                               dim3 grid, cudaStream_t st) {
+    using L = GemmSmem<BN, B_MN>;
+    auto kern = gemm_tc_kernel<MODE, BN, B_MN>;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    kern<<<grid, 192, L::kTotal, st>>>(p, a, b0, b1);
+    return cudaGetLastError();
+}
+
+}  // namespace tc
+}  // namespace gqla
