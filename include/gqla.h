@@ -86,13 +86,16 @@ gqla_status gqla_absorb_q(const gqla_dims* dims, gqla_dtype dtype, int32_t B, in
 
 /* Eq. (mqa), lines 3-5: split-KV attention of every head over the shared latent rows.
  *   q_hat [B, s_q, h_q, r_kv+d_r];  cache [N, r_kv+d_r] with row stride
- *   cache_row_stride (elements);  seq_start int64 [B], seqlens int32 [B] (device).
+ *   cache_row_stride (elements) and cache_rows = N rows in total (rows >= N are never read; rows
+ *   < N outside a sequence may be fetched by a tile and must hold finite values -- they get
+ *   zero weight);  seq_start int64 [B], seqlens int32 [B] (device).
  *   o_part   [B, S, s_q, h_q, r_kv] fp32 (out),  lse_part [B, S, s_q, h_q] fp32 (out).
  *   S = num_splits >= 1.  Cache bytes are read once per step whatever s_q is (Sec. 4.2.1). */
 gqla_status gqla_decode_absorb(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
                                int32_t num_splits, const void* q_hat, const void* cache,
-                               int64_t cache_row_stride, const int64_t* seq_start, const int32_t* seqlens,
-                               float* o_part, float* lse_part, int32_t* status_word, void* stream);
+                               int64_t cache_row_stride, int64_t cache_rows, const int64_t* seq_start,
+                               const int32_t* seqlens, float* o_part, float* lse_part, int32_t* status_word,
+                               void* stream);
 
 /* Sec. 3.1: k^C = W^UK c^KV, v^C = W^UV c^KV per group, k^R carried over -- the one-shot
  * cache expansion that switches from the absorb path to the GQA path.
@@ -105,12 +108,14 @@ gqla_status gqla_expand_cache(const gqla_dims* dims, gqla_dtype dtype, int64_t N
 
 /* Eq. (mha): split-KV attention of each head over its group's K_C, V plus the shared k^R.
  *   q [B, s_q, h_q, d_h+d_r] (= [q^C ; q^R]);  k_c, v [N, g, d_h];  k_r [N, .] with row stride
- *   k_r_row_stride (elements; d_r for a dense plane, r_kv+d_r when aliasing the latent cache).
+ *   k_r_row_stride (elements; d_r for a dense plane, r_kv+d_r when aliasing the latent cache);
+ *   n_rows = N, the row count of the three planes (same reading rule as cache_rows above).
  *   o_part [B, S, s_q, h_q, d_h] fp32 (out),  lse_part [B, S, s_q, h_q] fp32 (out). */
 gqla_status gqla_decode_gqa(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
                             int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
-                            int64_t k_r_row_stride, const int64_t* seq_start, const int32_t* seqlens,
-                            float* o_part, float* lse_part, int32_t* status_word, void* stream);
+                            int64_t k_r_row_stride, int64_t n_rows, const int64_t* seq_start,
+                            const int32_t* seqlens, float* o_part, float* lse_part, int32_t* status_word,
+                            void* stream);
 
 /* Log-sum-exp merge of split partials (split-KV is not in the paper; it is the flash-decoding
  * reduction of the same softmax):  M = max_k lse_k, w_k = exp(lse_k - M),

@@ -36,12 +36,12 @@ _PROTOTYPES = {
     "gqla_get_policy": (c_int32, []),
     "gqla_absorb_q": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_decode_absorb": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
-                                     c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+                                     c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_expand_cache": (c_int32, [c_void_p, c_int32, c_int64, c_void_p, c_int64, c_void_p, c_void_p, c_void_p,
                                     c_void_p, c_void_p, c_void_p]),
     "gqla_decode_gqa": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
-                                  c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
-                                  c_void_p]),
+                                  c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                                  c_void_p, c_void_p]),
     "gqla_combine_splits": (c_int32, [c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p]),
     "gqla_up_proj": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -141,7 +141,7 @@ def gqla_decode_absorb(dims: GqlaDims, q_hat: torch.Tensor, cache: torch.Tensor,
     assert o_part.dtype == torch.float32 and lse_part.dtype == torch.float32
     B, s_q = q_hat.shape[0], q_hat.shape[1]
     _check(lib().gqla_decode_absorb(ctypes.byref(dims), _dtype_code(q_hat), B, s_q, scale, num_splits, _ptr(q_hat),
-                                    _ptr(cache), cache.stride(0), _ptr(seq_start), _ptr(seqlens), _ptr(o_part),
+                                    _ptr(cache), cache.stride(0), cache.shape[0], _ptr(seq_start), _ptr(seqlens), _ptr(o_part),
                                     _ptr(lse_part), _ptr(status_word), _stream()), "gqla_decode_absorb")
 
 
@@ -165,7 +165,7 @@ def gqla_decode_gqa(dims: GqlaDims, q: torch.Tensor, k_c: torch.Tensor, v: torch
     assert o_part.dtype == torch.float32 and lse_part.dtype == torch.float32
     B, s_q = q.shape[0], q.shape[1]
     _check(lib().gqla_decode_gqa(ctypes.byref(dims), _dtype_code(q), B, s_q, scale, num_splits, _ptr(q), _ptr(k_c),
-                                 _ptr(v), _ptr(k_r), k_r.stride(0), _ptr(seq_start), _ptr(seqlens), _ptr(o_part),
+                                 _ptr(v), _ptr(k_r), k_r.stride(0), k_c.shape[0], _ptr(seq_start), _ptr(seqlens), _ptr(o_part),
                                  _ptr(lse_part), _ptr(status_word), _stream()), "gqla_decode_gqa")
 
 

@@ -188,17 +188,17 @@ static gqla_status check_decode_common(const gqla_dims* d, gqla_dtype dtype, int
 
 gqla_status gqla_decode_absorb(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
                                int32_t num_splits, const void* q_hat, const void* cache, int64_t cache_row_stride,
-                               const int64_t* seq_start, const int32_t* seqlens, float* o_part, float* lse_part,
-                               int32_t* status_word, void* stream) {
+                               int64_t cache_rows, const int64_t* seq_start, const int32_t* seqlens, float* o_part,
+                               float* lse_part, int32_t* status_word, void* stream) {
     gqla_status s = check_decode_common(d, dtype, B, s_q, num_splits, seq_start, seqlens, o_part, lse_part);
     if (s != GQLA_OK) return s;
     if (B == 0) return GQLA_OK;
     if (q_hat == nullptr || cache == nullptr) return GQLA_ERR_NULL;
     if (!aligned16(q_hat) || !aligned16(cache)) return GQLA_ERR_ALIGN;
-    if (cache_row_stride < d->r_kv + d->d_r) return GQLA_ERR_SHAPE;
+    if (cache_row_stride < d->r_kv + d->d_r || cache_rows < 0) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, 0)) {
-        s = tc_decode_absorb(*d, B, s_q, scale, num_splits, q_hat, cache, cache_row_stride, seq_start, seqlens,
+        s = tc_decode_absorb(*d, B, s_q, scale, num_splits, q_hat, cache, cache_row_stride, cache_rows, seq_start, seqlens,
                              o_part, lse_part, status_word, st);
         if (s != GQLA_ERR_UNSUPPORTED) return s;
     }
@@ -215,17 +215,17 @@ gqla_status gqla_decode_absorb(const gqla_dims* d, gqla_dtype dtype, int32_t B, 
 
 gqla_status gqla_decode_gqa(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
                             int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
-                            int64_t k_r_row_stride, const int64_t* seq_start, const int32_t* seqlens, float* o_part,
-                            float* lse_part, int32_t* status_word, void* stream) {
+                            int64_t k_r_row_stride, int64_t n_rows, const int64_t* seq_start, const int32_t* seqlens,
+                            float* o_part, float* lse_part, int32_t* status_word, void* stream) {
     gqla_status s = check_decode_common(d, dtype, B, s_q, num_splits, seq_start, seqlens, o_part, lse_part);
     if (s != GQLA_OK) return s;
     if (B == 0) return GQLA_OK;
     if (q == nullptr || k_c == nullptr || v == nullptr || (d->d_r > 0 && k_r == nullptr)) return GQLA_ERR_NULL;
     if (!aligned16(q) || !aligned16(k_c) || !aligned16(v) || !aligned16(k_r)) return GQLA_ERR_ALIGN;
-    if (d->d_r > 0 && k_r_row_stride < d->d_r) return GQLA_ERR_SHAPE;
+    if ((d->d_r > 0 && k_r_row_stride < d->d_r) || n_rows < 0) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, 1)) {
-        s = tc_decode_gqa(*d, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, seq_start, seqlens, o_part,
+        s = tc_decode_gqa(*d, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, n_rows, seq_start, seqlens, o_part,
                           lse_part, status_word, st);
         if (s != GQLA_ERR_UNSUPPORTED) return s;
     }

@@ -4,6 +4,7 @@
 #pragma once
 #include "../../include/gqla.h"
 #include "common.cuh"
+#include "tc_decode_gqa.cuh"
 #include "tc_gemm.cuh"
 
 namespace gqla {
@@ -19,8 +20,21 @@ inline bool tc_gemm_covers(const gqla_dims& d, gqla_dtype dtype) {
 }
 
 // path: 0 = absorb, 1 = GQA
+inline int gqa_rows(const gqla_dims& d, int32_t s_q, int* hpg_box) {
+    const int hpg = d.h_q / d.g;
+    const int hb = hpg * s_q >= 8 ? hpg : 8 / s_q;
+    if (hpg_box != nullptr) *hpg_box = hb;
+    return hb * s_q;
+}
+inline bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
 inline bool tc_covers(const gqla_dims& d, gqla_dtype dtype, int32_t s_q, int32_t path) {
-    (void)d; (void)dtype; (void)s_q; (void)path;
+    if (dtype != GQLA_BF16) return false;
+    if (path == 1) {
+        if (d.d_h != 128 || d.d_r != 64 || (s_q != 1 && s_q != 2)) return false;
+        const int R = gqa_rows(d, s_q, nullptr);
+        return is_pow2(d.h_q / d.g) && R >= 8 && R <= 128;
+    }
     return false;
 }
 
@@ -116,13 +130,66 @@ inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, i
 }
 
 inline gqla_status tc_decode_absorb(const gqla_dims&, int32_t, int32_t, float, int32_t, const void*, const void*,
-                                    int64_t, const int64_t*, const int32_t*, float*, float*, int32_t*, cudaStream_t) {
+                                    int64_t, int64_t, const int64_t*, const int32_t*, float*, float*, int32_t*,
+                                    cudaStream_t) {
     return GQLA_ERR_UNSUPPORTED;
 }
-inline gqla_status tc_decode_gqa(const gqla_dims&, int32_t, int32_t, float, int32_t, const void*, const void*,
-                                 const void*, const void*, int64_t, const int64_t*, const int32_t*, float*, float*,
-                                 int32_t*, cudaStream_t) {
-    return GQLA_ERR_UNSUPPORTED;
+template <int R>
+inline cudaError_t gqa_launch(const tc::GqaParams& p, const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& r,
+                              const CUtensorMap& v, unsigned grid, cudaStream_t st) {
+    auto kern = tc::decode_gqa_tc_kernel<R>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::GqaSmem::kTotal);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, 192, tc::GqaSmem::kTotal, st>>>(p, q, k, r, v);
+    return cudaGetLastError();
+}
+
+inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S, const void* q,
+                                 const void* k_c, const void* v, const void* k_r, int64_t k_r_row_stride,
+                                 int64_t n_rows, const int64_t* seq_start, const int32_t* seqlens, float* o_part,
+                                 float* lse_part, int32_t* status, cudaStream_t st) {
+    if (!tc_covers(d, GQLA_BF16, s_q, 1) || !stride_ok(k_r_row_stride) || n_rows > 0x7fffffffLL || n_rows < 1)
+        return GQLA_ERR_UNSUPPORTED;
+    const int64_t units = (int64_t)B * S * d.g;
+    if (units > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
+    const int hpg = d.h_q / d.g;
+    int hpg_box = 0;
+    const int R = gqa_rows(d, s_q, &hpg_box);
+    CUtensorMap tmQ, tmK, tmR, tmV;
+    {
+        const int feat = d.d_h + d.d_r;
+        const uint64_t dims[4] = {(uint64_t)feat, (uint64_t)hpg, (uint64_t)d.g, (uint64_t)B * s_q};
+        const uint64_t str[3] = {(uint64_t)feat * 2, (uint64_t)hpg * feat * 2, (uint64_t)d.h_q * feat * 2};
+        const uint32_t box[4] = {64, (uint32_t)hpg_box, 1, (uint32_t)s_q};
+        if (!tc::make_tmap_bf16(&tmQ, q, 4, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[3] = {(uint64_t)d.d_h, (uint64_t)d.g, (uint64_t)n_rows};
+        const uint64_t str[2] = {(uint64_t)d.d_h * 2, (uint64_t)d.g * d.d_h * 2};
+        const uint32_t box[3] = {64, 1, 128};
+        if (!tc::make_tmap_bf16(&tmK, k_c, 3, dims, str, box)) return GQLA_ERR_CUDA;
+        if (!tc::make_tmap_bf16(&tmV, v, 3, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)d.d_r, (uint64_t)n_rows};
+        const uint64_t str[1] = {(uint64_t)k_r_row_stride * 2};
+        const uint32_t box[2] = {64, 128};
+        if (!tc::make_tmap_bf16(&tmR, k_r, 2, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    tc::GqaParams p{};
+    p.B = B; p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpg_box = hpg_box;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.seq_start = seq_start; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
+    cudaError_t e;
+    switch (R) {
+        case 8: e = gqa_launch<8>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
+        case 16: e = gqa_launch<16>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
+        case 32: e = gqa_launch<32>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
+        case 64: e = gqa_launch<64>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
+        case 128: e = gqa_launch<128>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
+        default: return GQLA_ERR_UNSUPPORTED;
+    }
+    return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
 }
 
 }  // namespace gqla

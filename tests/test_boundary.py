@@ -79,12 +79,12 @@ def test_argument_errors_return_before_launch():
     assert L.gqla_expand_cache(r(d), 0, 10, p, 575, p, p, p, p, p, None) == 2  # stride < r_kv + d_r
     assert L.gqla_expand_cache(r(d), 0, 10, p, 576, p, p, None, p, p, None) == 1
     assert L.gqla_expand_cache(r(d), 0, 0, None, 576, None, None, None, None, None, None) == 0
-    assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 0, p, p, 576, p, p, p, p, None, None) == 2  # splits < 1
-    assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, p, p, 576, None, p, p, p, None, None) == 1
-    assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, p, p, 100, p, p, p, p, None, None) == 2
-    assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, odd, p, 576, p, p, p, p, None, None) == 3
-    assert L.gqla_decode_gqa(r(d), 0, 1, 1, 0.1, 1, p, p, p, p, 32, p, p, p, p, None, None) == 2  # k_r stride < d_r
-    assert L.gqla_decode_gqa(r(d), 0, 1, 1, 0.1, 1, p, None, p, p, 64, p, p, p, p, None, None) == 1
+    assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 0, p, p, 576, 10, p, p, p, p, None, None) == 2  # splits < 1
+    assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, p, p, 576, 10, None, p, p, p, None, None) == 1
+    assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, p, p, 100, 10, p, p, p, p, None, None) == 2
+    assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, odd, p, 576, 10, p, p, p, p, None, None) == 3
+    assert L.gqla_decode_gqa(r(d), 0, 1, 1, 0.1, 1, p, p, p, p, 32, 10, p, p, p, p, None, None) == 2  # k_r stride < d_r
+    assert L.gqla_decode_gqa(r(d), 0, 1, 1, 0.1, 1, p, None, p, p, 64, 10, p, p, p, p, None, None) == 1
     assert L.gqla_combine_splits(1, 128, 0, 512, 0, p, p, p, None, None) == 2
     assert L.gqla_combine_splits(1, 128, 4, 512, 0, p, None, p, None, None) == 1
     assert L.gqla_combine_splits(1, 128, 4, 512, 9, p, p, p, None, None) == 4
