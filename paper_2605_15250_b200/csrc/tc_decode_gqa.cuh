@@ -37,7 +37,7 @@ struct GqaSmem {
     static constexpr int kStages = 2;
     static constexpr int kTileBytes = kQBytes + kStages * kStageBytes;
     static constexpr int kMergeStride = 132;                 // floats per lane row of the merge buffer
-    static constexpr int kNumBars = 14;
+    static constexpr int kNumBars = 15;
     static constexpr int kTotal = 1024 + kTileBytes + kNumBars * 8 + 16 + 2 * 128 * 4;
     static_assert(128 * kMergeStride * 4 <= kStages * kStageBytes, "merge buffer must fit in the stage area");
 };
@@ -71,7 +71,7 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
     uint64_t* vempty = bars + 7;   // [2]
     uint64_t* s_full = bars + 9;   // [2]
     uint64_t* p_ready = bars + 11; // [2]
-    uint64_t* pv_done = bars + 13;
+    uint64_t* pv_done = bars + 13; // [2]: P.V(t) arrives on pv_done[t & 1]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + L::kNumBars);
     volatile int32_t* abort_flag = reinterpret_cast<volatile int32_t*>(tmem_slot + 1);
     float* sm_m = reinterpret_cast<float*>(tmem_slot + 4);
@@ -175,7 +175,7 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
                     umma_ts(tmem_base + kColO, tmem_base + kColP + (uint32_t)s * 64 + ks * 8,
                             desc_mnmajor_sw128(v_addr + ks * 2048, 16384), idesc_pv, (t | ks) != 0);
                 umma_commit(&vempty[s]);
-                umma_commit(pv_done);
+                umma_commit(&pv_done[s]);
             }
         }
     } else {
@@ -227,8 +227,10 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
             const bool need = m_t > m_used + kRescaleThreshold;
             const float factor = need ? ex2(m_used - m_t) : 1.f;  // ex2(-inf) = 0 on first use
             if (__any_sync(0xffffffffu, need) && t > 0) {
-                // O is only touched between P.V(t-1) completing and P.V(t) being issued
-                ok = __all_sync(0xffffffffu, mbar_wait(pv_done, (t - 1) & 1, ab, 8));
+                // O is only touched between P.V(t-1) completing and P.V(t) being issued.  A warp may run one
+                // tile ahead of the others, so completions are counted on two alternating barriers: with a
+                // single one, parity alone could not tell "P.V(t-1) done" from "P.V(t-3) done".
+                ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(t - 1) & 1], ((t - 1) >> 1) & 1, ab, 8));
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll 1
@@ -274,7 +276,7 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
 
         // ------------------------------------------------------------------ merge the F replicas of each row
         float* merge = reinterpret_cast<float*>(stage0);
-        if (n_tiles > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(pv_done, (n_tiles - 1) & 1, ab, 9));
+        if (n_tiles > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, ab, 9));
         tc_fence_after();
         sm_m[Lr] = m_used;
         sm_l[Lr] = l;

@@ -4,6 +4,7 @@
 #pragma once
 #include "../../include/gqla.h"
 #include "common.cuh"
+#include "tc_decode_absorb.cuh"
 #include "tc_decode_gqa.cuh"
 #include "tc_gemm.cuh"
 
@@ -35,7 +36,8 @@ inline bool tc_covers(const gqla_dims& d, gqla_dtype dtype, int32_t s_q, int32_t
         const int R = gqa_rows(d, s_q, nullptr);
         return is_pow2(d.h_q / d.g) && R >= 8 && R <= 128;
     }
-    return false;
+    // absorb path: the pair kernel is specialised for the 512 + 64 latent row
+    return d.r_kv == 512 && d.d_r == 64 && s_q >= 1 && s_q <= 8;
 }
 
 inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t N, const void* cache,
@@ -129,11 +131,41 @@ inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, i
     return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
 }
 
-inline gqla_status tc_decode_absorb(const gqla_dims&, int32_t, int32_t, float, int32_t, const void*, const void*,
-                                    int64_t, int64_t, const int64_t*, const int32_t*, float*, float*, int32_t*,
-                                    cudaStream_t) {
-    return GQLA_ERR_UNSUPPORTED;
+inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S,
+                                    const void* q_hat, const void* cache, int64_t cache_row_stride,
+                                    int64_t cache_rows, const int64_t* seq_start, const int32_t* seqlens,
+                                    float* o_part, float* lse_part, int32_t* status, cudaStream_t st) {
+    if (!tc_covers(d, GQLA_BF16, s_q, 0) || !stride_ok(cache_row_stride) || cache_rows > 0x7fffffffLL ||
+        cache_rows < 1)
+        return GQLA_ERR_UNSUPPORTED;
+    const int rows_total = s_q * d.h_q;
+    const int row_blocks = (rows_total + 127) / 128;
+    const int64_t pairs = (int64_t)B * S * row_blocks;
+    if (2 * pairs > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
+    CUtensorMap tmQ, tmC;
+    {
+        const uint64_t dims[2] = {(uint64_t)(d.r_kv + d.d_r), (uint64_t)B * rows_total};
+        const uint64_t str[1] = {(uint64_t)(d.r_kv + d.d_r) * 2};
+        const uint32_t box[2] = {64, 64};
+        if (!tc::make_tmap_bf16(&tmQ, q_hat, 2, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)(d.r_kv + d.d_r), (uint64_t)cache_rows};
+        const uint64_t str[1] = {(uint64_t)cache_row_stride * 2};
+        const uint32_t box[2] = {64, 64};
+        if (!tc::make_tmap_bf16(&tmC, cache, 2, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    tc::AbsorbParams p{};
+    p.B = B; p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.rows_total = rows_total; p.row_blocks = row_blocks;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.seq_start = seq_start; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
+    auto kern = tc::decode_absorb_tc_kernel<0>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AbsorbSmem::kTotal) != cudaSuccess)
+        return GQLA_ERR_CUDA;
+    kern<<<(unsigned)(2 * pairs), 192, tc::AbsorbSmem::kTotal, st>>>(p, tmQ, tmC);
+    return cudaGetLastError() == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
 }
+
 template <int R>
 inline cudaError_t gqa_launch(const tc::GqaParams& p, const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& r,
                               const CUtensorMap& v, unsigned grid, cudaStream_t st) {
