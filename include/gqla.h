@@ -66,7 +66,8 @@ typedef enum {
     GQLA_ERR_DTYPE = 4,       /* unknown dtype                                  */
     GQLA_ERR_UNSUPPORTED = 5, /* valid but no kernel covers it                  */
     GQLA_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed            */
-    GQLA_ERR_TIMEOUT = 7      /* value written to *status_word by a bounded wait */
+    GQLA_ERR_TIMEOUT = 7,     /* value written to *status_word by a bounded wait */
+    GQLA_ERR_CAPACITY = 8     /* the call needs more built-in scratch than the library holds */
 } gqla_status;
 
 typedef enum { GQLA_BF16 = 0, GQLA_F32 = 1 } gqla_dtype;
@@ -116,6 +117,29 @@ gqla_status gqla_decode_gqa(const gqla_dims* dims, gqla_dtype dtype, int32_t B, 
                             int64_t k_r_row_stride, int64_t n_rows, const int64_t* seq_start,
                             const int32_t* seqlens, float* o_part, float* lse_part, int32_t* status_word,
                             void* stream);
+
+/* The same GQA-path step as gqla_decode_gqa followed by gqla_combine_splits, for callers that cannot
+ * supply the split partials.  (The paper has no counterpart: it concerns who owns memory, not what is
+ * computed.)  Meant for hosts that may not allocate on the device while decoding: a server whose memory
+ * manager claimed the whole GPU at start-up, a loop that cannot afford the device-wide synchronisation of
+ * cudaMalloc/cudaFree, or a C caller with no allocator of its own.  The partials are kept in an array built
+ * into the library's device image, so the call allocates and frees nothing.
+ *   Inputs as for gqla_decode_gqa.  out [B, s_q, h_q, d_h] of `dtype` (device, 16-byte aligned),
+ *   lse [B, s_q, h_q] fp32 (device) or NULL.
+ *   Limits: B*num_splits*s_q*h_q <= 65536 rows and rows*d_h <= 4194304 floats (16 MiB + 256 KiB in all);
+ *   anything larger returns GQLA_ERR_CAPACITY before any launch -- use gqla_decode_gqa with your own
+ *   buffers then.  Each GPU that runs the library's kernels holds the array until the process exits.
+ *   The first call on a device looks up the array's device address (one runtime query, remembered per
+ *   device; the device must be current, as for every call).  Make that first call before starting any
+ *   stream capture.
+ *   All calls on one GPU share the array and it keeps the previous call's contents.  Nothing needs
+ *   clearing (every partial is rewritten before it is read), but two calls that may run concurrently on
+ *   the same GPU race on it: issue them on one stream or order them yourself. */
+gqla_status gqla_decode_gqa_noalloc(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                                    int32_t num_splits, const void* q, const void* k_c, const void* v,
+                                    const void* k_r, int64_t k_r_row_stride, int64_t n_rows,
+                                    const int64_t* seq_start, const int32_t* seqlens, void* out, float* lse,
+                                    int32_t* status_word, void* stream);
 
 /* Log-sum-exp merge of split partials (split-KV is not in the paper; it is the flash-decoding
  * reduction of the same softmax):  M = max_k lse_k, w_k = exp(lse_k - M),

@@ -42,6 +42,9 @@ _PROTOTYPES = {
     "gqla_decode_gqa": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
                                   c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                                   c_void_p, c_void_p]),
+    "gqla_decode_gqa_noalloc": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
+                                          c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                                          c_void_p, c_void_p]),
     "gqla_combine_splits": (c_int32, [c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p]),
     "gqla_up_proj": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -167,6 +170,25 @@ def gqla_decode_gqa(dims: GqlaDims, q: torch.Tensor, k_c: torch.Tensor, v: torch
     _check(lib().gqla_decode_gqa(ctypes.byref(dims), _dtype_code(q), B, s_q, scale, num_splits, _ptr(q), _ptr(k_c),
                                  _ptr(v), _ptr(k_r), k_r.stride(0), k_c.shape[0], _ptr(seq_start), _ptr(seqlens), _ptr(o_part),
                                  _ptr(lse_part), _ptr(status_word), _stream()), "gqla_decode_gqa")
+
+
+def gqla_decode_gqa_noalloc(dims: GqlaDims, q: torch.Tensor, k_c: torch.Tensor, v: torch.Tensor, k_r: torch.Tensor,
+                            seq_start: torch.Tensor, seqlens: torch.Tensor, scale: float, num_splits: int,
+                            out: torch.Tensor, lse: torch.Tensor | None = None,
+                            status_word: torch.Tensor | None = None) -> None:
+    """GQA-path step (attention + split merge) that keeps its split partials in the library's built-in
+    device array instead of caller buffers, for hosts that must not allocate device memory while decoding.
+    out is [B, s_q, h_q, d_h]; raises (capacity) when B*num_splits*s_q*h_q > 65536 or that times d_h > 4 Mi.
+    Calls on one GPU share the array: keep them on one stream."""
+    _contig(q, k_c, v, seq_start, seqlens, out, lse)
+    assert k_r.dim() == 2 and k_r.stride(1) == 1
+    assert seq_start.dtype == torch.int64 and seqlens.dtype == torch.int32
+    assert out.dtype == q.dtype and (lse is None or lse.dtype == torch.float32)
+    B, s_q = q.shape[0], q.shape[1]
+    _check(lib().gqla_decode_gqa_noalloc(ctypes.byref(dims), _dtype_code(q), B, s_q, scale, num_splits, _ptr(q),
+                                         _ptr(k_c), _ptr(v), _ptr(k_r), k_r.stride(0), k_c.shape[0], _ptr(seq_start),
+                                         _ptr(seqlens), _ptr(out), _ptr(lse), _ptr(status_word), _stream()),
+           "gqla_decode_gqa_noalloc")
 
 
 def gqla_combine_splits(o_part: torch.Tensor, lse_part: torch.Tensor, out: torch.Tensor,

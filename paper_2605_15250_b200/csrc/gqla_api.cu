@@ -57,6 +57,7 @@ const char* gqla_status_str(gqla_status s) {
         case GQLA_ERR_UNSUPPORTED: return "unsupported configuration";
         case GQLA_ERR_CUDA: return "CUDA error";
         case GQLA_ERR_TIMEOUT: return "device wait timed out";
+        case GQLA_ERR_CAPACITY: return "call exceeds the library's built-in scratch capacity";
     }
     return "unknown status";
 }
