@@ -9,12 +9,20 @@
 // lanes for half as many columns (lanes 0-63: columns [0, N/2), lanes 64-127: columns [N/2, N) of
 // the same 64 rows), so O takes 256 columns and S (128 tokens) 64.  Each CTA also supplies half of
 // every B operand from its own shared memory: 64 of the tile's 128 cache rows for S = Qh Kh^T, and
-// 128 of every 256 latent columns for O = P V.  The cache is fetched from HBM once; the two operand
-// shapes are staged separately through L2 ([64 rows x 64 columns] 8 KB boxes, 128-byte swizzle).
+// 128 of every 256 latent columns for O = P V.  The cache is fetched from HBM once; the second
+// operand shape comes out of L2 ([64 rows x 64 columns] 8 KB boxes, 128-byte swizzle).
+//
+// Staging: two rings per CTA, one of K groups (three 8 KB boxes = 192 columns of 64 rows) and one of
+// V groups (two box pairs = one token half of a tile), each one tile deep, filled by one producer
+// thread that polls both rings so that neither blocks the other; the loads of tile t+1 are in flight
+// while the MMAs of tile t run.  Barriers are per group, not per box: every barrier operation of the
+// issuing threads costs on the order of 100 cycles next to tensor-core operand traffic, and one MMA
+// of this shape is only 32-64 cycles of tensor work.
 //
 // Warp roles per CTA: warp 0 TMA producer, warp 1 TMEM owner (+ MMA issuer in the leader CTA),
-// warps 2-5 softmax: thread = TMEM lane = (row, token half); the two threads of a row share the
-// running max through shared memory and keep separate partial sums.
+// warps 2-9 softmax.  A softmax thread owns one TMEM lane = (row, token half) and one half of that
+// lane's 64 score columns, so a row's 128 scores of a tile sit in four threads of four different
+// warps; they share the tile maximum through shared memory and keep separate partial sums.
 #pragma once
 #include "common.cuh"
 #include "tc_common.cuh"
@@ -36,29 +44,41 @@ struct AbsorbSmem {
     static constexpr int kBox = 8192;              // 64 rows x 64 bf16, 128-byte swizzle
     static constexpr int kQBytes = 9 * kBox;       // 64 query rows x 576
     static constexpr int kPBytes = 2 * kBox;       // 64 rows x 128 tokens (two 64-token k-blocks)
-    static constexpr int kNK = 6;                  // ring of K boxes (Qh Kh^T operand)
-    static constexpr int kNV = 4;                  // ring of V box PAIRS (P V operand: 64 tokens x 128 columns)
+    static constexpr int kKGroup = 3 * kBox;       // three column blocks of this CTA's 64 rows of a tile
+    static constexpr int kVGroup = 4 * kBox;       // 64 tokens x this CTA's 2 x 128 latent columns
+    static constexpr int kNK = 3;                  // ring of K groups (Qh Kh^T operand): one tile
+    static constexpr int kNV = 2;                  // ring of V groups (P V operand): one tile
     static constexpr int kOffP = kQBytes;
-    static constexpr int kOffK = kOffP + 2 * kPBytes;
-    static constexpr int kOffV = kOffK + kNK * kBox;
-    static constexpr int kTileBytes = kOffV + kNV * 2 * kBox;
+    static constexpr int kOffK = kOffP + kPBytes;
+    static constexpr int kOffV = kOffK + kNK * kKGroup;
+    static constexpr int kTileBytes = kOffV + kNV * kVGroup;
     // barriers: kfull[kNK] kempty[kNK] vfull[kNV] vempty[kNV] q_full s_full[2] p_ready[2] pv_done[2] xch[2] fin
     static constexpr int kNumBars = 2 * kNK + 2 * kNV + 10;
-    static constexpr int kBarPReady = 2 * kNK + 2 * kNV + 3;  // index of p_ready[0]
-    static constexpr int kBarXch = 2 * kNK + 2 * kNV + 7;     // index of xch[0]
-    static constexpr int kTotal = 1024 + kTileBytes + kNumBars * 8 + 16 + 3 * 128 * 4 + 2 * 128 * 4;
+    static constexpr int kSoftmaxWarps = 8;
+    static constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
+    // output staging for the epilogue (reuses P and both rings): 64 rows of 512 fp32, padded pitch
+    static constexpr int kOutPitch = 512 * 4 + 16;
+    static_assert(64 * kOutPitch <= kTileBytes - kOffP, "output staging must fit behind Q");
+    // after the barriers: tmem slot + abort flag (16 B), sm_max [2][4][64] (sm_l [4][64] reuses it).  No slack for
+    // re-aligning the base: the kernel checks that the dynamic segment starts on a 1 KB boundary.
+    static constexpr int kTotal = kTileBytes + kNumBars * 8 + 16 + 2 * 4 * 64 * 4;
+    static_assert(kTotal <= 232448, "shared memory budget of one CTA");
 };
 
 constexpr uint32_t kAColO = 0;    // O: MMA m (latent columns [256m, 256m+256)) at TMEM columns [128m, 128m+128)
 constexpr uint32_t kAColS = 256;  // two 64-column score buffers
 
 template <int DUMMY>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(AbsorbSmem::kThreads, 1)
 decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap tmQ,
                         const __grid_constant__ CUtensorMap tmC) {
     using L = AbsorbSmem;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* tiles = smem_raw;
+    if ((smem_u32(tiles) & 1023u) != 0) {  // swizzled tiles need 1 KB alignment; same answer in both CTAs
+        if (threadIdx.x == 0 && p.status != nullptr) atomicCAS(p.status, 0, kStatusTimeout | (15 << 8));
+        return;
+    }
     uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + L::kTileBytes);
     uint64_t* kfull = bars;
     uint64_t* kempty = kfull + L::kNK;
@@ -66,14 +86,16 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
     uint64_t* vempty = vfull + L::kNV;
     uint64_t* q_full = vempty + L::kNV;
     uint64_t* s_full = q_full + 1;   // [2]
-    uint64_t* p_ready = s_full + 2;  // [2] leader only, 256 arrivals
+    uint64_t* p_ready = s_full + 2;  // [2] leader only: one arrival per softmax warp of the pair
     uint64_t* pv_done = p_ready + 2; // [2]
-    uint64_t* xch = pv_done + 2;     // [2] softmax threads of this CTA: per-tile max exchange (128 arrivals)
+    uint64_t* xch = pv_done + 2;     // [2] softmax warps of this CTA: per-tile max exchange
     uint64_t* fin = xch + 2;         //     and the final partial-sum exchange
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + L::kNumBars);
     volatile int32_t* abort_flag = reinterpret_cast<volatile int32_t*>(tmem_slot + 1);
-    float* sm_l = reinterpret_cast<float*>(tmem_slot + 4);  // [128] final partial sums
-    float* sm_max = sm_l + 128;                              // [2][128] per-tile local maxima
+    float* sm_max = reinterpret_cast<float*>(tmem_slot + 4);  // [2][4][64] per-tile partial maxima
+    // [4][64] final partial sums; written only after the last P.V, i.e. after every warp has arrived
+    // on p_ready of the last tile and hence finished reading sm_max
+    float* sm_l = sm_max;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cta = cluster_ctarank();  // 0 = leader
@@ -93,8 +115,10 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::kNumBars; ++i) {
-            const bool pr = i == L::kBarPReady || i == L::kBarPReady + 1;
-            mbar_init(&bars[i], pr ? 256 : (i >= L::kBarXch ? 128 : 1));
+            uint64_t* bar = &bars[i];
+            const bool pr = bar == &p_ready[0] || bar == &p_ready[1];
+            const bool xc = bar == &xch[0] || bar == &xch[1] || bar == fin;
+            mbar_init(bar, pr ? 2 * L::kSoftmaxWarps : (xc ? L::kSoftmaxWarps : 1));
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -119,36 +143,50 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
             if (cta == 0) mbar_expect_tx(q_full, 2 * L::kQBytes);
             for (int kb = 0; kb < 9; ++kb)
                 tma_load_2d_pair(tiles + kb * L::kBox, &tmQ, kb * 64, b * p.rows_total + rho0, q_full_l);
-            int ik = 0, iv = 0;  // running box / pair counters
-            auto load_k = [&](int t) -> bool {
-                const int32_t row = (int32_t)(row0 + (int64_t)t * 128 + cta * 64);
-                for (int kb = 0; kb < 9; ++kb, ++ik) {
-                    const int s = ik % L::kNK;
-                    if (!mbar_wait(&kempty[s], ((ik / L::kNK) & 1) ^ 1, ab, 1)) return false;
-                    if (cta == 0) mbar_expect_tx(&kfull[s], 2 * L::kBox);
-                    tma_load_2d_pair(tiles + L::kOffK + s * L::kBox, &tmC, kb * 64, row, mapa(smem_u32(&kfull[s]), 0));
+            // K groups in the order (tile, column third); V groups in the order (tile, token half).
+            // Both rings are polled with a non-blocking probe: a full ring never keeps the other one
+            // from being refilled.
+            const int total_k = 3 * n_tiles, total_v = 2 * n_tiles;
+            int ik = 0, ks = 0, kt = 0, kg = 0;          // K: running index, ring slot, tile, column third
+            int iv = 0, vs = 0, vt = 0, vh = 0;          // V: running index, ring slot, tile, token half
+            uint32_t kph = 1, vph = 1;                   // parity that means "slot is free"
+            uint32_t idle = 0;
+            while (ik < total_k || iv < total_v) {
+                bool progressed = false;
+                if (ik < total_k && mbar_test_wait(&kempty[ks], kph)) {
+                    if (cta == 0) mbar_expect_tx(&kfull[ks], 2 * L::kKGroup);
+                    const int32_t row = (int32_t)(row0 + (int64_t)kt * 128 + cta * 64);
+                    const uint32_t bar = mapa(smem_u32(&kfull[ks]), 0);
+                    uint8_t* dst = tiles + L::kOffK + ks * L::kKGroup;
+#pragma unroll
+                    for (int i = 0; i < 3; ++i) tma_load_2d_pair(dst + i * L::kBox, &tmC, (3 * kg + i) * 64, row, bar);
+                    ++ik;
+                    if (++ks == L::kNK) { ks = 0; kph ^= 1; }
+                    if (++kg == 3) { kg = 0; ++kt; }
+                    progressed = true;
                 }
-                return true;
-            };
-            auto load_v = [&](int t) -> bool {
-                // order: token half h, then MMA m; this CTA supplies latent columns [256m + 128cta, +128)
-                for (int h = 0; h < 2; ++h)
-                    for (int m = 0; m < 2; ++m, ++iv) {
-                        const int s = iv % L::kNV;
-                        if (!mbar_wait(&vempty[s], ((iv / L::kNV) & 1) ^ 1, ab, 2)) return false;
-                        if (cta == 0) mbar_expect_tx(&vfull[s], 4 * L::kBox);
-                        const int32_t row = (int32_t)(row0 + (int64_t)t * 128 + h * 64);
-                        const uint32_t bar = mapa(smem_u32(&vfull[s]), 0);
-                        uint8_t* dst = tiles + L::kOffV + s * 2 * L::kBox;
-                        tma_load_2d_pair(dst, &tmC, 256 * m + 128 * (int)cta, row, bar);
-                        tma_load_2d_pair(dst + L::kBox, &tmC, 256 * m + 128 * (int)cta + 64, row, bar);
-                    }
-                return true;
-            };
-            bool ok = load_k(0);
-            for (int t = 0; t < n_tiles && ok; ++t) {
-                if (t + 1 < n_tiles) ok = load_k(t + 1);
-                if (ok) ok = load_v(t);
+                // the V boxes of a tile are re-reads of its K boxes: issue them after those, so they hit L2
+                if (iv < total_v && kt > vt && mbar_test_wait(&vempty[vs], vph)) {
+                    if (cta == 0) mbar_expect_tx(&vfull[vs], 2 * L::kVGroup);
+                    const int32_t row = (int32_t)(row0 + (int64_t)vt * 128 + vh * 64);
+                    const uint32_t bar = mapa(smem_u32(&vfull[vs]), 0);
+                    uint8_t* dst = tiles + L::kOffV + vs * L::kVGroup;
+                    // box (m, i): latent columns [256m + 128cta + 64i, +64) -- this CTA's half of MMA m's N
+#pragma unroll
+                    for (int mi = 0; mi < 4; ++mi)
+                        tma_load_2d_pair(dst + mi * L::kBox, &tmC, 256 * (mi >> 1) + 128 * (int)cta + 64 * (mi & 1), row, bar);
+                    ++iv;
+                    if (++vs == L::kNV) { vs = 0; vph ^= 1; }
+                    if (++vh == 2) { vh = 0; ++vt; }
+                    progressed = true;
+                }
+                if (progressed) {
+                    idle = 0;
+                } else {
+                    ++idle;
+                    if ((idle & 63u) == 63u && ab.raised()) break;
+                    if (idle > kWaitSpins) { ab.raise(1); break; }
+                }
             }
         }
     } else if (warp == 1) {
@@ -157,19 +195,25 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
             constexpr uint32_t idesc_qk = idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t idesc_pv = idesc_bf16(128, 256, 0, 1);
             const uint32_t q_addr = smem_u32(tiles);
-            int ik = 0, iv = 0;
+            const uint32_t p_addr = smem_u32(tiles + L::kOffP);
+            int ks = 0, vs = 0;
+            uint32_t kph = 0, vph = 0;
             auto issue_qk = [&](int t) -> bool {
                 const uint32_t d = tmem_base + kAColS + (uint32_t)(t & 1) * 64;
-                for (int kb = 0; kb < 9; ++kb, ++ik) {
-                    const int s = ik % L::kNK;
-                    if (!mbar_wait(&kfull[s], (ik / L::kNK) & 1, ab, 3)) return false;
+#pragma unroll 1
+                for (int g3 = 0; g3 < 3; ++g3) {
+                    if (!mbar_wait(&kfull[ks], kph, ab, 3)) return false;
                     tc_fence_after();
-                    const uint32_t k_addr = smem_u32(tiles + L::kOffK + s * L::kBox);
+                    const uint32_t k_addr = smem_u32(tiles + L::kOffK + ks * L::kKGroup);
+                    const uint32_t qg = q_addr + g3 * 3 * L::kBox;
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_ss2(d, desc_kmajor_sw128(q_addr + kb * L::kBox + ks * 32),
-                                 desc_kmajor_sw128(k_addr + ks * 32), idesc_qk, (kb | ks) != 0);
-                    umma_commit2(&kempty[s], 3);
+                    for (int i = 0; i < 3; ++i)
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma_ss2(d, desc_kmajor_sw128(qg + i * L::kBox + kk * 32),
+                                     desc_kmajor_sw128(k_addr + i * L::kBox + kk * 32), idesc_qk, (g3 | i | kk) != 0);
+                    umma_commit2(&kempty[ks], 3);
+                    if (++ks == L::kNK) { ks = 0; kph ^= 1; }
                 }
                 umma_commit2(&s_full[t & 1], 3);
                 return true;
@@ -180,30 +224,35 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
                 if (t + 1 < n_tiles) ok = issue_qk(t + 1);
                 if (!ok) break;
                 if (!(ok = mbar_wait(&p_ready[t & 1], (t >> 1) & 1, ab, 5))) break;
-                const uint32_t p_addr = smem_u32(tiles + L::kOffP + (t & 1) * L::kPBytes);
-                for (int h = 0; h < 2 && ok; ++h)
-                    for (int m = 0; m < 2; ++m, ++iv) {
-                        const int s = iv % L::kNV;
-                        if (!(ok = mbar_wait(&vfull[s], (iv / L::kNV) & 1, ab, 6))) break;
-                        tc_fence_after();
-                        const uint32_t v_addr = smem_u32(tiles + L::kOffV + s * 2 * L::kBox);
+                tc_fence_after();
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
+                    if (!(ok = mbar_wait(&vfull[vs], vph, ab, 6))) break;
+                    tc_fence_after();
+                    const uint32_t v_addr = smem_u32(tiles + L::kOffV + vs * L::kVGroup);
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
+                    for (int m = 0; m < 2; ++m)
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
                             umma_ss2(tmem_base + kAColO + (uint32_t)m * 128,
-                                     desc_kmajor_sw128(p_addr + h * L::kBox + ks * 32),
-                                     desc_mnmajor_sw128(v_addr + ks * 2048, L::kBox), idesc_pv, (t | h | ks) != 0);
-                        umma_commit2(&vempty[s], 3);
-                    }
+                                     desc_kmajor_sw128(p_addr + h * L::kBox + kk * 32),
+                                     desc_mnmajor_sw128(v_addr + m * 2 * L::kBox + kk * 2048, L::kBox), idesc_pv,
+                                     (t | h | kk) != 0);
+                    umma_commit2(&vempty[vs], 3);
+                    if (++vs == L::kNV) { vs = 0; vph ^= 1; }
+                }
                 if (ok) umma_commit2(&pv_done[t & 1], 3);
             }
         }
     } else {
-        // ------------------------------------------------------------------ softmax: thread = TMEM lane
-        const int q = warp & 3;
-        const int Lr = q * 32 + lane;  // TMEM lane
-        const int r = Lr & 63;         // row within this CTA
-        const int hf = Lr >> 6;        // token half of each 128-token tile / column half of each O block
-        const int rho = rho0 + r;      // (query, head) row of the sequence
+        // ------------------------------------------------------------------ softmax
+        const int q = warp & 3;              // TMEM lane quadrant this warp may access
+        const int ch = (warp - 2) >> 2;      // which 32 of the lane's 64 score columns
+        const int Lr = q * 32 + lane;        // TMEM lane
+        const int r = Lr & 63;               // row within this CTA
+        const int hf = Lr >> 6;              // token half of each 128-token tile / column half of each O block
+        const int part = hf * 2 + ch;        // one of the four threads of row r
+        const int rho = rho0 + r;            // (query, head) row of the sequence
         const bool row_valid = rho < p.rows_total;
         const int pq = row_valid ? rho / p.h_q : 0;
         int32_t lim = visible_limit(T, p.s_q, pq);
@@ -220,85 +269,112 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
             ok = __all_sync(0xffffffffu, mbar_wait(&s_full[sb], (t >> 1) & 1, ab, 7));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t s_addr = lane_base + kAColS + (uint32_t)sb * 64;
-            const int tok0 = t * 128 + hf * 64;
-            uint32_t x[64];
-            tmem_ld32(s_addr, x);
-            tmem_ld32(s_addr + 32, x + 32);
+            const int tok0 = t * 128 + hf * 64 + ch * 32;
+            uint32_t x[32];
+            tmem_ld32(lane_base + kAColS + (uint32_t)sb * 64 + ch * 32, x);
             tmem_wait_ld();
+            const bool full = tok0 + 32 <= lim;  // every score of this thread is visible
             float mx = -INFINITY;
+            if (full) {
 #pragma unroll
-            for (int c = 0; c < 64; ++c)
-                if (tok0 + c < lim) mx = fmaxf(mx, __uint_as_float(x[c]));
-            // the other token half of this row lives in lane Lr ^ 64
-            sm_max[sb * 128 + Lr] = mx;
-            mbar_arrive(&xch[sb]);
+                for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(x[c]));
+            } else {
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                    if (tok0 + c < lim) mx = fmaxf(mx, __uint_as_float(x[c]));
+            }
+            // the other three parts of this row live in other warps
+            float* mxs = sm_max + sb * 256;
+            mxs[part * 64 + r] = mx;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&xch[sb]);
             ok = __all_sync(0xffffffffu, mbar_wait(&xch[sb], (t >> 1) & 1, ab, 10));
             if (!ok) break;
-            mx = fmaxf(mx, sm_max[sb * 128 + (Lr ^ 64)]);
+            mx = fmaxf(fmaxf(mxs[r], mxs[64 + r]), fmaxf(mxs[128 + r], mxs[192 + r]));
             const float m_t = mx * p.scale_log2;
             const bool need = m_t > m_used + 8.0f;
             const float factor = need ? ex2(m_used - m_t) : 1.f;
-            if (__any_sync(0xffffffffu, need) && t > 0) {
-                ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(t - 1) & 1], ((t - 1) >> 1) & 1, ab, 8));
-                if (!ok) break;
-                tc_fence_after();
-#pragma unroll 1
-                for (int c = 0; c < 256; c += 32) {
-                    uint32_t o[32];
-                    tmem_ld32(lane_base + kAColO + c, o);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-                    tmem_st32(lane_base + kAColO + c, o);
-                }
-                tmem_wait_st();
-            }
             if (need) {
                 l *= factor;
                 m_used = m_t;
             }
             const float m_sub = m_used == -INFINITY ? 0.f : m_used;
-            // P row r, k-block hf: 128 bytes = 8 chunks of 8 bf16, chunk index XORed with (r & 7)
-            uint8_t* prow = tiles + L::kOffP + sb * L::kPBytes + hf * L::kBox + r * 128;
+            uint32_t pk[16];
+            if (full) {
 #pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {
-                uint32_t pk[4];
-#pragma unroll
-                for (int c = 0; c < 8; c += 2) {
-                    const int tok = tok0 + ch * 8 + c;
-                    const float e0 = tok < lim ? ex2(fmaf(__uint_as_float(x[ch * 8 + c]), p.scale_log2, -m_sub)) : 0.f;
-                    const float e1 =
-                        tok + 1 < lim ? ex2(fmaf(__uint_as_float(x[ch * 8 + c + 1]), p.scale_log2, -m_sub)) : 0.f;
+                for (int c = 0; c < 32; c += 2) {
+                    const float e0 = ex2(fmaf(__uint_as_float(x[c]), p.scale_log2, -m_sub));
+                    const float e1 = ex2(fmaf(__uint_as_float(x[c + 1]), p.scale_log2, -m_sub));
                     l += e0 + e1;
                     pk[c / 2] = pack_bf16(e0, e1);
                 }
-                *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            } else {
+#pragma unroll
+                for (int c = 0; c < 32; c += 2) {
+                    const float e0 = tok0 + c < lim ? ex2(fmaf(__uint_as_float(x[c]), p.scale_log2, -m_sub)) : 0.f;
+                    const float e1 =
+                        tok0 + c + 1 < lim ? ex2(fmaf(__uint_as_float(x[c + 1]), p.scale_log2, -m_sub)) : 0.f;
+                    l += e0 + e1;
+                    pk[c / 2] = pack_bf16(e0, e1);
+                }
             }
+            // O may be rescaled, and the P buffer rewritten, only once P.V(t-1) has completed
+            if (t > 0) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(t - 1) & 1], ((t - 1) >> 1) & 1, ab, 8));
+                if (!ok) break;
+                tc_fence_after();
+            }
+            if (__any_sync(0xffffffffu, need) && t > 0) {
+                // this thread's share of the lane's O: columns [128m + 64ch, +64) for m = 0, 1
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t col = kAColO + (uint32_t)(c >> 1) * 128 + ch * 64 + (c & 1) * 32;
+                    uint32_t o[32];
+                    tmem_ld32(lane_base + col, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                    tmem_st32(lane_base + col, o);
+                }
+                tmem_wait_st();
+            }
+            // P row r, k-block hf: 128 bytes = 8 chunks of 8 bf16, chunk index XORed with (r & 7)
+            uint8_t* prow = tiles + L::kOffP + hf * L::kBox + r * 128;
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4)
+                *reinterpret_cast<uint4*>(prow + (((ch * 4 + c4) ^ (r & 7)) << 4)) =
+                    make_uint4(pk[4 * c4], pk[4 * c4 + 1], pk[4 * c4 + 2], pk[4 * c4 + 3]);
             fence_proxy_async_smem();  // generic-proxy writes of P -> visible to the tensor core
             tc_fence_before();
-            mbar_arrive_cluster(p_ready_l[sb]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(p_ready_l[sb]);
         }
 
         // ------------------------------------------------------------------ epilogue: normalise and store
         if (n_tiles > 0 && ok)
             ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, ab, 9));
         tc_fence_after();
-        sm_l[Lr] = l;
-        mbar_arrive(fin);
+        sm_l[part * 64 + r] = l;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(fin);
         if (!__all_sync(0xffffffffu, mbar_wait(fin, 0, ab, 11))) ok = false;
-        const float Lt = l + sm_l[Lr ^ 64];
+        const float Lt = (sm_l[r] + sm_l[64 + r]) + (sm_l[128 + r] + sm_l[192 + r]);
         const bool live = ok && n_tiles > 0 && Lt > 0.f && m_used > -INFINITY;
         const float inv = live ? 1.f / Lt : 0.f;
-        float* orow = p.o_part + ((int64_t)(b * p.S + k) * p.rows_total + (row_valid ? rho : 0)) * 512;
-        for (int m = 0; m < 2; ++m) {
-            float4* dst = reinterpret_cast<float4*>(orow + 256 * m + 128 * hf);
+        // The CTA's 64 output rows are staged in shared memory (P and both rings are idle now: the last
+        // P.V has completed, and with it every MMA that read them) and leave as one 2 KB bulk store per
+        // row.  The padded pitch keeps the 16-byte stores of a quarter warp on distinct banks.
+        if (ok) {
+            uint8_t* stage = tiles + L::kOffP;
+            for (int m = 0; m < 2; ++m) {
+                float4* dst = reinterpret_cast<float4*>(stage + r * L::kOutPitch + (256 * m + 128 * hf + 64 * ch) * 4);
 #pragma unroll 1
-            for (int c = 0; c < 128; c += 32) {
-                uint32_t o[32];
-                tmem_ld32(lane_base + kAColO + m * 128 + c, o);  // warp-collective: never under a per-thread branch
-                tmem_wait_ld();
-                if (row_valid) {
+                for (int c = 0; c < 64; c += 32) {
+                    uint32_t o[32];
+                    if (n_tiles > 0) {  // CTA-uniform
+                        tmem_ld32(lane_base + kAColO + m * 128 + ch * 64 + c, o);
+                        tmem_wait_ld();
+                    }
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
                         dst[c / 4 + i] =
@@ -307,8 +383,21 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
                                  : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
+            fence_proxy_async_smem();  // staged rows -> visible to the bulk-copy engine
         }
-        if (row_valid && hf == 0)
+        __syncwarp();
+        if (lane == 0) mbar_arrive(fin);
+        if (!__all_sync(0xffffffffu, mbar_wait(fin, 1, ab, 12))) ok = false;
+        if (ok && lane < 8) {
+            const int rr = (warp - 2) * 8 + lane;  // each softmax warp ships eight rows
+            if (rho0 + rr < p.rows_total) {
+                float* grow = p.o_part + ((int64_t)(b * p.S + k) * p.rows_total + rho0 + rr) * 512;
+                bulk_store(grow, tiles + L::kOffP + rr * L::kOutPitch, 512 * 4);
+                bulk_commit();
+                bulk_wait_read();
+            }
+        }
+        if (row_valid && part == 0)
             p.lse_part[(int64_t)(b * p.S + k) * p.rows_total + rho] =
                 live ? (m_used + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
     }

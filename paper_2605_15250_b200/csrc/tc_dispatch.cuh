@@ -162,7 +162,7 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
     auto kern = tc::decode_absorb_tc_kernel<0>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AbsorbSmem::kTotal) != cudaSuccess)
         return GQLA_ERR_CUDA;
-    kern<<<(unsigned)(2 * pairs), 192, tc::AbsorbSmem::kTotal, st>>>(p, tmQ, tmC);
+    kern<<<(unsigned)(2 * pairs), tc::AbsorbSmem::kThreads, tc::AbsorbSmem::kTotal, st>>>(p, tmQ, tmC);
     return cudaGetLastError() == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
 }
 
