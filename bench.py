@@ -85,10 +85,11 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def pick_splits(batch: int, ctas_per_seq: int, min_len: int, n_sm: int = 148) -> int:
-    """Smallest split count that gives every SM about two work units, with >= 512 rows per split."""
+def pick_splits(batch: int, units_per_seq: int, min_len: int, slots: int) -> int:
+    """Smallest split count that keeps at least 80 % of the resident work slots (CTAs, or CTA pairs
+    on the absorb path) busy, with >= 512 rows per split.  Every extra split costs partial traffic."""
     s = 1
-    while batch * ctas_per_seq * s < 2 * n_sm and (min_len // (2 * s)) >= 512:
+    while batch * units_per_seq * s < 0.8 * slots and (min_len // (2 * s)) >= 512:
         s *= 2
     return s
 
@@ -205,7 +206,8 @@ def run_ours(args):
     q_c, q_r = x["q_c"].to(dev), x["q_r"].to(dev)
     total_tokens = int(x["seqlens"].sum())
     kern_a = B.kernel_for(dec.dims, torch.bfloat16, w1.s_q, "absorb")
-    S_a = args.splits if args.splits > 0 else pick_splits(w1.batch, 2 if kern_a == "tcgen05" else 1, w1.seqlen)
+    n_sm = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    S_a = args.splits if args.splits > 0 else pick_splits(w1.batch, (w1.s_q * w1.h_q + 127) // 128, w1.seqlen, n_sm // 2)
 
     def absorb_step():
         dec.absorb_step(q_c, q_r, S_a)
@@ -298,7 +300,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     expand_ms = ev0.elapsed_time(ev1)
     kern_g = B.kernel_for(dec.dims, torch.bfloat16, w2.s_q, "gqa")
-    S_g = args.splits if args.splits > 0 else pick_splits(w2.batch, w2.g, w2.seqlen)
+    S_g = args.splits if args.splits > 0 else pick_splits(w2.batch, w2.g, w2.seqlen, n_sm)
     og_part = dec._get("o_part_g", (w2.batch, S_g, w2.s_q, w2.h_q, w2.d_h), torch.float32)
     lg_part = dec._get("lse_part_g", (w2.batch, S_g, w2.s_q, w2.h_q), torch.float32)
     og = dec._get("o_g", (w2.batch, w2.s_q, w2.h_q, w2.d_h), torch.bfloat16)

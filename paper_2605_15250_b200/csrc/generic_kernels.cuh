@@ -130,6 +130,67 @@ __global__ void __launch_bounds__(128) combine_generic_kernel(int32_t B, int32_t
     if (lse != nullptr && threadIdx.x == 0) lse[r] = dead ? -INFINITY : mx + logf(den);
 }
 
+// Vectorised log-sum-exp merge for d_out % 4 == 0: one warp per (b, row); 16-byte loads of the
+// partials, each lane owning every 32nd float4 of the row.  Same arithmetic as the kernel above.
+__device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t*>(&lo);
+    u.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p) = u;
+}
+template <typename TO>
+__global__ void __launch_bounds__(256) combine_vec_kernel(int64_t rows, int32_t rows_per_seq, int32_t S, int32_t d_out,
+                                                          const float* __restrict__ o_part,
+                                                          const float* __restrict__ lse_part, TO* __restrict__ out,
+                                                          float* __restrict__ lse) {
+    const int lane = threadIdx.x & 31;
+    const int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (r >= rows) return;
+    const int64_t b = r / rows_per_seq;
+    const int rr = (int)(r % rows_per_seq);
+    const float* lp = lse_part + b * S * rows_per_seq + rr;
+    float mx = -INFINITY;
+    for (int k = lane; k < S; k += 32) mx = fmaxf(mx, lp[(int64_t)k * rows_per_seq]);
+    mx = warp_max(mx);
+    const bool dead = !(mx > -INFINITY);
+    float den = 0.f;
+    for (int k = lane; k < S; k += 32) den += dead ? 0.f : expf(lp[(int64_t)k * rows_per_seq] - mx);
+    den = warp_sum(den);
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+    const float* op = o_part + (b * S * rows_per_seq + rr) * d_out;
+    const int64_t kstride = (int64_t)rows_per_seq * d_out;
+    for (int c0 = 0; c0 < d_out; c0 += 512) {  // up to four float4 per lane and pass
+        float4 acc[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int k = 0; k < S; ++k) {
+            const float wk = dead ? 0.f : expf(lp[(int64_t)k * rows_per_seq] - mx);
+            if (wk == 0.f) continue;  // an empty split's partial is never read
+            const float* ok = op + k * kstride;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = c0 + (lane + 32 * u) * 4;
+                if (c < d_out) {
+                    const float4 x = *reinterpret_cast<const float4*>(ok + c);
+                    acc[u].x = fmaf(wk, x.x, acc[u].x);
+                    acc[u].y = fmaf(wk, x.y, acc[u].y);
+                    acc[u].z = fmaf(wk, x.z, acc[u].z);
+                    acc[u].w = fmaf(wk, x.w, acc[u].w);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int c = c0 + (lane + 32 * u) * 4;
+            if (c < d_out)
+                store4(out + r * d_out + c, make_float4(acc[u].x * inv, acc[u].y * inv, acc[u].z * inv, acc[u].w * inv));
+        }
+    }
+    if (lse != nullptr && lane == 0) lse[r] = dead ? -INFINITY : mx + logf(den);
+}
+
 // q_hat[row, r] = sum_d W_UK[j][r][d] * q_c[row, d]  (r < r_kv);  q_hat[row, r_kv + d] = q_r[row, d].
 // One block per row (b, p, i); the q_c row is staged in shared memory.
 template <typename T>

@@ -252,9 +252,20 @@ gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_spl
     if (!aligned16(o_part) || !aligned16(out)) return GQLA_ERR_ALIGN;
     const int64_t rows = (int64_t)B * rows_per_seq;
     if (rows > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (d_out % 4 == 0) {
+        const int warps = 8;
+        const unsigned blocks = (unsigned)((rows + warps - 1) / warps);
+        if (out_dtype == GQLA_BF16)
+            combine_vec_kernel<__nv_bfloat16><<<blocks, warps * 32, 0, st>>>(rows, rows_per_seq, num_splits, d_out, o_part,
+                                                                            lse_part, (__nv_bfloat16*)out, lse);
+        else
+            combine_vec_kernel<float><<<blocks, warps * 32, 0, st>>>(rows, rows_per_seq, num_splits, d_out, o_part,
+                                                                    lse_part, (float*)out, lse);
+        return launch_status();
+    }
     const size_t smem = (size_t)num_splits * sizeof(float);
     if (smem > 48 * 1024) return GQLA_ERR_UNSUPPORTED;
-    cudaStream_t st = (cudaStream_t)stream;
     if (out_dtype == GQLA_BF16)
         combine_generic_kernel<__nv_bfloat16><<<(unsigned)rows, 128, smem, st>>>(B, rows_per_seq, num_splits, d_out,
                                                                                  o_part, lse_part,
