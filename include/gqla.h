@@ -34,6 +34,16 @@
  *     chunk = ceil(ceil(T/S)/64)*64; a split may be empty (o = 0, lse = -inf).
  *     Each partial is normalised within its split; lse is the natural-log
  *     sum-exp of the scaled scores.
+ *   - Balanced split-KV: a decode call given num_splits = -S (S >= 2) lets the library cut the batch
+ *     itself.  The 128-row tiles of all sequences are laid end to end (sequence 0 first) and divided
+ *     into equal shares, one per resident worker (a CTA, or a CTA pair on the absorb path), so that
+ *     every SM gets the same amount of cache to read however ragged the batch is:  tile n belongs to
+ *     worker n / share,  share = max(ceil(total/W), ceil(max_b tiles_b/(S-1)), 1).  The pieces of a
+ *     sequence are numbered in row order; o_part / lse_part still have S slots per sequence, unused
+ *     slots get lse = -inf and their o_part is left unwritten (gqla_combine_splits never reads it).
+ *     W depends on the GPU and the shape: gqla_balanced_workers reports it, gqla_balanced_plan lists
+ *     the row ranges.  Where no kernel with this scheduler covers the call (gqla_balanced_workers
+ *     returns 0) the fixed plan with S splits is used instead -- also a valid set of partials.
  *   - Errors: argument violations return a code before anything is launched.
  *     A launch failure returns GQLA_ERR_CUDA.  Device-side waits are bounded;
  *     if one expires the kernel writes a non-zero code to *status_word (device
@@ -159,6 +169,14 @@ gqla_status gqla_up_proj(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int
  * HOST pointers. */
 /* Split ranges of a sequence of `seqlen` rows: begin[k], end[k] for k < num_splits. */
 gqla_status gqla_split_plan(int32_t seqlen, int32_t num_splits, int32_t* begin, int32_t* end);
+/* Balanced plan (see the conventions above) of a batch, on the host: begin/end [B * S] receive the row
+ * range of every (sequence, slot), (0, 0) for an unused slot; worker [B * S] (may be NULL) the worker
+ * that produces it, -1 for an unused slot.  s_cap = S >= 2, workers = W >= 1.  HOST pointers. */
+gqla_status gqla_balanced_plan(const int32_t* seqlens, int32_t B, int32_t s_cap, int32_t workers, int32_t* begin,
+                               int32_t* end, int32_t* worker);
+/* Number of workers W a balanced decode call of this shape is cut for on the CURRENT device
+ * (path: 0 = absorb, 1 = GQA); 0 if such a call falls back to the fixed plan; -1 on error. */
+int32_t gqla_balanced_workers(const gqla_dims* dims, gqla_dtype dtype, int32_t s_q, int32_t path);
 /* Rows visible to query p of an s_q-token step: max(0, seqlen - (s_q-1-p)). */
 int32_t gqla_visible_limit(int32_t seqlen, int32_t s_q, int32_t p);
 /* 0-indexed group of 0-indexed head: the paper's j(i) = ceil(i/(h_q/g)); -1 on bad input. */

@@ -91,6 +91,39 @@ def split_plan(seqlen: int, num_splits: int) -> list[tuple[int, int]]:
     return out
 
 
+TILE_ROWS = 128
+
+
+def balanced_plan(seqlens, num_splits: int, workers: int) -> list[list[tuple[int, int]]]:
+    """Balanced split-KV partition of a whole batch (not in the paper; a reading fixed by this build).
+
+    The 128-row tiles of all sequences are numbered end to end, sequence 0 first.  Tile number n goes to
+    worker n // share with share = max(ceil(total / workers), ceil(max_b tiles_b / (S - 1)), 1).  The tiles
+    of one sequence that one worker holds form one piece; a sequence's pieces are numbered in row order
+    and its unused slots are empty, written (0, 0).  Returned: per sequence, S (begin, end) row ranges.
+    Stated tile by tile on purpose: no closed forms shared with the library's arithmetic."""
+    S = num_splits
+    assert S >= 2 and workers >= 1
+    tiles = [(-(-int(T) // TILE_ROWS) if T > 0 else 0) for T in seqlens]
+    total = sum(tiles)
+    share = max(-(-total // workers), -(-max(tiles + [0]) // (S - 1)), 1)
+    plans = []
+    n = 0
+    for T, nt in zip(seqlens, tiles):
+        by_worker = {}
+        for i in range(nt):
+            by_worker.setdefault((n + i) // share, []).append(i)
+        n += nt
+        pieces = []
+        for wkr in sorted(by_worker):
+            idx = by_worker[wkr]
+            assert idx == list(range(idx[0], idx[-1] + 1))
+            pieces.append((idx[0] * TILE_ROWS, min((idx[-1] + 1) * TILE_ROWS, int(T))))
+        assert len(pieces) <= S
+        plans.append(pieces + [(0, 0)] * (S - len(pieces)))
+    return plans
+
+
 # --------------------------------------------------------------------------
 # the three plain contractions (absorb q, expand cache, up-project)
 # --------------------------------------------------------------------------
@@ -161,7 +194,7 @@ def _attend(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float, lo: int, 
     return o, lse
 
 
-def _decode(dims, q_rows_of, K_of, V_of, Dv, B, s_q, seq_start, seqlens, scale, num_splits):
+def _decode(dims, q_rows_of, K_of, V_of, Dv, B, s_q, seq_start, seqlens, scale, num_splits, plans=None):
     """Shared driver for the two paths: loops (b, split, p) and calls the
     definition on the rows each query may see.  q_rows_of(b, p) -> list of
     (head slice, q [n, D]); K_of/V_of (b, head slice) -> arrays over the
@@ -172,7 +205,8 @@ def _decode(dims, q_rows_of, K_of, V_of, Dv, B, s_q, seq_start, seqlens, scale, 
     lse_part = np.full((B, S, s_q, h_q), NEG_INF, dtype=np.float64)
     for b in range(B):
         T = int(seqlens[b])
-        plan = split_plan(T, S)
+        plan = split_plan(T, S) if plans is None else plans[b]
+        assert len(plan) == S
         for p in range(s_q):
             lim = visible_limit(T, s_q, p)
             for hs, q in q_rows_of(b, p):
@@ -185,7 +219,7 @@ def _decode(dims, q_rows_of, K_of, V_of, Dv, B, s_q, seq_start, seqlens, scale, 
     return o_part, lse_part
 
 
-def decode_absorb_partials(dims: Dims, q_hat, cache, seq_start, seqlens, s_q, scale, num_splits):
+def decode_absorb_partials(dims: Dims, q_hat, cache, seq_start, seqlens, s_q, scale, num_splits, plans=None):
     """Eq. (mqa): k_hat_s = [c_s ; k^R_s], v_hat_s = c_s, all heads share them.
 
     q_hat [B, s_q, h_q, r_kv+d_r]; cache [N, r_kv+d_r]; sequence b owns rows
@@ -213,10 +247,10 @@ def decode_absorb_partials(dims: Dims, q_hat, cache, seq_start, seqlens, s_q, sc
     def q_rows_of(b, p):
         return [(slice(0, dims.h_q), q64[b, p])]
 
-    return _decode(dims, q_rows_of, K_of, V_of, r, B, s_q, seq_start, seqlens, scale, num_splits)
+    return _decode(dims, q_rows_of, K_of, V_of, r, B, s_q, seq_start, seqlens, scale, num_splits, plans)
 
 
-def decode_gqa_partials(dims: Dims, q, k_c, v, k_r, seq_start, seqlens, s_q, scale, num_splits):
+def decode_gqa_partials(dims: Dims, q, k_c, v, k_r, seq_start, seqlens, s_q, scale, num_splits, plans=None):
     """Eq. (mha): head i attends k_{s,i} = [k^C_{s,j(i)} ; k^R_s] with values v^C_{s,j(i)}.
 
     q [B, s_q, h_q, d_h+d_r]; k_c, v [N, g, d_h]; k_r [N, d_r]."""
@@ -243,7 +277,7 @@ def decode_gqa_partials(dims: Dims, q, k_c, v, k_r, seq_start, seqlens, s_q, sca
     def q_rows_of(b, p):
         return [(slice(j * hpg, (j + 1) * hpg), q64[b, p, j * hpg:(j + 1) * hpg]) for j in range(dims.g)]
 
-    return _decode(dims, q_rows_of, K_of, V_of, dims.d_h, B, s_q, seq_start, seqlens, scale, num_splits)
+    return _decode(dims, q_rows_of, K_of, V_of, dims.d_h, B, s_q, seq_start, seqlens, scale, num_splits, plans)
 
 
 def combine_splits(o_part: np.ndarray, lse_part: np.ndarray):

@@ -50,6 +50,8 @@ _PROTOTYPES = {
     "gqla_up_proj": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_split_plan": (c_int32, [c_int32, c_int32, c_void_p, c_void_p]),
     "gqla_visible_limit": (c_int32, [c_int32, c_int32, c_int32]),
+    "gqla_balanced_plan": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p]),
+    "gqla_balanced_workers": (c_int32, [c_void_p, c_int32, c_int32, c_int32]),
     "gqla_group_of_head": (c_int32, [c_void_p, c_int32]),
     "gqla_kernel_for": (c_char_p, [c_void_p, c_int32, c_int32, c_int32]),
     "gqla_status_str": (c_char_p, [c_int32]),
@@ -217,6 +219,26 @@ def gqla_split_plan(seqlen: int, num_splits: int) -> list[tuple[int, int]]:
     end = (c_int32 * num_splits)()
     _check(lib().gqla_split_plan(seqlen, num_splits, begin, end), "gqla_split_plan")
     return [(int(begin[k]), int(end[k])) for k in range(num_splits)]
+
+
+def gqla_balanced_plan(seqlens, s_cap: int, workers: int):
+    """Balanced split plan of a batch: (plans, owners) with plans[b] = s_cap (begin, end) row ranges
+    ((0, 0) = unused slot) and owners[b][k] the worker that produces the slot (-1 = unused)."""
+    n = len(seqlens)
+    sl = (c_int32 * max(n, 1))(*[int(t) for t in seqlens])
+    begin = (c_int32 * max(n * s_cap, 1))()
+    end = (c_int32 * max(n * s_cap, 1))()
+    own = (c_int32 * max(n * s_cap, 1))()
+    _check(lib().gqla_balanced_plan(sl, n, s_cap, workers, begin, end, own), "gqla_balanced_plan")
+    plans = [[(int(begin[b * s_cap + k]), int(end[b * s_cap + k])) for k in range(s_cap)] for b in range(n)]
+    owners = [[int(own[b * s_cap + k]) for k in range(s_cap)] for b in range(n)]
+    return plans, owners
+
+
+def gqla_balanced_workers(dims: GqlaDims, dtype: torch.dtype, s_q: int, path: str) -> int:
+    """Workers a balanced decode call is cut for on the current device (0: fixed plan is used instead)."""
+    code = GQLA_BF16 if dtype == torch.bfloat16 else GQLA_F32
+    return int(lib().gqla_balanced_workers(ctypes.byref(dims), code, s_q, 0 if path == "absorb" else 1))
 
 
 def gqla_visible_limit(seqlen: int, s_q: int, p: int) -> int:

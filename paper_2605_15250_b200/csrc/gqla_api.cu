@@ -5,6 +5,7 @@
 
 #include "common.cuh"
 #include "generic_kernels.cuh"
+#include "sched.cuh"
 #include "tc_dispatch.cuh"
 
 using namespace gqla;
@@ -70,6 +71,48 @@ gqla_status gqla_split_plan(int32_t seqlen, int32_t num_splits, int32_t* begin, 
 }
 
 int32_t gqla_visible_limit(int32_t seqlen, int32_t s_q, int32_t p) { return visible_limit(seqlen, s_q, p); }
+
+gqla_status gqla_balanced_plan(const int32_t* seqlens, int32_t B, int32_t s_cap, int32_t workers, int32_t* begin,
+                               int32_t* end, int32_t* worker) {
+    if (seqlens == nullptr || begin == nullptr || end == nullptr) return GQLA_ERR_NULL;
+    if (B < 0 || s_cap < 2 || workers < 1) return GQLA_ERR_SHAPE;
+    for (int32_t b = 0; b < B; ++b)
+        if (seqlens[b] < 0) return GQLA_ERR_SHAPE;
+    const int64_t n = (int64_t)B * s_cap;
+    for (int64_t i = 0; i < n; ++i) {
+        begin[i] = end[i] = -1;  // "not written yet"
+        if (worker != nullptr) worker[i] = -1;
+    }
+    // every worker walks its share exactly as the kernels' roles do
+    for (int32_t w = 0; w < workers; ++w) {
+        Walker wk;
+        wk.init_balanced(seqlens, B, s_cap, w, workers, balanced_start_serial(seqlens, B, s_cap, w, workers));
+        Piece pc;
+        while (wk.next(pc)) {
+            if (pc.n_tiles > 0) {
+                const int64_t i = (int64_t)pc.b * s_cap + pc.k;
+                if (pc.k < 0 || pc.k >= s_cap || begin[i] != -1) return GQLA_ERR_UNSUPPORTED;  // would be a bug
+                begin[i] = pc.tok_begin;
+                end[i] = pc.tok_end;
+                if (worker != nullptr) worker[i] = w;
+            }
+            for (int32_t k = pc.fill_begin; k < pc.fill_end; ++k) {
+                const int64_t i = (int64_t)pc.b * s_cap + k;
+                if (begin[i] != -1) return GQLA_ERR_UNSUPPORTED;
+                begin[i] = end[i] = 0;
+            }
+        }
+    }
+    for (int64_t i = 0; i < n; ++i)
+        if (begin[i] == -1) return GQLA_ERR_UNSUPPORTED;  // a slot nobody owns: would be a bug
+    return GQLA_OK;
+}
+
+int32_t gqla_balanced_workers(const gqla_dims* d, gqla_dtype dtype, int32_t s_q, int32_t path) {
+    if (check_dims(d) != GQLA_OK) return -1;
+    if (g_policy.load() != GQLA_POLICY_AUTO || !tc_covers(*d, dtype, s_q, path)) return 0;
+    return tc_balanced_workers(*d, s_q, path);
+}
 
 int32_t gqla_group_of_head(const gqla_dims* d, int32_t head) {
     if (check_dims(d) != GQLA_OK || head < 0 || head >= d->h_q) return -1;

@@ -40,6 +40,31 @@ inline bool tc_covers(const gqla_dims& d, gqla_dtype dtype, int32_t s_q, int32_t
     return d.r_kv == 512 && d.d_r == 64 && s_q >= 1 && s_q <= 8;
 }
 
+// SMs of the current device (cached per device ordinal); 0 on failure.
+inline int sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+// Workers of the balanced plan: the GQA path runs one CTA per SM and keeps the cut points of all g
+// groups identical (so the CTAs of the g groups read one k_R tile together): W = SMs / g workers per
+// group.  The absorb path runs one CTA pair per two SMs: W = (SMs / 2) / row_blocks per row block.
+// 0 when the device cannot be queried (or has no GPU): the fixed plan is used then.
+inline int32_t tc_balanced_workers(const gqla_dims& d, int32_t s_q, int32_t path) {
+    const int sms = sm_count();
+    if (sms <= 0) return 0;
+    if (path == 1) return sms / d.g > 0 ? sms / d.g : 0;
+    const int row_blocks = (s_q * d.h_q + 127) / 128;
+    return (sms / 2) / row_blocks > 0 ? (sms / 2) / row_blocks : 0;
+}
+
 inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t N, const void* cache,
                                    int64_t cache_row_stride, const void* w_uk, const void* w_uv, void* k_c, void* v,
                                    void* k_r, cudaStream_t st) {

@@ -48,6 +48,39 @@ def test_split_plan_matches_oracle():
         assert B.gqla_split_plan(T, S) == O.split_plan(T, S), (T, S)
 
 
+def test_balanced_plan_matches_oracle():
+    """The library's balanced split plan (walked worker by worker, as its kernels do) against the
+    oracle's tile-by-tile statement of the same rule: ragged batches, empty sequences, more workers
+    than tiles, a single worker, and the smallest slot count."""
+    rng = np.random.default_rng(11)
+    cases = [([4096] * 64, 3, 74), ([4096] * 64, 2, 18), ([0, 0, 0], 2, 5), ([1], 2, 148), ([0, 129, 0, 128, 0], 2, 3),
+             ([131072] * 4, 8, 74), ([131072] * 4, 2, 18), ([5000, 0, 0], 4, 1), ([], 2, 4)]
+    for _ in range(300):
+        n = int(rng.integers(1, 40))
+        sl = [int(x) for x in rng.integers(0, 40000, size=n)]
+        for i in rng.integers(0, n, size=n // 4):
+            sl[int(i)] = 0
+        cases.append((sl, int(rng.integers(2, 9)), int(rng.integers(1, 160))))
+    for sl, S, W in cases:
+        plans, owners = B.gqla_balanced_plan(sl, S, W)
+        assert plans == O.balanced_plan(sl, S, W), (sl, S, W)
+        # the owner of a piece is the worker whose share holds its tiles; shares do not exceed `share`
+        load = {}
+        for b, T in enumerate(sl):
+            for k, (lo, hi) in enumerate(plans[b]):
+                if hi > lo:
+                    assert owners[b][k] >= 0
+                    load[owners[b][k]] = load.get(owners[b][k], 0) + -(-(hi - lo) // 128)
+                else:
+                    assert owners[b][k] == -1
+        tiles = [-(-t // 128) for t in sl]
+        share = max(-(-sum(tiles) // W), -(-max(tiles + [0]) // (S - 1)), 1)
+        assert all(v <= share for v in load.values())
+    assert B.lib().gqla_balanced_plan(None, 1, 2, 1, None, None, None) == 1
+    buf = (ctypes.c_int32 * 8)()
+    assert B.lib().gqla_balanced_plan(buf, 2, 1, 4, buf, buf, None) == 2  # fewer than two slots
+
+
 def test_group_map_and_mask_limit_match_oracle():
     for h_q, g in ((128, 8), (32, 8), (8, 2), (28, 4), (20, 4), (64, 64), (7, 1)):
         d = B.make_dims(h_q, g, 128, 512, 64)

@@ -354,3 +354,49 @@ def test_combine_closed_form_and_dead_rows():
     o, l = O.combine_splits(o_part, lse_part)
     assert o[0, 0, 0] == 1.0 and l[0, 0] == 0.5
     assert o[1, 0, 0] == 0.0 and np.isneginf(l[1, 0]) and not np.isnan(o).any()
+
+
+def test_balanced_plan_invariants():
+    """Pins of the oracle's balanced split plan that follow from its definition alone: the pieces of a
+    sequence are disjoint, ordered, cover exactly [0, T), start on 128-row tile boundaries and are at
+    most S; with one worker nothing is cut; a uniform batch on as many workers as sequences is not cut
+    either; hand-worked case: T = (300, 100, 0, 260) rows = (3, 1, 0, 3) tiles on 3 workers, S = 3 ->
+    share 3: worker 0 gets sequence 0, worker 1 sequence 1 and tiles 0-1 of sequence 3, worker 2 its tile 2."""
+    rng = np.random.default_rng(5)
+    for _ in range(200):
+        n = int(rng.integers(1, 30))
+        sl = [int(x) for x in rng.integers(0, 20000, size=n)]
+        S, W = int(rng.integers(2, 7)), int(rng.integers(1, 100))
+        plans = O.balanced_plan(sl, S, W)
+        assert len(plans) == n
+        for T, plan in zip(sl, plans):
+            assert len(plan) == S
+            live = [(lo, hi) for lo, hi in plan if hi > lo]
+            assert plan[:len(live)] == live and all(pc == (0, 0) for pc in plan[len(live):])
+            pos = 0
+            for lo, hi in live:
+                assert lo == pos and lo % 128 == 0
+                pos = hi
+            assert pos == T
+    assert O.balanced_plan([4096] * 8, 2, 1) == [[(0, 4096), (0, 0)]] * 8
+    assert O.balanced_plan([4096] * 8, 2, 8) == [[(0, 4096), (0, 0)]] * 8
+    assert O.balanced_plan([300, 100, 0, 260], 3, 3) == [
+        [(0, 300), (0, 0), (0, 0)], [(0, 100), (0, 0), (0, 0)], [(0, 0)] * 3, [(0, 256), (256, 260), (0, 0)]]
+
+
+def test_partials_with_an_explicit_plan_combine_to_the_same_output():
+    """Any partition of the rows gives the same attention output after the LSE merge (fp64)."""
+    w = synth.Workload("bp", 8, 2, 16, 32, 8, batch=3, s_q=2, dtype="f32", seed=21)
+    x = synth.make_inputs(w, seqlens=np.array([300, 0, 517], dtype=np.int32), q_gain=3.0)
+    f = {k: synth.to_f64(v) for k, v in x.items() if k not in ("seq_start", "seqlens")}
+    od = O.Dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)
+    ss, sl = x["seq_start"].numpy(), x["seqlens"].numpy()
+    qh = O.absorb_q(od, f["q_c"], f["q_r"], f["w_uk"])
+    ref, ref_lse = O.combine_splits(*O.decode_absorb_partials(od, qh, f["cache"], ss, sl, w.s_q, w.scale, 1))
+    for S, W in ((2, 3), (3, 2), (4, 7)):
+        plans = O.balanced_plan([int(t) for t in sl], S, W)
+        o, lse = O.combine_splits(*O.decode_absorb_partials(od, qh, f["cache"], ss, sl, w.s_q, w.scale, S, plans))
+        np.testing.assert_allclose(o, ref, rtol=1e-12, atol=1e-13)
+        fin = np.isfinite(ref_lse)
+        assert np.array_equal(np.isneginf(lse), np.isneginf(ref_lse))
+        np.testing.assert_allclose(lse[fin], ref_lse[fin], rtol=1e-12, atol=1e-12)
