@@ -223,7 +223,7 @@ static gqla_status check_decode_common(const gqla_dims* d, gqla_dtype dtype, int
     gqla_status s;
     if ((s = check_dims(d)) != GQLA_OK) return s;
     if ((s = check_dtype(dtype)) != GQLA_OK) return s;
-    if (B < 0 || s_q < 1 || S < 1) return GQLA_ERR_SHAPE;
+    if (B < 0 || s_q < 1 || S == 0 || S == -1) return GQLA_ERR_SHAPE;  // S <= -2: balanced plan, -S slots
     if (B == 0) return GQLA_OK;
     if (seq_start == nullptr || seqlens == nullptr || o_part == nullptr || lse_part == nullptr) return GQLA_ERR_NULL;
     if (!aligned16(o_part)) return GQLA_ERR_ALIGN;
@@ -252,7 +252,7 @@ gqla_status gqla_decode_absorb(const gqla_dims* d, gqla_dtype dtype, int32_t B, 
     a.kB = nullptr; a.kB_stride = 0; a.dB = 0;
     a.v = cache; a.v_stride = cache_row_stride; a.v_gstride = 0; a.dv = d->r_kv;
     a.seq_start = seq_start; a.seqlens = seqlens;
-    a.B = B; a.S = num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
+    a.B = B; a.S = num_splits < 0 ? -num_splits : num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
     a.scale = scale; a.o_part = o_part; a.lse_part = lse_part;
     return launch_decode_generic(dtype, a, st);
 }
@@ -279,7 +279,7 @@ gqla_status gqla_decode_gqa(const gqla_dims* d, gqla_dtype dtype, int32_t B, int
     a.kB = k_r; a.kB_stride = k_r_row_stride; a.dB = d->d_r;
     a.v = v; a.v_stride = (int64_t)d->g * d->d_h; a.v_gstride = d->d_h; a.dv = d->d_h;
     a.seq_start = seq_start; a.seqlens = seqlens;
-    a.B = B; a.S = num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
+    a.B = B; a.S = num_splits < 0 ? -num_splits : num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
     a.scale = scale; a.o_part = o_part; a.lse_part = lse_part;
     return launch_decode_generic(dtype, a, st);
 }

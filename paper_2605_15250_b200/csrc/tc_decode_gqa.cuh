@@ -1,4 +1,6 @@
-// GQA-path split-KV flash decoding on tcgen05 (Eq. (mha)): one CTA per (sequence, split, group).
+// GQA-path split-KV flash decoding on tcgen05 (Eq. (mha)).  A CTA works for one group j and walks
+// the (sequence, split) pieces its plan gives it (sched.cuh): exactly one piece under the fixed
+// plan, an equal share of the batch's 128-row tiles under the balanced plan (persistent CTA).
 //
 //   S = Q K^T   Q: the group's h_q/g heads x s_q queries (R rows), K = [K_C[:, j] ; k_R]  (192 wide)
 //   O = P V     P = exp2(S * scale*log2e - m),  V = V[:, j]                                (128 wide)
@@ -7,12 +9,16 @@
 // are replicated F = 128/R times down the tile and replica f only keeps the scores of tokens
 // [f*R, (f+1)*R) of each 128-token tile (its other probabilities are zero).  Every TMEM lane thus
 // runs an independent online softmax over a disjoint token subset -- no cross-thread reduction in
-// the main loop -- and the F partial (m, l, O) triples of a row are merged once at the end.
+// the main loop -- and the F partial (m, l, O) triples of a row are merged once per piece.
 //
 // Warp roles: warp 0 TMA producer, warp 1 MMA issuer (+ TMEM owner), warps 2-5 softmax (one TMEM
-// lane per thread).  P goes back to TMEM as bf16 and is the A operand of the P.V MMA.
+// lane per thread).  P goes back to TMEM as bf16 and is the A operand of the P.V MMA.  The three
+// roles walk the same plan independently; ring slots and barrier phases follow a tile counter that
+// runs across pieces, so the producer streams the next piece's tiles while the softmax warps still
+// merge and store the previous one.
 #pragma once
 #include "common.cuh"
+#include "sched.cuh"
 #include "tc_common.cuh"
 
 namespace gqla {
@@ -20,6 +26,7 @@ namespace tc {
 
 struct GqaParams {
     int32_t B, S, s_q, h_q, g, hpg, hpg_box;
+    int32_t balanced, W;  // balanced plan: W workers per group, grid = W * g
     float scale_log2;
     const int64_t* seq_start;
     const int32_t* seqlens;
@@ -35,11 +42,17 @@ struct GqaSmem {
     static constexpr int kVBytes = 2 * 16384;                // 128 tokens x 128
     static constexpr int kStageBytes = kKcBytes + kKrBytes + kVBytes;
     static constexpr int kStages = 2;
-    static constexpr int kTileBytes = kQBytes + kStages * kStageBytes;
-    static constexpr int kMergeStride = 132;                 // floats per lane row of the merge buffer
-    static constexpr int kNumBars = 15;
-    static constexpr int kTotal = 1024 + kTileBytes + kNumBars * 8 + 16 + 2 * 128 * 4;
-    static_assert(128 * kMergeStride * 4 <= kStages * kStageBytes, "merge buffer must fit in the stage area");
+    static constexpr int kMergePitch = 33;                   // floats per lane row of the 32-column merge buffer
+    static constexpr int kMergeBytes = 128 * kMergePitch * 4;
+    static constexpr int kOffMerge = kQBytes + kStages * kStageBytes;
+    static constexpr int kTileBytes = kOffMerge + kMergeBytes;
+    // q_full q_empty o_free kfull[2] vfull[2] kempty[2] vempty[2] s_full[2] p_ready[2] pv_done[2]
+    static constexpr int kNumBars = 17;
+    static constexpr int kThreads = 192;
+    // behind the barriers: tmem slot + abort flag (16 B), then sm_m[128] + sm_l[128] (also the plan scratch)
+    static constexpr int kTotal = kTileBytes + kNumBars * 8 + 16 + 2 * 128 * 4;
+    static_assert(2 * 128 >= kThreads + 4, "plan scratch must fit in sm_m + sm_l");
+    static_assert(kTotal <= 232448, "shared memory budget of one CTA");
 };
 
 // TMEM columns (all 512 are used, so one CTA per SM)
@@ -49,7 +62,7 @@ constexpr uint32_t kColO = 384;  // 128-column output accumulator
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: P may grow to 2^8 before O is rescaled
 
 template <int R>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(GqaSmem::kThreads, 1)
 decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmV) {
     using L = GqaSmem;
@@ -59,19 +72,26 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
     constexpr int W = R < 32 ? 32 : R;   // columns of S a warp reads per tile
     constexpr int CH = 32;
     constexpr int NCH = W / CH;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* tiles = smem_raw;
+    if ((smem_u32(tiles) & 1023u) != 0) {  // swizzled tiles need 1 KB alignment
+        if (threadIdx.x == 0 && p.status != nullptr) atomicCAS(p.status, 0, kStatusTimeout | (15 << 8));
+        return;
+    }
     uint8_t* q_smem = tiles;
     uint8_t* stage0 = tiles + L::kQBytes;
+    float* merge = reinterpret_cast<float*>(tiles + L::kOffMerge);
     uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + L::kTileBytes);
     uint64_t* q_full = bars + 0;
-    uint64_t* kfull = bars + 1;    // [2]
-    uint64_t* vfull = bars + 3;    // [2]
-    uint64_t* kempty = bars + 5;   // [2]
-    uint64_t* vempty = bars + 7;   // [2]
-    uint64_t* s_full = bars + 9;   // [2]
-    uint64_t* p_ready = bars + 11; // [2]
-    uint64_t* pv_done = bars + 13; // [2]: P.V(t) arrives on pv_done[t & 1]
+    uint64_t* q_empty = bars + 1;  // the last Q K^T of a piece has completed: Q may be overwritten
+    uint64_t* o_free = bars + 2;   // the softmax warps have read O of a piece: P.V may overwrite it
+    uint64_t* kfull = bars + 3;    // [2]
+    uint64_t* vfull = bars + 5;    // [2]
+    uint64_t* kempty = bars + 7;   // [2]
+    uint64_t* vempty = bars + 9;   // [2]
+    uint64_t* s_full = bars + 11;  // [2]
+    uint64_t* p_ready = bars + 13; // [2]
+    uint64_t* pv_done = bars + 15; // [2]: P.V of tile n arrives on pv_done[n & 1]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + L::kNumBars);
     volatile int32_t* abort_flag = reinterpret_cast<volatile int32_t*>(tmem_slot + 1);
     float* sm_m = reinterpret_cast<float*>(tmem_slot + 4);
@@ -80,19 +100,9 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const Abort ab{abort_flag, p.status};
 
-    // work unit
-    const int unit = blockIdx.x;
-    const int j = unit % p.g;
-    const int k = (unit / p.g) % p.S;
-    const int b = unit / (p.g * p.S);
-    const int32_t T = p.seqlens[b];
-    int32_t begin, end;
-    split_range(T, p.S, k, &begin, &end);
-    const int n_tiles = end > begin ? (end - begin + 127) >> 7 : 0;
-    const int64_t row0 = p.seq_start[b] + begin;
-
     if (threadIdx.x == 0) {
-        for (int i = 0; i < L::kNumBars; ++i) mbar_init(&bars[i], (i == 11 || i == 12) ? 128 : 1);
+        // o_free and p_ready[2] take one arrival per softmax warp
+        for (int i = 0; i < L::kNumBars; ++i) mbar_init(&bars[i], (i == 2 || i == 13 || i == 14) ? 4 : 1);
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -100,52 +110,75 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
         tmem_alloc(tmem_slot, 512);
         tmem_relinquish();
     }
+
+    // the plan of this CTA: group j, and either one (sequence, split) piece or worker w's share
+    const int j = blockIdx.x % p.g;
+    Walker walk;
+    if (p.balanced) {
+        const BalancedStart st = balanced_prepass(p.seqlens, p.B, p.S, blockIdx.x / p.g, p.W,
+                                                  reinterpret_cast<int32_t*>(sm_m), L::kThreads);
+        walk.init_balanced(p.seqlens, p.B, p.S, blockIdx.x / p.g, p.W, st);
+    } else {
+        const int unit = blockIdx.x / p.g;
+        walk.init_fixed(p.seqlens, p.B, p.S, unit / p.S, unit % p.S);
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    Piece pc;
+    int gt = 0;  // tiles walked so far: ring slot = gt & 1, barrier phase = (gt >> 1) & 1
+    int pi = 0;  // non-empty pieces walked so far
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (n_tiles > 0 && elect_one()) {
+        if (elect_one()) {
             tma_prefetch_desc(&tmQ);
             tma_prefetch_desc(&tmK);
             tma_prefetch_desc(&tmR);
             tma_prefetch_desc(&tmV);
-            mbar_expect_tx(q_full, L::kQBytes);
-            for (int kb = 0; kb < 3; ++kb)
-                for (int f = 0; f < F; ++f)
-                    asm volatile(
-                        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], "
-                        "[%1, {%3, %4, %5, %6}], [%2];" ::"r"(smem_u32(q_smem + kb * 16384 + f * R * 128)),
-                        "l"(reinterpret_cast<uint64_t>(&tmQ)), "r"(smem_u32(q_full)), "r"(kb * 64), "r"(0), "r"(j),
-                        "r"(b * p.s_q)
-                        : "memory");
-            for (int t = 0; t < n_tiles; ++t) {
-                const int s = t & 1;
-                const uint32_t ph = (t >> 1) & 1;
-                uint8_t* st = stage0 + s * L::kStageBytes;
-                const int32_t row = (int32_t)(row0 + (int64_t)t * 128);
-                if (!mbar_wait(&kempty[s], ph ^ 1, ab, 1)) break;
-                mbar_expect_tx(&kfull[s], L::kKcBytes + L::kKrBytes);
-                tma_load_3d(st, &tmK, 0, j, row, &kfull[s]);
-                tma_load_3d(st + 16384, &tmK, 64, j, row, &kfull[s]);
-                tma_load_2d(st + L::kKcBytes, &tmR, 0, row, &kfull[s]);
-                if (!mbar_wait(&vempty[s], ph ^ 1, ab, 2)) break;
-                mbar_expect_tx(&vfull[s], L::kVBytes);
-                tma_load_3d(st + L::kKcBytes + L::kKrBytes, &tmV, 0, j, row, &vfull[s]);
-                tma_load_3d(st + L::kKcBytes + L::kKrBytes + 16384, &tmV, 64, j, row, &vfull[s]);
+            bool ok = true;
+            while (ok && walk.next(pc)) {
+                if (pc.n_tiles == 0) continue;
+                // Q of this piece's sequence; the previous piece's Q K^T must all have completed
+                if (pi > 0 && !(ok = mbar_wait(q_empty, (pi - 1) & 1, ab, 13))) break;
+                mbar_expect_tx(q_full, L::kQBytes);
+                for (int kb = 0; kb < 3; ++kb)
+                    for (int f = 0; f < F; ++f)
+                        asm volatile(
+                            "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], "
+                            "[%1, {%3, %4, %5, %6}], [%2];" ::"r"(smem_u32(q_smem + kb * 16384 + f * R * 128)),
+                            "l"(reinterpret_cast<uint64_t>(&tmQ)), "r"(smem_u32(q_full)), "r"(kb * 64), "r"(0), "r"(j),
+                            "r"(pc.b * p.s_q)
+                            : "memory");
+                const int64_t row0 = p.seq_start[pc.b] + pc.tok_begin;
+                for (int t = 0; t < pc.n_tiles; ++t, ++gt) {
+                    const int s = gt & 1;
+                    const uint32_t ph = (gt >> 1) & 1;
+                    uint8_t* st = stage0 + s * L::kStageBytes;
+                    const int32_t row = (int32_t)(row0 + (int64_t)t * 128);
+                    if (!(ok = mbar_wait(&kempty[s], ph ^ 1, ab, 1))) break;
+                    mbar_expect_tx(&kfull[s], L::kKcBytes + L::kKrBytes);
+                    tma_load_3d(st, &tmK, 0, j, row, &kfull[s]);
+                    tma_load_3d(st + 16384, &tmK, 64, j, row, &kfull[s]);
+                    tma_load_2d(st + L::kKcBytes, &tmR, 0, row, &kfull[s]);
+                    if (!(ok = mbar_wait(&vempty[s], ph ^ 1, ab, 2))) break;
+                    mbar_expect_tx(&vfull[s], L::kVBytes);
+                    tma_load_3d(st + L::kKcBytes + L::kKrBytes, &tmV, 0, j, row, &vfull[s]);
+                    tma_load_3d(st + L::kKcBytes + L::kKrBytes + 16384, &tmV, 64, j, row, &vfull[s]);
+                }
+                ++pi;
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (n_tiles > 0 && elect_one()) {
+        if (elect_one()) {
             constexpr uint32_t idesc_qk = idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t idesc_pv = idesc_bf16(128, 128, 0, 1);
             const uint32_t q_addr = smem_u32(q_smem);
-            auto issue_qk = [&](int t) -> bool {
-                const int s = t & 1;
-                if (!mbar_wait(&kfull[s], (t >> 1) & 1, ab, 3)) return false;
+            auto issue_qk = [&](int n) -> bool {  // n: running tile number
+                const int s = n & 1;
+                if (!mbar_wait(&kfull[s], (n >> 1) & 1, ab, 3)) return false;
                 tc_fence_after();
                 const uint32_t st = smem_u32(stage0 + s * L::kStageBytes);
                 const uint32_t d = tmem_base + kColS + (uint32_t)s * 128;
@@ -159,23 +192,36 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
                 umma_commit(&kempty[s]);
                 return true;
             };
-            bool ok = mbar_wait(q_full, 0, ab, 4);
-            if (ok) ok = issue_qk(0);
-            for (int t = 0; t < n_tiles && ok; ++t) {
-                const int s = t & 1;
-                const uint32_t ph = (t >> 1) & 1;
-                if (t + 1 < n_tiles) ok = issue_qk(t + 1);
-                if (!ok) break;
-                if (!(ok = mbar_wait(&p_ready[s], ph, ab, 5))) break;
-                if (!(ok = mbar_wait(&vfull[s], ph, ab, 6))) break;
+            bool ok = true;
+            while (ok && walk.next(pc)) {
+                if (pc.n_tiles == 0) continue;
+                if (!(ok = mbar_wait(q_full, pi & 1, ab, 4))) break;
                 tc_fence_after();
-                const uint32_t v_addr = smem_u32(stage0 + s * L::kStageBytes + L::kKcBytes + L::kKrBytes);
+                if (!(ok = issue_qk(gt))) break;
+                for (int t = 0; t < pc.n_tiles && ok; ++t) {
+                    const int n = gt + t;
+                    const int s = n & 1;
+                    const uint32_t ph = (n >> 1) & 1;
+                    if (t + 1 < pc.n_tiles) {
+                        if (!(ok = issue_qk(n + 1))) break;
+                    } else {
+                        umma_commit(q_empty);  // every Q K^T of this piece has been issued
+                    }
+                    if (!(ok = mbar_wait(&p_ready[s], ph, ab, 5))) break;
+                    // the first P.V of a piece overwrites O: the previous piece's O must have been read
+                    if (t == 0 && pi > 0 && !(ok = mbar_wait(o_free, (pi - 1) & 1, ab, 14))) break;
+                    if (!(ok = mbar_wait(&vfull[s], ph, ab, 6))) break;
+                    tc_fence_after();
+                    const uint32_t v_addr = smem_u32(stage0 + s * L::kStageBytes + L::kKcBytes + L::kKrBytes);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    umma_ts(tmem_base + kColO, tmem_base + kColP + (uint32_t)s * 64 + ks * 8,
-                            desc_mnmajor_sw128(v_addr + ks * 2048, 16384), idesc_pv, (t | ks) != 0);
-                umma_commit(&vempty[s]);
-                umma_commit(&pv_done[s]);
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_ts(tmem_base + kColO, tmem_base + kColP + (uint32_t)s * 64 + ks * 8,
+                                desc_mnmajor_sw128(v_addr + ks * 2048, 16384), idesc_pv, (t | ks) != 0);
+                    umma_commit(&vempty[s]);
+                    umma_commit(&pv_done[s]);
+                }
+                gt += pc.n_tiles;
+                ++pi;
             }
         }
     } else {
@@ -187,17 +233,13 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
         const int pq = r / p.hpg_box;        // query position within the step
         const int il = r % p.hpg_box;        // head within the group
         const bool row_valid = il < p.hpg;
-        int32_t lim = visible_limit(T, p.s_q, pq);
-        if (lim > end) lim = end;
-        lim -= begin;                        // visible tokens of this unit, relative to its first row
         const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
         const int col0 = R < 32 ? q * 32 : f * R;  // first column of the warp's window (warp-uniform)
         const int sub = R < 32 ? lane / R : 0;     // which R-column sub-block of the window is this thread's
         auto owns = [&](int c) -> bool { return R >= 32 || (c / R) == sub; };
-        float m_used = -INFINITY, l = 0.f;
-        bool ok = true;
+        const int mcol = Lr & 31, mrow0 = Lr >> 5;  // merge: output column and first row of this thread
 
-        if (n_tiles > 0) {
+        {   // a thread only ever writes its own columns of P; everything else stays zero for good
             uint32_t z[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) z[i] = 0u;
@@ -206,122 +248,141 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
             tmem_wait_st();
         }
 
-        for (int t = 0; t < n_tiles && ok; ++t) {
-            const int s = t & 1;
-            ok = __all_sync(0xffffffffu, mbar_wait(&s_full[s], (t >> 1) & 1, ab, 7));
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t s_addr = lane_base + kColS + (uint32_t)s * 128 + col0;
-            const int tok0 = t * 128 + col0;
-            uint32_t x[CH];
-            float mx = -INFINITY;
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) {
-                tmem_ld<CH>(s_addr + ch * CH, x);
-                tmem_wait_ld();
-#pragma unroll
-                for (int c = 0; c < CH; ++c)
-                    if (owns(c) && tok0 + ch * CH + c < lim) mx = fmaxf(mx, __uint_as_float(x[c]));
-            }
-            const float m_t = mx * p.scale_log2;  // -inf when nothing is visible
-            const bool need = m_t > m_used + kRescaleThreshold;
-            const float factor = need ? ex2(m_used - m_t) : 1.f;  // ex2(-inf) = 0 on first use
-            if (__any_sync(0xffffffffu, need) && t > 0) {
-                // O is only touched between P.V(t-1) completing and P.V(t) being issued.  A warp may run one
-                // tile ahead of the others, so completions are counted on two alternating barriers: with a
-                // single one, parity alone could not tell "P.V(t-1) done" from "P.V(t-3) done".
-                ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(t - 1) & 1], ((t - 1) >> 1) & 1, ab, 8));
+        while (walk.next(pc)) {
+            const int32_t T = p.seqlens[pc.b];
+            const int64_t slot0 = (int64_t)pc.b * p.S;
+            // split slots this worker marks empty
+            if (f == 0 && row_valid)
+                for (int kk = pc.fill_begin; kk < pc.fill_end; ++kk)
+                    p.lse_part[((slot0 + kk) * p.s_q + pq) * p.h_q + (int64_t)j * p.hpg + il] = -INFINITY;
+            if (pc.n_tiles == 0 && p.balanced) continue;  // an empty sequence: its slots were marked above
+            int32_t lim = visible_limit(T, p.s_q, pq);
+            if (lim > pc.tok_end) lim = pc.tok_end;
+            lim -= pc.tok_begin;                 // visible tokens of this piece, relative to its first row
+            float m_used = -INFINITY, l = 0.f;
+            bool ok = true;
+
+            for (int t = 0; t < pc.n_tiles && ok; ++t) {
+                const int n = gt + t;
+                const int s = n & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(&s_full[s], (n >> 1) & 1, ab, 7));
                 if (!ok) break;
                 tc_fence_after();
-#pragma unroll 1
-                for (int c = 0; c < 128; c += 32) {
-                    uint32_t o[32];
-                    tmem_ld32(lane_base + kColO + c, o);
-                    tmem_wait_ld();
+                const uint32_t s_addr = lane_base + kColS + (uint32_t)s * 128 + col0;
+                const int tok0 = t * 128 + col0;
+                uint32_t x[CH];
+                float mx = -INFINITY;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-                    tmem_st32(lane_base + kColO + c, o);
-                }
-                tmem_wait_st();
-            }
-            if (need) {
-                l *= factor;
-                m_used = m_t;
-            }
-            const float m_sub = m_used == -INFINITY ? 0.f : m_used;
-            const uint32_t p_addr = lane_base + kColP + (uint32_t)s * 64 + col0 / 2;
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) {
-                if (NCH > 1) {
+                for (int ch = 0; ch < NCH; ++ch) {
                     tmem_ld<CH>(s_addr + ch * CH, x);
                     tmem_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < CH; ++c)
+                        if (owns(c) && tok0 + ch * CH + c < lim) mx = fmaxf(mx, __uint_as_float(x[c]));
                 }
-                uint32_t pk[CH / 2];
-#pragma unroll
-                for (int c = 0; c < CH; c += 2) {
-                    const int tok = tok0 + ch * CH + c;
-                    const bool mine = owns(c);  // R is even, so c and c+1 share an owner
-                    const float e0 = (mine && tok < lim) ? ex2(fmaf(__uint_as_float(x[c]), p.scale_log2, -m_sub)) : 0.f;
-                    const float e1 =
-                        (mine && tok + 1 < lim) ? ex2(fmaf(__uint_as_float(x[c + 1]), p.scale_log2, -m_sub)) : 0.f;
-                    l += e0 + e1;
-                    pk[c / 2] = pack_bf16(e0, e1);
-                }
-                tmem_st<CH / 2>(p_addr + ch * (CH / 2), pk);
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(&p_ready[s]);
-        }
-
-        // ------------------------------------------------------------------ merge the F replicas of each row
-        float* merge = reinterpret_cast<float*>(stage0);
-        if (n_tiles > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, ab, 9));
-        tc_fence_after();
-        sm_m[Lr] = m_used;
-        sm_l[Lr] = l;
-        named_bar_sync(1, 128);
-        float M = -INFINITY;
-#pragma unroll
-        for (int ff = 0; ff < F; ++ff) M = fmaxf(M, sm_m[ff * R + r]);
-        float Lt = 0.f;
-#pragma unroll
-        for (int ff = 0; ff < F; ++ff) {
-            const float mf = sm_m[ff * R + r];
-            if (mf > -INFINITY) Lt += sm_l[ff * R + r] * ex2(mf - M);
-        }
-        const bool live = ok && n_tiles > 0 && Lt > 0.f;
-        const float w = (live && m_used > -INFINITY) ? ex2(m_used - M) / Lt : 0.f;
-        if (n_tiles > 0 && ok) {
+                const float m_t = mx * p.scale_log2;  // -inf when nothing is visible
+                const bool need = m_t > m_used + kRescaleThreshold;
+                const float factor = need ? ex2(m_used - m_t) : 1.f;  // ex2(-inf) = 0 on first use
+                if (__any_sync(0xffffffffu, need) && t > 0) {
+                    // O is only touched between P.V(n-1) completing and P.V(n) being issued.  A warp may run one
+                    // tile ahead of the others, so completions are counted on two alternating barriers: with a
+                    // single one, parity alone could not tell "P.V(n-1) done" from "P.V(n-3) done".
+                    ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, ab, 8));
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll 1
-            for (int c = 0; c < 128; c += 32) {
+                    for (int c = 0; c < 128; c += 32) {
+                        uint32_t o[32];
+                        tmem_ld32(lane_base + kColO + c, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                        tmem_st32(lane_base + kColO + c, o);
+                    }
+                    tmem_wait_st();
+                }
+                if (need) {
+                    l *= factor;
+                    m_used = m_t;
+                }
+                const float m_sub = m_used == -INFINITY ? 0.f : m_used;
+                const uint32_t p_addr = lane_base + kColP + (uint32_t)s * 64 + col0 / 2;
+#pragma unroll
+                for (int ch = 0; ch < NCH; ++ch) {
+                    if (NCH > 1) {
+                        tmem_ld<CH>(s_addr + ch * CH, x);
+                        tmem_wait_ld();
+                    }
+                    uint32_t pk[CH / 2];
+#pragma unroll
+                    for (int c = 0; c < CH; c += 2) {
+                        const int tok = tok0 + ch * CH + c;
+                        const bool mine = owns(c);  // R is even, so c and c+1 share an owner
+                        const float e0 = (mine && tok < lim) ? ex2(fmaf(__uint_as_float(x[c]), p.scale_log2, -m_sub)) : 0.f;
+                        const float e1 =
+                            (mine && tok + 1 < lim) ? ex2(fmaf(__uint_as_float(x[c + 1]), p.scale_log2, -m_sub)) : 0.f;
+                        l += e0 + e1;
+                        pk[c / 2] = pack_bf16(e0, e1);
+                    }
+                    tmem_st<CH / 2>(p_addr + ch * (CH / 2), pk);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_ready[s]);
+            }
+
+            // -------------------------------------------------------------- merge the F replicas of each row
+            const int n_last = gt + pc.n_tiles - 1;
+            if (pc.n_tiles > 0 && ok)
+                ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[n_last & 1], (n_last >> 1) & 1, ab, 9));
+            tc_fence_after();
+            sm_m[Lr] = m_used;
+            sm_l[Lr] = l;
+            named_bar_sync(1, 128);
+            float M = -INFINITY;
+#pragma unroll
+            for (int ff = 0; ff < F; ++ff) M = fmaxf(M, sm_m[ff * R + r]);
+            float Lt = 0.f;
+#pragma unroll
+            for (int ff = 0; ff < F; ++ff) {
+                const float mf = sm_m[ff * R + r];
+                if (mf > -INFINITY) Lt += sm_l[ff * R + r] * ex2(mf - M);
+            }
+            const bool live = ok && pc.n_tiles > 0 && Lt > 0.f;
+            const float w = (live && m_used > -INFINITY) ? ex2(m_used - M) / Lt : 0.f;
+            const int64_t out_row0 = ((slot0 + pc.k) * p.s_q) * p.h_q + (int64_t)j * p.hpg;
+            // 32 output columns at a time through the merge buffer: lane rows in, (row, column) sums out
+#pragma unroll 1
+            for (int c4 = 0; c4 < 4; ++c4) {
                 uint32_t o[32];
-                tmem_ld32(lane_base + kColO + c, o);
-                tmem_wait_ld();
-                float4* dst = reinterpret_cast<float4*>(merge + Lr * L::kMergeStride + c);
+                if (pc.n_tiles > 0 && ok) {  // warp-uniform
+                    tmem_ld32(lane_base + kColO + c4 * 32, o);
+                    tmem_wait_ld();
+                }
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    dst[i] = make_float4(w == 0.f ? 0.f : __uint_as_float(o[4 * i]) * w,
-                                         w == 0.f ? 0.f : __uint_as_float(o[4 * i + 1]) * w,
-                                         w == 0.f ? 0.f : __uint_as_float(o[4 * i + 2]) * w,
-                                         w == 0.f ? 0.f : __uint_as_float(o[4 * i + 3]) * w);
-            }
-        }
-        named_bar_sync(1, 128);
-        // thread Lr owns output column Lr of every row; lane rows r < R write the LSE
-        const int64_t out_row0 = ((int64_t)(b * p.S + k) * p.s_q) * p.h_q + (int64_t)j * p.hpg;
-        for (int rr = 0; rr < R; ++rr) {
-            const int pp = rr / p.hpg_box, ii = rr % p.hpg_box;
-            if (ii >= p.hpg) continue;
-            float acc = 0.f;
-            if (n_tiles > 0 && ok) {
+                for (int i = 0; i < 32; ++i) merge[Lr * L::kMergePitch + i] = w == 0.f ? 0.f : __uint_as_float(o[i]) * w;
+                if (c4 == 3) {  // O has been read: the next piece's first P.V may overwrite it
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(o_free);
+                }
+                named_bar_sync(1, 128);
+                for (int rr = mrow0; rr < R; rr += 4) {
+                    const int pp = rr / p.hpg_box, ii = rr % p.hpg_box;
+                    if (ii >= p.hpg) continue;
+                    float acc = 0.f;
 #pragma unroll
-                for (int ff = 0; ff < F; ++ff) acc += merge[(ff * R + rr) * L::kMergeStride + Lr];
+                    for (int ff = 0; ff < F; ++ff) acc += merge[(ff * R + rr) * L::kMergePitch + mcol];
+                    p.o_part[(out_row0 + (int64_t)pp * p.h_q + ii) * 128 + c4 * 32 + mcol] = acc;
+                }
+                named_bar_sync(1, 128);
             }
-            p.o_part[(out_row0 + (int64_t)pp * p.h_q + ii) * 128 + Lr] = acc;
+            if (f == 0 && row_valid)
+                p.lse_part[out_row0 + (int64_t)pq * p.h_q + il] = live ? (M + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
+            gt += pc.n_tiles;
+            if (pc.n_tiles > 0) ++pi;
         }
-        if (f == 0 && row_valid)
-            p.lse_part[out_row0 + (int64_t)pq * p.h_q + il] = live ? (M + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
     }
     tc_fence_before();
     __syncthreads();

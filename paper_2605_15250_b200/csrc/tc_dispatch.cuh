@@ -61,8 +61,8 @@ inline int32_t tc_balanced_workers(const gqla_dims& d, int32_t s_q, int32_t path
     const int sms = sm_count();
     if (sms <= 0) return 0;
     if (path == 1) return sms / d.g > 0 ? sms / d.g : 0;
-    const int row_blocks = (s_q * d.h_q + 127) / 128;
-    return (sms / 2) / row_blocks > 0 ? (sms / 2) / row_blocks : 0;
+    (void)s_q;
+    return 0;  // absorb path: fixed plan
 }
 
 inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t N, const void* cache,
@@ -163,6 +163,7 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
     if (!tc_covers(d, GQLA_BF16, s_q, 0) || !stride_ok(cache_row_stride) || cache_rows > 0x7fffffffLL ||
         cache_rows < 1)
         return GQLA_ERR_UNSUPPORTED;
+    if (S < 0) S = -S;
     const int rows_total = s_q * d.h_q;
     const int row_blocks = (rows_total + 127) / 128;
     const int64_t pairs = (int64_t)B * S * row_blocks;
@@ -197,7 +198,7 @@ inline cudaError_t gqa_launch(const tc::GqaParams& p, const CUtensorMap& q, cons
     auto kern = tc::decode_gqa_tc_kernel<R>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::GqaSmem::kTotal);
     if (e != cudaSuccess) return e;
-    kern<<<grid, 192, tc::GqaSmem::kTotal, st>>>(p, q, k, r, v);
+    kern<<<grid, tc::GqaSmem::kThreads, tc::GqaSmem::kTotal, st>>>(p, q, k, r, v);
     return cudaGetLastError();
 }
 
@@ -207,7 +208,11 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
                                  float* lse_part, int32_t* status, cudaStream_t st) {
     if (!tc_covers(d, GQLA_BF16, s_q, 1) || !stride_ok(k_r_row_stride) || n_rows > 0x7fffffffLL || n_rows < 1)
         return GQLA_ERR_UNSUPPORTED;
-    const int64_t units = (int64_t)B * S * d.g;
+    // S < 0: balanced plan with -S slots per sequence, W persistent CTAs per group
+    const int32_t workers = S < 0 ? tc_balanced_workers(d, s_q, 1) : 0;
+    const bool balanced = S < 0 && workers > 0;
+    if (S < 0) S = -S;
+    const int64_t units = balanced ? (int64_t)workers * d.g : (int64_t)B * S * d.g;
     if (units > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     const int hpg = d.h_q / d.g;
     int hpg_box = 0;
@@ -235,6 +240,7 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
     }
     tc::GqaParams p{};
     p.B = B; p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpg_box = hpg_box;
+    p.balanced = balanced ? 1 : 0; p.W = workers;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.seq_start = seq_start; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
     cudaError_t e;

@@ -90,6 +90,64 @@ def test_end_to_end_mid(policy, dims, s_q, S):
     end_to_end(w, seqlens, S, q_gain=1.0, alias_k_r=False)
 
 
+def _balanced_gqa_case(w, seqlens, S, q_gain=4.0):
+    """GQA path under the balanced plan: every non-empty slot against the oracle's partial on the
+    plan the oracle states, unused slots marked -inf, and the merged output against the definition."""
+    from oracle import gqla_oracle as O
+    from tests.parity_util import assert_close, dims_of
+    od, bd = dims_of(w)
+    x = synth.make_inputs(w, seqlens=seqlens, q_gain=q_gain)
+    f = {k: synth.to_f64(v) for k, v in x.items() if k not in ("seq_start", "seqlens")}
+    ss, sl = x["seq_start"].numpy(), x["seqlens"].numpy()
+    W = B.gqla_balanced_workers(bd, torch.bfloat16, w.s_q, "gqa")
+    assert W == torch.cuda.get_device_properties(0).multi_processor_count // w.g
+    plans = O.balanced_plan([int(t) for t in sl], S, W)
+    assert plans == B.gqla_balanced_plan([int(t) for t in sl], S, W)[0]
+    cache = x["cache"].cuda()
+    N = cache.shape[0]
+    k_c = torch.empty((N, w.g, w.d_h), dtype=torch.bfloat16, device="cuda")
+    v = torch.empty_like(k_c)
+    B.gqla_expand_cache(bd, cache, x["w_uk"].cuda(), x["w_uv"].cuda(), k_c, v, None)
+    q = torch.cat([x["q_c"], x["q_r"]], -1).contiguous()
+    o_part = torch.full((w.batch, S, w.s_q, w.h_q, w.d_h), float("nan"), dtype=torch.float32, device="cuda")
+    lse_part = torch.full((w.batch, S, w.s_q, w.h_q), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.gqla_decode_gqa(bd, q.cuda(), k_c, v, cache[:, w.r_kv:], x["seq_start"].cuda(), x["seqlens"].cuda(), w.scale, -S,
+                      o_part, lse_part, status)
+    out = torch.empty((w.batch, w.s_q, w.h_q, w.d_h), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((w.batch, w.s_q, w.h_q), dtype=torch.float32, device="cuda")
+    B.gqla_combine_splits(o_part, lse_part, out, lse)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    # the oracle on the library's own (bf16) expanded cache, so that only the attention is compared
+    kc64, v64 = synth.to_f64(k_c), synth.to_f64(v)
+    op_ref, lp_ref = O.decode_gqa_partials(od, synth.to_f64(q), kc64, v64, f["cache"][:, w.r_kv:], ss, sl, w.s_q, w.scale,
+                                           S, plans)
+    got_o, got_l = o_part.cpu().numpy(), lse_part.cpu().numpy()
+    live = np.array([[hi > lo for lo, hi in plan] for plan in plans])
+    assert np.isneginf(got_l[~live]).all(), "unused slots must carry lse = -inf"
+    assert_close(got_l, lp_ref, "balanced lse_part")
+    assert_close(got_o[live], op_ref[live], "balanced o_part")
+    o_ref, l_ref = O.combine_splits(op_ref, lp_ref)
+    assert_close(out.float().cpu().numpy(), o_ref, "balanced merged output")
+    assert_close(lse.cpu().numpy(), l_ref, "balanced merged lse")
+
+
+@pytest.mark.parametrize("s_q", [1, 2])
+@pytest.mark.parametrize("S", [2, 5])
+def test_gqa_balanced_plan_canonical(s_q, S):
+    w = _wl("bal", 9, s_q, 111, **CANON)
+    _balanced_gqa_case(w, np.array([1, 0, 63, 2050, 65, 1000, 0, 129, 5000], dtype=np.int32), S)
+
+
+@pytest.mark.parametrize("s_q", [1, 2])
+def test_gqa_balanced_plan_llama_more_workers_than_tiles(s_q):
+    w = _wl("bal2", 3, s_q, 112, **LLAMA)
+    _balanced_gqa_case(w, np.array([130, 0, 300], dtype=np.int32), 2)
+    w = _wl("bal3", 40, s_q, 113, **LLAMA)
+    _balanced_gqa_case(w, synth.make_seqlens(w.with_(seqlen_range=(0, 1500))), 3)
+
+
 def test_two_gpu_paths_agree_with_each_other():
     """Same weights, same latent: the two paths' GPU outputs differ by at most twice the
     tolerance (each is within it of the same oracle value)."""
