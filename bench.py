@@ -58,7 +58,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                          "-lms", "20", "-i", str(self.index)], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -207,7 +207,7 @@ def run_ours(args):
     total_tokens = int(x["seqlens"].sum())
     kern_a = B.kernel_for(dec.dims, torch.bfloat16, w1.s_q, "absorb")
     n_sm = torch.cuda.get_device_properties(local_rank).multi_processor_count
-    S_a = args.splits if args.splits > 0 else pick_splits(w1.batch, (w1.s_q * w1.h_q + 127) // 128, w1.seqlen, n_sm // 2)
+    S_a = args.splits if args.splits != 0 else pick_splits(w1.batch, (w1.s_q * w1.h_q + 127) // 128, w1.seqlen, n_sm // 2)
 
     def absorb_step():
         dec.absorb_step(q_c, q_r, S_a)
@@ -294,15 +294,29 @@ def run_ours(args):
     x2 = synth.make_inputs(w2)
     q2 = torch.cat([x2["q_c"], x2["q_r"]], -1).contiguous().to(dev)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dec.expand_cache()  # first call also loads the kernel; the second is timed
+    torch.cuda.synchronize()
     ev0.record()
-    dec.expand_cache()
+    B.gqla_expand_cache(dec.dims, dec.cache, dec.w_uk, dec.w_uv, dec.k_c, dec.v, None)
     ev1.record()
     torch.cuda.synchronize()
     expand_ms = ev0.elapsed_time(ev1)
     kern_g = B.kernel_for(dec.dims, torch.bfloat16, w2.s_q, "gqa")
-    S_g = args.splits if args.splits > 0 else pick_splits(w2.batch, w2.g, w2.seqlen, n_sm)
-    og_part = dec._get("o_part_g", (w2.batch, S_g, w2.s_q, w2.h_q, w2.d_h), torch.float32)
-    lg_part = dec._get("lse_part_g", (w2.batch, S_g, w2.s_q, w2.h_q), torch.float32)
+    # balanced plan (negative split count = slots per sequence) unless a fixed split count is forced
+    W_g = B.gqla_balanced_workers(dec.dims, torch.bfloat16, w2.s_q, "gqa")
+    if args.splits != 0:
+        S_g = args.splits
+    elif W_g > 0:
+        S_g = -2
+    else:
+        S_g = pick_splits(w2.batch, w2.g, w2.seqlen, n_sm)
+    if S_g < 0:
+        plan_g, _ = B.gqla_balanced_plan([int(t) for t in x["seqlens"]], -S_g, W_g)
+        pieces_g = sum(1 for pl in plan_g for lo, hi in pl if hi > lo) / w2.batch
+    else:
+        pieces_g = S_g
+    og_part = dec._get("o_part_g", (w2.batch, abs(S_g), w2.s_q, w2.h_q, w2.d_h), torch.float32)
+    lg_part = dec._get("lse_part_g", (w2.batch, abs(S_g), w2.s_q, w2.h_q), torch.float32)
     og = dec._get("o_g", (w2.batch, w2.s_q, w2.h_q, w2.d_h), torch.bfloat16)
     gev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     it["i"] = 0
@@ -322,13 +336,14 @@ def run_ours(args):
     dec.check_status()
     gk_ms = statistics.mean(a.elapsed_time(b) for a, b in gev)
     gbytes = acct.decode_kernel_bytes("gqa", h_q=w2.h_q, g=w2.g, d_h=w2.d_h, r_kv=w2.r_kv, d_r=w2.d_r, s_q=w2.s_q,
-                                      batch=w2.batch, total_tokens=total_tokens, num_splits=S_g)
+                                      batch=w2.batch, total_tokens=total_tokens, num_splits=pieces_g)
     gflops = acct.gqa_flops(w2.h_q, w2.d_h, w2.d_r, w2.s_q, total_tokens)
     g_gbs = gbytes / (gk_ms * 1e-3) / 1e9
     paths = {
         "absorb": {"workload": "C1", "s_q": w1.s_q, "num_splits": S_a, "kernel": kern_a, "ms_per_step": ms_per_step,
                    "tokens_per_s": value, "decode_kernel_us": kern_ms * 1e3, "gbs": gbs, "tflops": tfs},
-        "gqa": {"workload": "C2", "s_q": w2.s_q, "num_splits": S_g, "kernel": kern_g, "ms_per_step": gqa_ms,
+        "gqa": {"workload": "C2", "s_q": w2.s_q, "num_splits": S_g,
+                "plan": "balanced" if S_g < 0 else "fixed", "pieces_per_sequence": pieces_g, "kernel": kern_g, "ms_per_step": gqa_ms,
                 "tokens_per_s": world * w2.batch * w2.s_q / (gqa_ms * 1e-3), "decode_kernel_us": gk_ms * 1e3,
                 "gbs": g_gbs, "tflops": gflops / (gk_ms * 1e-3) / 1e12,
                 "roofline": {"bound": "hbm", "achieved": g_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -368,7 +383,8 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--splits", type=int, default=0, help="force the split count (0 = automatic)")
+    ap.add_argument("--splits", type=int, default=0,
+                    help="force the split count of both paths (0 = automatic; negative = balanced plan with that many slots)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

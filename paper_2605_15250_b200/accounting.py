@@ -27,8 +27,9 @@ def gqa_flops(h_q: int, d_h: int, d_r: int, s_q: int, total_tokens: int) -> int:
 
 
 def decode_kernel_bytes(path: str, *, h_q: int, g: int, d_h: int, r_kv: int, d_r: int, s_q: int, batch: int,
-                        total_tokens: int, num_splits: int, elem: int = 2) -> int:
-    """Algorithmic bytes of ONE decode-kernel launch: cache once + queries + fp32 partials and LSE."""
+                        total_tokens: int, num_splits: float, elem: int = 2) -> int:
+    """Algorithmic bytes of ONE decode-kernel launch: cache once + queries + fp32 partials and LSE.
+    num_splits = partials written per sequence (under the balanced plan: live pieces / batch)."""
     rows = batch * s_q * h_q
     if path == "absorb":
         cache = absorb_cache_bytes(r_kv, d_r, total_tokens, elem)
@@ -38,7 +39,7 @@ def decode_kernel_bytes(path: str, *, h_q: int, g: int, d_h: int, r_kv: int, d_r
         cache = gqa_cache_bytes(g, d_h, d_r, total_tokens, elem)
         q = elem * rows * (d_h + d_r)
         part = 4 * rows * num_splits * (d_h + 1)
-    return cache + q + part
+    return int(cache + q + part)
 
 
 def roofline_time(flops: float, nbytes: float, peak_flops: float, bw: float) -> float:

@@ -54,9 +54,10 @@ class GqlaDecoder:
     # ---- absorb path ----
     def absorb_step(self, q_c: torch.Tensor, q_r: torch.Tensor, num_splits: int = 1, want_lse: bool = False):
         Bn, s_q = q_c.shape[0], q_c.shape[1]
+        slots = abs(num_splits)  # num_splits < 0: balanced plan with that many slots per sequence
         q_hat = self._get("q_hat", (Bn, s_q, self.h_q, self.r_kv + self.d_r), self.dtype)
-        o_part = self._get("o_part_a", (Bn, num_splits, s_q, self.h_q, self.r_kv), torch.float32)
-        lse_part = self._get("lse_part_a", (Bn, num_splits, s_q, self.h_q), torch.float32)
+        o_part = self._get("o_part_a", (Bn, slots, s_q, self.h_q, self.r_kv), torch.float32)
+        lse_part = self._get("lse_part_a", (Bn, slots, s_q, self.h_q), torch.float32)
         o_hat = self._get("o_hat", (Bn, s_q, self.h_q, self.r_kv), self.dtype)
         lse = self._get("lse_a", (Bn, s_q, self.h_q), torch.float32) if want_lse else None
         o = self._get("o_a", (Bn, s_q, self.h_q, self.d_h), self.dtype)
@@ -73,8 +74,9 @@ class GqlaDecoder:
         if self.k_c is None:
             raise B.GqlaError("expand_cache() must run before the GQA path")
         Bn, s_q = q.shape[0], q.shape[1]
-        o_part = self._get("o_part_g", (Bn, num_splits, s_q, self.h_q, self.d_h), torch.float32)
-        lse_part = self._get("lse_part_g", (Bn, num_splits, s_q, self.h_q), torch.float32)
+        slots = abs(num_splits)
+        o_part = self._get("o_part_g", (Bn, slots, s_q, self.h_q, self.d_h), torch.float32)
+        lse_part = self._get("lse_part_g", (Bn, slots, s_q, self.h_q), torch.float32)
         lse = self._get("lse_g", (Bn, s_q, self.h_q), torch.float32) if want_lse else None
         o = self._get("o_g", (Bn, s_q, self.h_q, self.d_h), self.dtype)
         B.gqla_decode_gqa(self.dims, q, self.k_c, self.v, self.k_r, self.seq_start, self.seqlens, self.scale,
