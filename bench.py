@@ -207,7 +207,18 @@ def run_ours(args):
     total_tokens = int(x["seqlens"].sum())
     kern_a = B.kernel_for(dec.dims, torch.bfloat16, w1.s_q, "absorb")
     n_sm = torch.cuda.get_device_properties(local_rank).multi_processor_count
-    S_a = args.splits if args.splits != 0 else pick_splits(w1.batch, (w1.s_q * w1.h_q + 127) // 128, w1.seqlen, n_sm // 2)
+    W_a = B.gqla_balanced_workers(dec.dims, torch.bfloat16, w1.s_q, "absorb")
+    if args.splits != 0:
+        S_a = args.splits
+    elif W_a > 0 and args.plan != "fixed":
+        S_a = -3
+    else:
+        S_a = pick_splits(w1.batch, (w1.s_q * w1.h_q + 127) // 128, w1.seqlen, n_sm // 2)
+    if S_a < 0:
+        plan_a, _ = B.gqla_balanced_plan([int(t) for t in x["seqlens"]], -S_a, W_a)
+        pieces_a = sum(1 for pl in plan_a for lo, hi in pl if hi > lo) / w1.batch
+    else:
+        pieces_a = S_a
 
     def absorb_step():
         dec.absorb_step(q_c, q_r, S_a)
@@ -218,8 +229,8 @@ def run_ours(args):
 
     # dominant kernel alone, timed live with events around each launch inside the timed region
     q_hat = dec._get("q_hat", (w1.batch, w1.s_q, w1.h_q, w1.d_abs), torch.bfloat16)
-    o_part = dec._get("o_part_a", (w1.batch, S_a, w1.s_q, w1.h_q, w1.r_kv), torch.float32)
-    lse_part = dec._get("lse_part_a", (w1.batch, S_a, w1.s_q, w1.h_q), torch.float32)
+    o_part = dec._get("o_part_a", (w1.batch, abs(S_a), w1.s_q, w1.h_q, w1.r_kv), torch.float32)
+    lse_part = dec._get("lse_part_a", (w1.batch, abs(S_a), w1.s_q, w1.h_q), torch.float32)
     o_hat = dec._get("o_hat", (w1.batch, w1.s_q, w1.h_q, w1.r_kv), torch.bfloat16)
     o_out = dec._get("o_a", (w1.batch, w1.s_q, w1.h_q, w1.d_h), torch.bfloat16)
     kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
@@ -246,7 +257,7 @@ def run_ours(args):
     value = world * w1.batch * w1.s_q / (ms_per_step * 1e-3)
 
     kbytes = acct.decode_kernel_bytes("absorb", h_q=w1.h_q, g=w1.g, d_h=w1.d_h, r_kv=w1.r_kv, d_r=w1.d_r,
-                                      s_q=w1.s_q, batch=w1.batch, total_tokens=total_tokens, num_splits=S_a)
+                                      s_q=w1.s_q, batch=w1.batch, total_tokens=total_tokens, num_splits=pieces_a)
     kflops = acct.absorb_flops(w1.h_q, w1.r_kv, w1.d_r, w1.s_q, total_tokens)
     t_mem = kbytes / (peaks["hbm_gbs"] * 1e9)
     t_mma = kflops / (peaks["bf16_tflops"] * 1e12)
@@ -306,7 +317,7 @@ def run_ours(args):
     W_g = B.gqla_balanced_workers(dec.dims, torch.bfloat16, w2.s_q, "gqa")
     if args.splits != 0:
         S_g = args.splits
-    elif W_g > 0:
+    elif W_g > 0 and args.plan != "fixed":
         S_g = -2
     else:
         S_g = pick_splits(w2.batch, w2.g, w2.seqlen, n_sm)
@@ -340,7 +351,8 @@ def run_ours(args):
     gflops = acct.gqa_flops(w2.h_q, w2.d_h, w2.d_r, w2.s_q, total_tokens)
     g_gbs = gbytes / (gk_ms * 1e-3) / 1e9
     paths = {
-        "absorb": {"workload": "C1", "s_q": w1.s_q, "num_splits": S_a, "kernel": kern_a, "ms_per_step": ms_per_step,
+        "absorb": {"workload": "C1", "s_q": w1.s_q, "num_splits": S_a,
+                   "plan": "balanced" if S_a < 0 else "fixed", "pieces_per_sequence": pieces_a, "kernel": kern_a, "ms_per_step": ms_per_step,
                    "tokens_per_s": value, "decode_kernel_us": kern_ms * 1e3, "gbs": gbs, "tflops": tfs},
         "gqa": {"workload": "C2", "s_q": w2.s_q, "num_splits": S_g,
                 "plan": "balanced" if S_g < 0 else "fixed", "pieces_per_sequence": pieces_g, "kernel": kern_g, "ms_per_step": gqa_ms,
@@ -385,6 +397,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--splits", type=int, default=0,
                     help="force the split count of both paths (0 = automatic; negative = balanced plan with that many slots)")
+    ap.add_argument("--plan", default="auto", choices=["auto", "fixed"],
+                    help="auto: balanced split plan where the kernels support it; fixed: equal chunks per sequence")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

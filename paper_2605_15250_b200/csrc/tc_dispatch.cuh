@@ -53,6 +53,8 @@ inline int sm_count() {
     return cached[dev];
 }
 
+inline int absorb_resident_pairs();
+
 // Workers of the balanced plan: the GQA path runs one CTA per SM and keeps the cut points of all g
 // groups identical (so the CTAs of the g groups read one k_R tile together): W = SMs / g workers per
 // group.  The absorb path runs one CTA pair per two SMs: W = (SMs / 2) / row_blocks per row block.
@@ -61,8 +63,9 @@ inline int32_t tc_balanced_workers(const gqla_dims& d, int32_t s_q, int32_t path
     const int sms = sm_count();
     if (sms <= 0) return 0;
     if (path == 1) return sms / d.g > 0 ? sms / d.g : 0;
-    (void)s_q;
-    return 0;  // absorb path: fixed plan
+    const int row_blocks = (s_q * d.h_q + 127) / 128;
+    const int pairs = absorb_resident_pairs();
+    return pairs / row_blocks > 0 ? pairs / row_blocks : 0;
 }
 
 inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t N, const void* cache,
@@ -163,10 +166,13 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
     if (!tc_covers(d, GQLA_BF16, s_q, 0) || !stride_ok(cache_row_stride) || cache_rows > 0x7fffffffLL ||
         cache_rows < 1)
         return GQLA_ERR_UNSUPPORTED;
-    if (S < 0) S = -S;
     const int rows_total = s_q * d.h_q;
     const int row_blocks = (rows_total + 127) / 128;
-    const int64_t pairs = (int64_t)B * S * row_blocks;
+    // S < 0: balanced plan with -S slots per sequence, W persistent pairs per row block
+    const int32_t workers = S < 0 ? tc_balanced_workers(d, s_q, 0) : 0;
+    const bool balanced = S < 0 && workers > 0;
+    if (S < 0) S = -S;
+    const int64_t pairs = balanced ? (int64_t)workers * row_blocks : (int64_t)B * S * row_blocks;
     if (2 * pairs > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     CUtensorMap tmQ, tmC;
     {
@@ -183,6 +189,7 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
     }
     tc::AbsorbParams p{};
     p.B = B; p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.rows_total = rows_total; p.row_blocks = row_blocks;
+    p.balanced = balanced ? 1 : 0; p.W = workers;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.seq_start = seq_start; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
     auto kern = tc::decode_absorb_tc_kernel<0>;
@@ -190,6 +197,39 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
         return GQLA_ERR_CUDA;
     kern<<<(unsigned)(2 * pairs), tc::AbsorbSmem::kThreads, tc::AbsorbSmem::kTotal, st>>>(p, tmQ, tmC);
     return cudaGetLastError() == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
+}
+
+// CTA pairs of the absorb kernel that can be resident at once on the current device (cached).
+inline int absorb_resident_pairs() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (cached[dev] == 0) {
+        auto kern = tc::decode_absorb_tc_kernel<0>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AbsorbSmem::kTotal) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return 0;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * 148, 1, 1);
+        cfg.blockDim = dim3(tc::AbsorbSmem::kThreads, 1, 1);
+        cfg.dynamicSmemBytes = tc::AbsorbSmem::kTotal;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            const int sms = sm_count();
+            n = sms / 2;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
 }
 
 template <int R>

@@ -148,6 +148,54 @@ def test_gqa_balanced_plan_llama_more_workers_than_tiles(s_q):
     _balanced_gqa_case(w, synth.make_seqlens(w.with_(seqlen_range=(0, 1500))), 3)
 
 
+def _balanced_absorb_case(w, seqlens, S, q_gain=4.0):
+    """Absorb path under the balanced plan: same checks as _balanced_gqa_case."""
+    from oracle import gqla_oracle as O
+    from tests.parity_util import assert_close, dims_of
+    od, bd = dims_of(w)
+    x = synth.make_inputs(w, seqlens=seqlens, q_gain=q_gain)
+    f = {k: synth.to_f64(v) for k, v in x.items() if k not in ("seq_start", "seqlens")}
+    ss, sl = x["seq_start"].numpy(), x["seqlens"].numpy()
+    W = B.gqla_balanced_workers(bd, torch.bfloat16, w.s_q, "absorb")
+    assert W >= 1
+    plans = O.balanced_plan([int(t) for t in sl], S, W)
+    q_hat = torch.from_numpy(O.absorb_q(od, f["q_c"], f["q_r"], f["w_uk"])).to(torch.bfloat16)
+    o_part = torch.full((w.batch, S, w.s_q, w.h_q, w.r_kv), float("nan"), dtype=torch.float32, device="cuda")
+    lse_part = torch.full((w.batch, S, w.s_q, w.h_q), float("nan"), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.gqla_decode_absorb(bd, q_hat.cuda(), x["cache"].cuda(), x["seq_start"].cuda(), x["seqlens"].cuda(), w.scale, -S,
+                         o_part, lse_part, status)
+    out = torch.empty((w.batch, w.s_q, w.h_q, w.r_kv), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((w.batch, w.s_q, w.h_q), dtype=torch.float32, device="cuda")
+    B.gqla_combine_splits(o_part, lse_part, out, lse)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    op_ref, lp_ref = O.decode_absorb_partials(od, synth.to_f64(q_hat), f["cache"], ss, sl, w.s_q, w.scale, S, plans)
+    got_o, got_l = o_part.cpu().numpy(), lse_part.cpu().numpy()
+    live = np.array([[hi > lo for lo, hi in plan] for plan in plans])
+    assert np.isneginf(got_l[~live]).all(), "unused slots must carry lse = -inf"
+    assert_close(got_l, lp_ref, "balanced lse_part")
+    assert_close(got_o[live], op_ref[live], "balanced o_part")
+    o_ref, l_ref = O.combine_splits(op_ref, lp_ref)
+    assert_close(out.float().cpu().numpy(), o_ref, "balanced merged output")
+    assert_close(lse.cpu().numpy(), l_ref, "balanced merged lse")
+
+
+@pytest.mark.parametrize("s_q", [1, 2])
+@pytest.mark.parametrize("S", [2, 5])
+def test_absorb_balanced_plan_canonical(s_q, S):
+    w = _wl("abal", 9, s_q, 121, **CANON)
+    _balanced_absorb_case(w, np.array([1, 0, 63, 2050, 65, 1000, 0, 129, 5000], dtype=np.int32), S)
+
+
+@pytest.mark.parametrize("s_q", [1, 2])
+def test_absorb_balanced_plan_llama(s_q):
+    w = _wl("abal2", 3, s_q, 122, **LLAMA)
+    _balanced_absorb_case(w, np.array([130, 0, 300], dtype=np.int32), 2)
+    w = _wl("abal3", 200, s_q, 123, **LLAMA)
+    _balanced_absorb_case(w, synth.make_seqlens(w.with_(seqlen_range=(0, 1500))), 3)
+
+
 def test_two_gpu_paths_agree_with_each_other():
     """Same weights, same latent: the two paths' GPU outputs differ by at most twice the
     tolerance (each is within it of the same oracle value)."""
