@@ -208,9 +208,12 @@ def run_ours(args):
     kern_a = B.kernel_for(dec.dims, torch.bfloat16, w1.s_q, "absorb")
     n_sm = torch.cuda.get_device_properties(local_rank).multi_processor_count
     W_a = B.gqla_balanced_workers(dec.dims, torch.bfloat16, w1.s_q, "absorb")
+    # Absorb path: the balanced plan pays one more 128 KB output tile per cut, so it is only taken when the
+    # fixed plan with one split per sequence would leave more than a fifth of the CTA pairs idle.
+    units_a = w1.batch * ((w1.s_q * w1.h_q + 127) // 128)
     if args.splits != 0:
         S_a = args.splits
-    elif W_a > 0 and args.plan != "fixed":
+    elif W_a > 0 and args.plan != "fixed" and units_a < 0.8 * (n_sm // 2):
         S_a = -3
     else:
         S_a = pick_splits(w1.batch, (w1.s_q * w1.h_q + 127) // 128, w1.seqlen, n_sm // 2)
