@@ -130,8 +130,10 @@ __global__ void __launch_bounds__(128) combine_generic_kernel(int32_t B, int32_t
     if (lse != nullptr && threadIdx.x == 0) lse[r] = dead ? -INFINITY : mx + logf(den);
 }
 
-// Vectorised log-sum-exp merge for d_out % 4 == 0: one warp per (b, row); 16-byte loads of the
-// partials, each lane owning every 32nd float4 of the row.  Same arithmetic as the kernel above.
+// Vectorised log-sum-exp merge for d_out % 4 == 0: one thread per (row, four output columns).  Every
+// thread of a row recomputes the row's S weights from lse_part (a handful of cached, broadcast loads),
+// so there is no cross-thread step and all its 16-byte loads of the partials are independent and in
+// flight together; consecutive threads read consecutive float4, i.e. whole rows are streamed.
 __device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
 __device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {
     __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
@@ -140,55 +142,46 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {
     u.y = *reinterpret_cast<uint32_t*>(&hi);
     *reinterpret_cast<uint2*>(p) = u;
 }
+__device__ __forceinline__ float4 ld_stream4(const float* p) {  // read once: do not keep in L1
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "l"(p));
+    return v;
+}
 template <typename TO>
 __global__ void __launch_bounds__(256) combine_vec_kernel(int64_t rows, int32_t rows_per_seq, int32_t S, int32_t d_out,
                                                           const float* __restrict__ o_part,
                                                           const float* __restrict__ lse_part, TO* __restrict__ out,
                                                           float* __restrict__ lse) {
-    const int lane = threadIdx.x & 31;
-    const int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int32_t vec_per_row = d_out >> 2;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t r = idx / vec_per_row;
     if (r >= rows) return;
+    const int c = (int)(idx % vec_per_row) << 2;
     const int64_t b = r / rows_per_seq;
     const int rr = (int)(r % rows_per_seq);
     const float* lp = lse_part + b * S * rows_per_seq + rr;
     float mx = -INFINITY;
-    for (int k = lane; k < S; k += 32) mx = fmaxf(mx, lp[(int64_t)k * rows_per_seq]);
-    mx = warp_max(mx);
+    for (int k = 0; k < S; ++k) mx = fmaxf(mx, __ldg(lp + (int64_t)k * rows_per_seq));
     const bool dead = !(mx > -INFINITY);
-    float den = 0.f;
-    for (int k = lane; k < S; k += 32) den += dead ? 0.f : expf(lp[(int64_t)k * rows_per_seq] - mx);
-    den = warp_sum(den);
-    const float inv = den > 0.f ? 1.f / den : 0.f;
-    const float* op = o_part + (b * S * rows_per_seq + rr) * d_out;
+    const float* op = o_part + (b * S * rows_per_seq + rr) * d_out + c;
     const int64_t kstride = (int64_t)rows_per_seq * d_out;
-    for (int c0 = 0; c0 < d_out; c0 += 512) {  // up to four float4 per lane and pass
-        float4 acc[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int k = 0; k < S; ++k) {
-            const float wk = dead ? 0.f : expf(lp[(int64_t)k * rows_per_seq] - mx);
-            if (wk == 0.f) continue;  // an empty split's partial is never read
-            const float* ok = op + k * kstride;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int c = c0 + (lane + 32 * u) * 4;
-                if (c < d_out) {
-                    const float4 x = *reinterpret_cast<const float4*>(ok + c);
-                    acc[u].x = fmaf(wk, x.x, acc[u].x);
-                    acc[u].y = fmaf(wk, x.y, acc[u].y);
-                    acc[u].z = fmaf(wk, x.z, acc[u].z);
-                    acc[u].w = fmaf(wk, x.w, acc[u].w);
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int c = c0 + (lane + 32 * u) * 4;
-            if (c < d_out)
-                store4(out + r * d_out + c, make_float4(acc[u].x * inv, acc[u].y * inv, acc[u].z * inv, acc[u].w * inv));
-        }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float den = 0.f;
+    for (int k = 0; k < S; ++k) {
+        const float wk = dead ? 0.f : expf(__ldg(lp + (int64_t)k * rows_per_seq) - mx);
+        den += wk;
+        if (wk == 0.f) continue;  // an empty split's partial is never read
+        const float4 x = ld_stream4(op + k * kstride);
+        acc.x = fmaf(wk, x.x, acc.x);
+        acc.y = fmaf(wk, x.y, acc.y);
+        acc.z = fmaf(wk, x.z, acc.z);
+        acc.w = fmaf(wk, x.w, acc.w);
     }
-    if (lse != nullptr && lane == 0) lse[r] = dead ? -INFINITY : mx + logf(den);
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+    store4(out + r * d_out + c, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
+    if (lse != nullptr && c == 0) lse[r] = dead ? -INFINITY : mx + logf(den);
 }
 
 // q_hat[row, r] = sum_d W_UK[j][r][d] * q_c[row, d]  (r < r_kv);  q_hat[row, r_kv + d] = q_r[row, d].

@@ -297,14 +297,16 @@ gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_spl
     if (rows > 0x7fffffffLL) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (d_out % 4 == 0) {
-        const int warps = 8;
-        const unsigned blocks = (unsigned)((rows + warps - 1) / warps);
+        const int64_t items = rows * (d_out / 4);
+        const int64_t nblk = (items + 255) / 256;
+        if (nblk > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+        const unsigned blocks = (unsigned)nblk;
         if (out_dtype == GQLA_BF16)
-            combine_vec_kernel<__nv_bfloat16><<<blocks, warps * 32, 0, st>>>(rows, rows_per_seq, num_splits, d_out, o_part,
-                                                                            lse_part, (__nv_bfloat16*)out, lse);
+            combine_vec_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(rows, rows_per_seq, num_splits, d_out, o_part,
+                                                                     lse_part, (__nv_bfloat16*)out, lse);
         else
-            combine_vec_kernel<float><<<blocks, warps * 32, 0, st>>>(rows, rows_per_seq, num_splits, d_out, o_part,
-                                                                    lse_part, (float*)out, lse);
+            combine_vec_kernel<float><<<blocks, 256, 0, st>>>(rows, rows_per_seq, num_splits, d_out, o_part, lse_part,
+                                                             (float*)out, lse);
         return launch_status();
     }
     const size_t smem = (size_t)num_splits * sizeof(float);
