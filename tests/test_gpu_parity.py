@@ -238,6 +238,8 @@ def test_c2_full_gqa_mtp():
     from tests.parity_util import end_to_end
     end_to_end(synth.WORKLOADS["C2"], None, 1, sample_seqs=(0, 17, 63), paths=("gqa",))
     end_to_end(synth.WORKLOADS["C2"], None, 1, q_gain=4.0, sample_seqs=(5,), paths=("gqa", "absorb"))
+    # the launch configuration bench.py times: balanced plan, two slots per sequence
+    end_to_end(synth.WORKLOADS["C2"], None, -2, q_gain=4.0, sample_seqs=(3, 4, 60), paths=("gqa",))
 
 
 @pytest.mark.parametrize("s_q", [1, 2])
@@ -250,6 +252,7 @@ def test_c3_full_ragged(s_q):
     assert sl.min() >= 512 and sl.max() <= 32768
     sample = sorted({int(sl.argmin()), int(sl.argmax()), 3, 100})
     end_to_end(w, None, 4, q_gain=4.0, sample_seqs=sample)
+    end_to_end(w, None, -3, q_gain=4.0, sample_seqs=sample)  # balanced plan: cuts inside long sequences
 
 
 @pytest.mark.parametrize("s_q", [1, 2])
@@ -274,7 +277,7 @@ def test_c4_long_context_split_sweep(s_q):
     ref_g = O.gqa_path(*args)
     q = torch.cat([x["q_c"], x["q_r"]], -1).contiguous().cuda()
     qc, qr = x["q_c"].cuda(), x["q_r"].cuda()
-    for S in (1, 8, 32, 128):
+    for S in (1, 8, 32, 128, -32):
         a = dec.absorb_step(qc, qr, S).float().cpu().numpy()[b:b + 1]
         assert_close(a, ref_a, f"C4 absorb S={S}")
         gq = dec.gqa_step(q, S).float().cpu().numpy()[b:b + 1]
