@@ -1,7 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the GQLA decode hot path on B200.
 
-A step = one pass of the absorb path (absorb_q -> decode_absorb -> combine_splits -> up_proj)
+A step = one pass of the absorb path (absorb_q -> decode_absorb -> combine_up_proj, the split merge
+fused with the up-projection)
 over the canonical workload (h_q=128, g=8, d_h=128, r_kv=512, d_r=64, B=64, T=4096, s_q=1,
 bf16 cache).  The GQA path (decode_gqa -> combine_splits on the expanded cache, s_q=2) is
 measured in the same run and reported under "paths".  One JSON line on stdout.
@@ -266,8 +267,7 @@ def run_ours(args):
         B.gqla_decode_absorb(dec.dims, q_hat, dec.cache, dec.seq_start, dec.seqlens, dec.scale, S_a, o_part, lse_part,
                              dec.status)
         b.record()
-        B.gqla_combine_splits(o_part, lse_part, o_hat, None)
-        B.gqla_up_proj(dec.dims, o_hat, dec.w_uv, o_out)
+        B.gqla_combine_up_proj(dec.dims, o_part, lse_part, dec.w_uv, o_out, None)
 
     # The step as a user serves it: the four launches captured once in a CUDA graph, one replay per step
     # (the eager chain costs more host time per step than the GPU needs to run it).
@@ -415,8 +415,8 @@ def run_ours(args):
             "config": {"workload": "C1 canonical absorb path: h_q=128 g=8 d_h=128 r_kv=512 d_r=64 B=64 T=4096 s_q=1 "
                                    "bf16 cache (576 elems/token)", "num_splits": S_a, "parallelism": "replicas only",
                        "l2": "inputs larger than L2 (302 MB cache vs 126 MB L2); no flush",
-                       "launch": "one CUDA-graph replay per step (4 kernels); kernel time from an eager pass with events"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * steps, "roofline": roof, "cpu_baseline": cpu,
+                       "launch": "one CUDA-graph replay per step (3 kernels: absorb_q, decode_absorb, combine_up_proj); kernel time from an eager pass with events"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * steps, "roofline": roof, "cpu_baseline": cpu,
             "paths": paths,
         }
         print(json.dumps(line))

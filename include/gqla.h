@@ -165,6 +165,16 @@ gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_spl
 gqla_status gqla_up_proj(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, const void* o_hat,
                          const void* w_uv, void* o, void* stream);
 
+/* gqla_combine_splits followed by gqla_up_proj in one kernel (Eq. (mqa), line 6, applied to the merged
+ * latent output): the merged o_hat never goes to memory.  Same arguments as the two calls:
+ *   o_part [B, S, s_q, h_q, r_kv] fp32, lse_part [B, S, s_q, h_q] fp32, w_uv [g, r_kv, d_h]
+ *   o [B, s_q, h_q, d_h] (out, `dtype`),  lse [B, s_q, h_q] fp32 (out) or NULL.
+ * With GQLA_BF16 the tensor-core kernel rounds the merged o_hat to bf16 before the contraction, as
+ * gqla_up_proj's input is; the generic kernel keeps it in fp32. */
+gqla_status gqla_combine_up_proj(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, int32_t num_splits,
+                                 const float* o_part, const float* lse_part, const void* w_uv, void* o, float* lse,
+                                 void* stream);
+
 /* Integer bookkeeping, exported so it can be compared exactly with an independent statement.
  * HOST pointers. */
 /* Split ranges of a sequence of `seqlen` rows: begin[k], end[k] for k < num_splits. */

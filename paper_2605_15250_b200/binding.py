@@ -47,6 +47,8 @@ _PROTOTYPES = {
                                           c_void_p, c_void_p]),
     "gqla_combine_splits": (c_int32, [c_int32, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_void_p]),
+    "gqla_combine_up_proj": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
+                                       c_void_p, c_void_p, c_void_p]),
     "gqla_up_proj": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_split_plan": (c_int32, [c_int32, c_int32, c_void_p, c_void_p]),
     "gqla_visible_limit": (c_int32, [c_int32, c_int32, c_int32]),
@@ -209,6 +211,17 @@ def gqla_up_proj(dims: GqlaDims, o_hat: torch.Tensor, w_uv: torch.Tensor, o: tor
     B, s_q = o_hat.shape[0], o_hat.shape[1]
     _check(lib().gqla_up_proj(ctypes.byref(dims), _dtype_code(o_hat), B, s_q, _ptr(o_hat), _ptr(w_uv), _ptr(o),
                               _stream()), "gqla_up_proj")
+
+
+def gqla_combine_up_proj(dims: GqlaDims, o_part: torch.Tensor, lse_part: torch.Tensor, w_uv: torch.Tensor,
+                         o: torch.Tensor, lse: torch.Tensor | None = None) -> None:
+    """Split merge fused with the up-projection: o_part [B,S,s_q,h_q,r_kv], lse_part [B,S,s_q,h_q] ->
+    o[B,s_q,h_q,d_h] = W^UV_{j(i)} (merged o_hat)  (Eq. (mqa), line 6)."""
+    _contig(o_part, lse_part, w_uv, o, lse)
+    assert o_part.dtype == torch.float32 and lse_part.dtype == torch.float32
+    B, S, s_q = o_part.shape[0], o_part.shape[1], o_part.shape[2]
+    _check(lib().gqla_combine_up_proj(ctypes.byref(dims), _dtype_code(o), B, s_q, S, _ptr(o_part), _ptr(lse_part),
+                                      _ptr(w_uv), _ptr(o), _ptr(lse), _stream()), "gqla_combine_up_proj")
 
 
 # ------------------------------------------------------------------ integer helpers (host)

@@ -227,6 +227,47 @@ __global__ void __launch_bounds__(128) up_proj_generic_kernel(int32_t h_q, int32
     }
 }
 
+// Split merge fused with the up-projection: o[row, d] = sum_r W_UV[j][r][d] * (sum_k w_k o_part[row, k, r]).
+// One block per row; the merged latent row lives in shared memory only.
+template <typename T>
+__global__ void __launch_bounds__(128) combine_up_generic_kernel(int32_t h_q, int32_t hpg, int32_t d_h, int32_t r_kv,
+                                                                 int32_t rows_per_seq, int32_t S,
+                                                                 const float* __restrict__ o_part,
+                                                                 const float* __restrict__ lse_part,
+                                                                 const T* __restrict__ w_uv, T* __restrict__ o,
+                                                                 float* __restrict__ lse) {
+    extern __shared__ float os[];  // [r_kv]
+    const int64_t row = blockIdx.x;  // (b, p, i)
+    const int i = (int)(row % h_q);
+    const int j = i / hpg;
+    const int64_t b = row / rows_per_seq;
+    const int rr = (int)(row % rows_per_seq);
+    const float* lp = lse_part + b * S * rows_per_seq + rr;
+    float mx = -INFINITY;
+    for (int k = 0; k < S; ++k) mx = fmaxf(mx, lp[(int64_t)k * rows_per_seq]);
+    const bool dead = !(mx > -INFINITY);
+    float den = 0.f;
+    for (int k = 0; k < S; ++k) den += dead ? 0.f : expf(lp[(int64_t)k * rows_per_seq] - mx);
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+    const float* op = o_part + (b * S * rows_per_seq + rr) * r_kv;
+    for (int r = threadIdx.x; r < r_kv; r += blockDim.x) {
+        float acc = 0.f;
+        for (int k = 0; k < S; ++k) {
+            const float wk = dead ? 0.f : expf(lp[(int64_t)k * rows_per_seq] - mx);
+            if (wk != 0.f) acc = fmaf(wk, op[(int64_t)k * rows_per_seq * r_kv + r], acc);
+        }
+        os[r] = acc * inv;
+    }
+    __syncthreads();
+    const T* W = w_uv + (int64_t)j * r_kv * d_h;
+    for (int d = threadIdx.x; d < d_h; d += blockDim.x) {
+        float acc = 0.f;
+        for (int r = 0; r < r_kv; ++r) acc = fmaf(ldf(W + (int64_t)r * d_h + d), os[r], acc);
+        stf(o + row * d_h + d, acc);
+    }
+    if (lse != nullptr && threadIdx.x == 0) lse[row] = dead ? -INFINITY : mx + logf(den);
+}
+
 // K_C[n, j, d] = sum_r W_UK[j][r][d] c[n][r],  V likewise with W_UV,  k_R[n] = cache[n, r_kv:].
 // One block per kRows cache rows; the latent rows are staged in shared memory and every thread
 // owns one (j, d) output column of both planes for all staged rows.

@@ -184,6 +184,37 @@ gqla_status gqla_up_proj(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_
     return launch_status();
 }
 
+gqla_status gqla_combine_up_proj(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, int32_t num_splits,
+                                 const float* o_part, const float* lse_part, const void* w_uv, void* o, float* lse,
+                                 void* stream) {
+    gqla_status s;
+    if ((s = check_dims(d)) != GQLA_OK) return s;
+    if ((s = check_dtype(dtype)) != GQLA_OK) return s;
+    if (B < 0 || s_q < 1 || num_splits < 1) return GQLA_ERR_SHAPE;
+    if (o_part == nullptr || lse_part == nullptr || w_uv == nullptr || o == nullptr) return GQLA_ERR_NULL;
+    if (!aligned16(o_part) || !aligned16(w_uv) || !aligned16(o)) return GQLA_ERR_ALIGN;
+    const int64_t rows = (int64_t)B * s_q * d->h_q;
+    if (rows == 0) return GQLA_OK;
+    if (rows > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (g_policy.load() == GQLA_POLICY_AUTO) {
+        s = tc_combine_up_proj(*d, dtype, B, s_q, num_splits, o_part, lse_part, w_uv, o, lse, st);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
+    const size_t smem = (size_t)d->r_kv * sizeof(float);
+    if (smem > 48 * 1024) return GQLA_ERR_UNSUPPORTED;
+    const int hpg = d->h_q / d->g;
+    if (dtype == GQLA_BF16)
+        combine_up_generic_kernel<__nv_bfloat16><<<(unsigned)rows, 128, smem, st>>>(
+            d->h_q, hpg, d->d_h, d->r_kv, s_q * d->h_q, num_splits, o_part, lse_part, (const __nv_bfloat16*)w_uv,
+            (__nv_bfloat16*)o, lse);
+    else
+        combine_up_generic_kernel<float><<<(unsigned)rows, 128, smem, st>>>(d->h_q, hpg, d->d_h, d->r_kv, s_q * d->h_q,
+                                                                           num_splits, o_part, lse_part,
+                                                                           (const float*)w_uv, (float*)o, lse);
+    return launch_status();
+}
+
 gqla_status gqla_expand_cache(const gqla_dims* d, gqla_dtype dtype, int64_t N, const void* cache,
                               int64_t cache_row_stride, const void* w_uk, const void* w_uv, void* k_c, void* v,
                               void* k_r, void* stream) {

@@ -6,6 +6,7 @@
 #include "common.cuh"
 #include "tc_decode_absorb.cuh"
 #include "tc_decode_gqa.cuh"
+#include "tc_combine_up.cuh"
 #include "tc_gemm.cuh"
 
 namespace gqla {
@@ -157,6 +158,40 @@ inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, i
     cudaError_t e =
         tc::gemm_launch<tc::kGemmUpProj, 128, true>(p, tmA, tmB, tmB, dim3((unsigned)m_tiles, (unsigned)d.g, 1), st);
     return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
+}
+
+// Fused split merge + up-projection; covers what tc_up_proj covers with d_h = 128 and r_kv % 128 == 0.
+inline gqla_status tc_combine_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, int32_t s_q, int32_t S,
+                                      const float* o_part, const float* lse_part, const void* w_uv, void* o, float* lse,
+                                      cudaStream_t st) {
+    const int hpg = d.h_q / d.g;
+    if (!tc_gemm_covers(d, dtype) || S > tc::CombineUpSmem::kMaxS || hpg > 64 ||
+        d.r_kv > tc::CombineUpSmem::kMaxChunks * tc::CombineUpSmem::kChunkK)
+        return GQLA_ERR_UNSUPPORTED;
+    const int64_t positions = (int64_t)B * s_q;
+    const int64_t m_tiles = (positions + 64 / hpg - 1) / (64 / hpg);
+    if (m_tiles > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
+    CUtensorMap tmB;
+    {
+        const uint64_t dims[2] = {(uint64_t)d.d_h, (uint64_t)d.g * d.r_kv};
+        const uint64_t str[1] = {(uint64_t)d.d_h * 2};
+        const uint32_t box[2] = {64, 64};
+        if (!tc::make_tmap_bf16(&tmB, w_uv, 2, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    tc::CombineUpParams p{};
+    p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.r_kv = d.r_kv;
+    p.positions = positions; p.o_part = o_part; p.lse_part = lse_part; p.out = o; p.lse = lse; p.status = nullptr;
+    auto kern = tc::combine_up_tc_kernel;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::CombineUpSmem::kTotal) != cudaSuccess)
+            return GQLA_ERR_CUDA;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    kern<<<dim3((unsigned)m_tiles, (unsigned)d.g, 1), tc::CombineUpSmem::kThreads, tc::CombineUpSmem::kTotal, st>>>(p, tmB);
+    return cudaGetLastError() == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
 }
 
 inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S,

@@ -52,7 +52,9 @@ class GqlaDecoder:
             B.gqla_expand_cache(self.dims, self.cache, self.w_uk, self.w_uv, self.k_c, self.v, self.k_r)
 
     # ---- absorb path ----
-    def absorb_step(self, q_c: torch.Tensor, q_r: torch.Tensor, num_splits: int = 1, want_lse: bool = False):
+    def absorb_step(self, q_c: torch.Tensor, q_r: torch.Tensor, num_splits: int = 1, want_lse: bool = False,
+                    fused_tail: bool = True):
+        """absorb_q -> decode_absorb -> combine_up_proj (or combine_splits -> up_proj when fused_tail is off)."""
         Bn, s_q = q_c.shape[0], q_c.shape[1]
         slots = abs(num_splits)  # num_splits < 0: balanced plan with that many slots per sequence
         q_hat = self._get("q_hat", (Bn, s_q, self.h_q, self.r_kv + self.d_r), self.dtype)
@@ -64,8 +66,11 @@ class GqlaDecoder:
         B.gqla_absorb_q(self.dims, q_c, q_r, self.w_uk, q_hat)
         B.gqla_decode_absorb(self.dims, q_hat, self.cache, self.seq_start, self.seqlens, self.scale, num_splits,
                              o_part, lse_part, self.status)
-        B.gqla_combine_splits(o_part, lse_part, o_hat, lse)
-        B.gqla_up_proj(self.dims, o_hat, self.w_uv, o)
+        if fused_tail:
+            B.gqla_combine_up_proj(self.dims, o_part, lse_part, self.w_uv, o, lse)
+        else:
+            B.gqla_combine_splits(o_part, lse_part, o_hat, lse)
+            B.gqla_up_proj(self.dims, o_hat, self.w_uv, o)
         return (o, lse) if want_lse else o
 
     # ---- GQA path ----

@@ -83,6 +83,13 @@ def stagewise(w: synth.Workload, seqlens, num_splits: int, q_gain: float = 1.0, 
     errs["combine_o"] = assert_close(o_hat.float().cpu().numpy(), oh_ref, "combine o")
     errs["combine_lse"] = assert_close(lse.cpu().numpy(), l_ref, "combine lse")
 
+    # combine fused with up_proj, on the same partials, against the unrounded composition
+    o_f = torch.empty((Bn, s_q, w.h_q, w.d_h), dtype=dt, device="cuda")
+    lse_f = torch.empty((Bn, s_q, w.h_q), dtype=torch.float32, device="cuda")
+    B.gqla_combine_up_proj(bd, op_in.cuda(), lp_in.cuda(), dev["w_uv"], o_f, lse_f)
+    errs["combine_up_proj"] = assert_close(o_f.float().cpu().numpy(), O.up_proj(od, oh_ref, f["w_uv"]), "combine_up_proj")
+    errs["combine_up_lse"] = assert_close(lse_f.cpu().numpy(), l_ref, "combine_up_proj lse")
+
     # up_proj on the oracle's o_hat rounded to storage
     oh_in = round_to(w, oh_ref)
     o = torch.empty((Bn, s_q, w.h_q, w.d_h), dtype=dt, device="cuda")

@@ -121,6 +121,9 @@ def test_argument_errors_return_before_launch():
     assert L.gqla_combine_splits(1, 128, 0, 512, 0, p, p, p, None, None) == 2
     assert L.gqla_combine_splits(1, 128, 4, 512, 0, p, None, p, None, None) == 1
     assert L.gqla_combine_splits(1, 128, 4, 512, 9, p, p, p, None, None) == 4
+    assert L.gqla_combine_up_proj(r(d), 0, 1, 1, 0, p, p, p, p, None, None) == 2  # splits < 1
+    assert L.gqla_combine_up_proj(r(d), 0, 1, 1, 2, p, None, p, p, None, None) == 1
+    assert L.gqla_combine_up_proj(r(d), 0, 1, 1, 2, p, p, odd, p, None, None) == 3
     assert B.lib().gqla_status_str(3).decode().startswith("pointer")
 
 
