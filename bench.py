@@ -29,6 +29,7 @@ import numpy as np
 import torch
 
 from paper_2605_15250_b200 import accounting as acct
+from paper_2605_15250_b200 import replicas
 from paper_2605_15250_b200 import synth
 
 METRIC = "decode attn tokens/s (absorb path, canonical config, 1 B200)"
@@ -185,12 +186,7 @@ def time_region(fn, steps: int, dist_on: bool):
     torch.cuda.synchronize()
     if dist_on:
         dist.barrier()
-    ms = e0.elapsed_time(e1)
-    if dist_on:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    return ms
+    return replicas.max_over_ranks(e0.elapsed_time(e1), "cuda")
 
 
 def run_ours(args):
@@ -218,7 +214,7 @@ def run_ours(args):
     steps, warmup = args.steps, max(args.warmup, 3)
 
     # ---- workload: replicas only -- every rank owns an independent batch (no data-path collective)
-    w1 = synth.WORKLOADS["C1"].with_(seed=synth.WORKLOADS["C1"].seed + 0x100 * rank)
+    w1 = synth.WORKLOADS["C1"].with_(seed=replicas.replica_seed(synth.WORKLOADS["C1"].seed, rank))
     x = synth.make_inputs(w1)
     dev = torch.device("cuda", local_rank)
     dec = GqlaDecoder(w1.h_q, w1.g, w1.d_h, w1.r_kv, w1.d_r, x["w_uk"].to(dev), x["w_uv"].to(dev),
@@ -283,7 +279,7 @@ def run_ours(args):
     dec.check_status()
     ms_per_step = total_ms / steps
     kern_ms = statistics.mean(a.elapsed_time(b) for a, b in kev)
-    value = world * w1.batch * w1.s_q / (ms_per_step * 1e-3)
+    value = replicas.aggregate_tokens_per_s(world, w1.batch, w1.s_q, ms_per_step)
 
     kbytes = acct.decode_kernel_bytes("absorb", h_q=w1.h_q, g=w1.g, d_h=w1.d_h, r_kv=w1.r_kv, d_r=w1.d_r,
                                       s_q=w1.s_q, batch=w1.batch, total_tokens=total_tokens, num_splits=pieces_a)
@@ -306,28 +302,41 @@ def run_ours(args):
 
     # ---- end to end through the public API with host buffers: per step, the queries and the step's new
     # cache rows go host -> device from pinned memory, and the attention output comes back.
-    h_qc, h_qr = x["q_c"].pin_memory(), x["q_r"].pin_memory()
+    # One pinned staging buffer [q_c | q_r | new cache rows] -> one copy each way; the copies, the scatter
+    # of the new rows into the cache and the three kernels are captured together, so a step is one graph
+    # launch plus the wait for its result.
     T = w1.seqlen
     cache3 = dec.cache.view(w1.batch, T, w1.d_abs)
-    h_new = x["cache"].view(w1.batch, T, w1.d_abs)[:, T - w1.s_q:, :].contiguous().pin_memory()
-    d_new = torch.empty_like(h_new, device=dev)
+    new_rows = x["cache"].view(w1.batch, T, w1.d_abs)[:, T - w1.s_q:, :].contiguous()
+    n_qc, n_qr, n_new = x["q_c"].numel(), x["q_r"].numel(), new_rows.numel()
+    h_in = torch.empty(n_qc + n_qr + n_new, dtype=torch.bfloat16).pin_memory()
+    h_in[:n_qc] = x["q_c"].reshape(-1)
+    h_in[n_qc:n_qc + n_qr] = x["q_r"].reshape(-1)
+    h_in[n_qc + n_qr:] = new_rows.reshape(-1)
+    d_in = torch.empty(n_qc + n_qr + n_new, dtype=torch.bfloat16, device=dev)
+    d_qc = d_in[:n_qc].view_as(x["q_c"])
+    d_qr = d_in[n_qc:n_qc + n_qr].view_as(x["q_r"])
+    d_new = d_in[n_qc + n_qr:].view_as(new_rows)
     h_out = torch.empty((w1.batch, w1.s_q, w1.h_q, w1.d_h), dtype=torch.bfloat16).pin_memory()
 
-    def e2e_step():
-        q_c.copy_(h_qc, non_blocking=True)
-        q_r.copy_(h_qr, non_blocking=True)
-        d_new.copy_(h_new, non_blocking=True)
+    def e2e_body():
+        d_in.copy_(h_in, non_blocking=True)
         cache3[:, T - w1.s_q:, :].copy_(d_new)
-        o = dec.absorb_step(q_c, q_r, S_a)
+        o = dec.absorb_step(d_qc, d_qr, S_a)
         h_out.copy_(o, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        return o
+
+    replay_e2e, _ = dec.capture(e2e_body)
+
+    def e2e_step():
+        replay_e2e()
+        torch.cuda.current_stream().synchronize()  # the host reads the step's result before the next step
 
     for _ in range(3):
         e2e_step()
     e2e_ms = time_region(e2e_step, steps, dist_on) / steps
-    e2e = {"value": world * w1.batch * w1.s_q / (e2e_ms * 1e-3), "unit": UNIT,
-           "h2d_bytes_per_step": h_qc.numel() * 2 + h_qr.numel() * 2 + h_new.numel() * 2,
-           "d2h_bytes_per_step": h_out.numel() * 2, "ms_per_step": e2e_ms}
+    e2e = {"value": replicas.aggregate_tokens_per_s(world, w1.batch, w1.s_q, e2e_ms), "unit": UNIT,
+           "h2d_bytes_per_step": h_in.numel() * 2, "d2h_bytes_per_step": h_out.numel() * 2, "ms_per_step": e2e_ms}
 
     # ---- GQA path on the same weights and latent (config 2: expanded cache, s_q = 2)
     w2 = synth.WORKLOADS["C2"].with_(seed=w1.seed)
