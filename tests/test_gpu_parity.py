@@ -196,6 +196,31 @@ def test_absorb_balanced_plan_llama(s_q):
     _balanced_absorb_case(w, synth.make_seqlens(w.with_(seqlen_range=(0, 1500))), 3)
 
 
+@pytest.mark.parametrize("h_q,g", [(128, 4), (64, 8), (64, 4), (16, 8)])
+@pytest.mark.parametrize("s_q", [1, 2])
+def test_shape_variants_of_the_paper(h_q, g, s_q):
+    """Operating points the paper discusses besides the canonical one: g = 4 (cache 2176 B/token, Table
+    "roofline"), h_q = 64 (Sec. 4.2), and few heads per group; fixed and balanced plans."""
+    from tests.parity_util import end_to_end, stagewise
+    w = _wl("variant", 5, s_q, 131, h_q=h_q, g=g, d_h=128, r_kv=512, d_r=64)
+    seqlens = np.array([700, 0, 129, 2050, 64], dtype=np.int32)
+    stagewise(w, seqlens, 3, 4.0)
+    end_to_end(w, seqlens, -3, q_gain=4.0)
+
+
+@pytest.mark.parametrize("s_q", [3, 4])
+def test_speculative_query_counts(s_q):
+    """s_q >= 3 (speculative decoding, Sec. 4.2): the absorb path stays on the tensor-core kernel (more
+    row blocks), the GQA path falls back to the generic kernel; the causal mask covers all s_q positions."""
+    from tests.parity_util import end_to_end, stagewise
+    w = _wl("spec", 4, s_q, 132, **CANON)
+    assert B.kernel_for(B.make_dims(**CANON), torch.bfloat16, s_q, "absorb") == "tcgen05"
+    seqlens = np.array([300, 2, 1029, 64], dtype=np.int32)
+    stagewise(w, seqlens, 2, 4.0)
+    end_to_end(w, seqlens, 2, q_gain=4.0)
+    end_to_end(w, seqlens, -3, q_gain=4.0, paths=("absorb",))
+
+
 def test_two_gpu_paths_agree_with_each_other():
     """Same weights, same latent: the two paths' GPU outputs differ by at most twice the
     tolerance (each is within it of the same oracle value)."""
