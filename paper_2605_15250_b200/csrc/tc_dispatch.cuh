@@ -33,7 +33,8 @@ inline bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 inline bool tc_covers(const gqla_dims& d, gqla_dtype dtype, int32_t s_q, int32_t path) {
     if (dtype != GQLA_BF16) return false;
     if (path == 1) {
-        if (d.d_h != 128 || d.d_r != 64 || (s_q != 1 && s_q != 2)) return false;
+        // the group's R = (h_q/g) * s_q rows are replicated 128/R times down the MMA tile: R must divide 128
+        if (d.d_h != 128 || d.d_r != 64 || s_q < 1 || s_q > 8 || !is_pow2(s_q)) return false;
         const int R = gqa_rows(d, s_q, nullptr);
         return is_pow2(d.h_q / d.g) && R >= 8 && R <= 128;
     }

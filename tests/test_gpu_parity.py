@@ -211,14 +211,16 @@ def test_shape_variants_of_the_paper(h_q, g, s_q):
 @pytest.mark.parametrize("s_q", [3, 4])
 def test_speculative_query_counts(s_q):
     """s_q >= 3 (speculative decoding, Sec. 4.2): the absorb path stays on the tensor-core kernel (more
-    row blocks), the GQA path falls back to the generic kernel; the causal mask covers all s_q positions."""
+    row blocks); the GQA path does for s_q = 4 (its rows still divide the 128-row tile) and falls back to
+    the generic kernel for s_q = 3; the causal mask covers all s_q positions."""
     from tests.parity_util import end_to_end, stagewise
     w = _wl("spec", 4, s_q, 132, **CANON)
     assert B.kernel_for(B.make_dims(**CANON), torch.bfloat16, s_q, "absorb") == "tcgen05"
+    assert B.kernel_for(B.make_dims(**CANON), torch.bfloat16, s_q, "gqa") == ("tcgen05" if s_q == 4 else "generic")
     seqlens = np.array([300, 2, 1029, 64], dtype=np.int32)
     stagewise(w, seqlens, 2, 4.0)
     end_to_end(w, seqlens, 2, q_gain=4.0)
-    end_to_end(w, seqlens, -3, q_gain=4.0, paths=("absorb",))
+    end_to_end(w, seqlens, -3, q_gain=4.0)
 
 
 def test_two_gpu_paths_agree_with_each_other():
