@@ -223,8 +223,8 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
         if (cta == 0 && elect_one()) {
             constexpr uint32_t idesc_qk = idesc_bf16(128, 128, 0, 0);
             constexpr uint32_t idesc_pv = idesc_bf16(128, 256, 0, 1);
-            const uint32_t q_addr = smem_u32(tiles);
-            const uint32_t p_addr = smem_u32(tiles + L::kOffP);
+            const uint64_t q_desc = desc_kmajor_sw128(smem_u32(tiles));
+            const uint64_t p_desc = desc_kmajor_sw128(smem_u32(tiles + L::kOffP));
             int ks = 0, vs = 0;
             uint32_t kph = 0, vph = 0;
             int gt = 0;  // tiles issued so far: score buffer = gt & 1, phase = (gt >> 1) & 1
@@ -234,14 +234,20 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
                 for (int g3 = 0; g3 < 3; ++g3) {
                     if (!mbar_wait(&kfull[ks], kph, ab, 3)) return false;
                     tc_fence_after();
-                    const uint32_t k_addr = smem_u32(tiles + L::kOffK + ks * L::kKGroup);
-                    const uint32_t qg = q_addr + g3 * 3 * L::kBox;
+                    // descriptors as low words: the high word is a constant, stepping is one 32-bit add
+                    const uint32_t kd = desc_lo(desc_kmajor_sw128(smem_u32(tiles + L::kOffK + ks * L::kKGroup)));
+                    const uint32_t qd = desc_lo(q_desc) + ((g3 * 3 * L::kBox) >> 4);
+                    if (g3 == 0)
+                        umma_ss2_lo<false>(d, qd, kd, idesc_qk);  // the tile's first MMA overwrites S
+                    else
+                        umma_ss2_lo<true>(d, qd, kd, idesc_qk);
 #pragma unroll
                     for (int i = 0; i < 3; ++i)
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
-                            umma_ss2(d, desc_kmajor_sw128(qg + i * L::kBox + kk * 32),
-                                     desc_kmajor_sw128(k_addr + i * L::kBox + kk * 32), idesc_qk, (g3 | i | kk) != 0);
+                            if ((i | kk) != 0)
+                                umma_ss2_lo<true>(d, qd + ((i * L::kBox + kk * 32) >> 4), kd + ((i * L::kBox + kk * 32) >> 4),
+                                                  idesc_qk);
                     umma_commit2(&kempty[ks], 3);
                     if (++ks == L::kNK) { ks = 0; kph ^= 1; }
                 }
@@ -269,15 +275,19 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
                     for (int h = 0; h < 2; ++h) {
                         if (!(ok = mbar_wait(&vfull[vs], vph, ab, 6))) break;
                         tc_fence_after();
-                        const uint32_t v_addr = smem_u32(tiles + L::kOffV + vs * L::kVGroup);
+                        const uint32_t vd = desc_lo(desc_mnmajor_sw128(smem_u32(tiles + L::kOffV + vs * L::kVGroup), L::kBox));
+                        const uint32_t pd = desc_lo(p_desc) + ((h * L::kBox) >> 4);
 #pragma unroll
-                        for (int m = 0; m < 2; ++m)
+                        for (int m = 0; m < 2; ++m) {
+                            const uint32_t dm = tmem_base + kAColO + (uint32_t)m * 128;
+                            if ((t | h) == 0)
+                                umma_ss2_lo<false>(dm, pd, vd + ((m * 2 * L::kBox) >> 4), idesc_pv);  // first P.V of a piece
+                            else
+                                umma_ss2_lo<true>(dm, pd, vd + ((m * 2 * L::kBox) >> 4), idesc_pv);
 #pragma unroll
-                            for (int kk = 0; kk < 4; ++kk)
-                                umma_ss2(tmem_base + kAColO + (uint32_t)m * 128,
-                                         desc_kmajor_sw128(p_addr + h * L::kBox + kk * 32),
-                                         desc_mnmajor_sw128(v_addr + m * 2 * L::kBox + kk * 2048, L::kBox), idesc_pv,
-                                         (t | h | kk) != 0);
+                            for (int kk = 1; kk < 4; ++kk)
+                                umma_ss2_lo<true>(dm, pd + ((kk * 32) >> 4), vd + ((m * 2 * L::kBox + kk * 2048) >> 4), idesc_pv);
+                        }
                         umma_commit2(&vempty[vs], 3);
                         if (++vs == L::kNV) { vs = 0; vph ^= 1; }
                     }
