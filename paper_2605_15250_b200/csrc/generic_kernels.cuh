@@ -154,6 +154,9 @@ __global__ void __launch_bounds__(256) combine_vec_kernel(int64_t rows, int32_t 
                                                           const float* __restrict__ o_part,
                                                           const float* __restrict__ lse_part, TO* __restrict__ out,
                                                           float* __restrict__ lse) {
+    // (dependent-launch instructions; no-ops when the kernel is launched the ordinary way)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int32_t vec_per_row = d_out >> 2;
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t r = idx / vec_per_row;

@@ -332,13 +332,14 @@ gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_spl
         const int64_t nblk = (items + 255) / 256;
         if (nblk > 0x7fffffffLL) return GQLA_ERR_SHAPE;
         const unsigned blocks = (unsigned)nblk;
+        cudaError_t e;
         if (out_dtype == GQLA_BF16)
-            combine_vec_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(rows, rows_per_seq, num_splits, d_out, o_part,
-                                                                     lse_part, (__nv_bfloat16*)out, lse);
+            e = tc::launch_pdl(combine_vec_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, rows, rows_per_seq,
+                               num_splits, d_out, o_part, lse_part, (__nv_bfloat16*)out, lse);
         else
-            combine_vec_kernel<float><<<blocks, 256, 0, st>>>(rows, rows_per_seq, num_splits, d_out, o_part, lse_part,
-                                                             (float*)out, lse);
-        return launch_status();
+            e = tc::launch_pdl(combine_vec_kernel<float>, dim3(blocks), dim3(256), 0, st, rows, rows_per_seq, num_splits,
+                               d_out, o_part, lse_part, (float*)out, lse);
+        return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
     }
     const size_t smem = (size_t)num_splits * sizeof(float);
     if (smem > 48 * 1024) return GQLA_ERR_UNSUPPORTED;

@@ -62,6 +62,7 @@ combine_up_tc_kernel(const CombineUpParams p, const __grid_constant__ CUtensorMa
     const int m_tile = blockIdx.x, j = blockIdx.y;
     const int n_chunks = p.r_kv / L::kChunkK;
     const int rows_per_seq = p.s_q * p.h_q;
+    pdl_launch_dependents();
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::kNumBars; ++i) mbar_init(&bars[i], i == 0 ? 4 : 1);
@@ -76,6 +77,7 @@ combine_up_tc_kernel(const CombineUpParams p, const __grid_constant__ CUtensorMa
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // set-up done; the partials come from the previous kernel of the stream
 
     if (warp == 0) {
         // ------------------------------------------------------------------ W^UV chunks (MN-major B operand)

@@ -341,6 +341,30 @@ __device__ __forceinline__ void umma_commit2(uint64_t* bar, uint16_t mask) {
         : "memory");
 }
 
+// ----------------------------------------------------------------------------- dependent launches
+// Programmatic dependent launch: a kernel launched with launch_pdl may begin (its CTAs start and run their
+// set-up: barrier init, TMEM allocation) while the previous kernel of the stream is still running, once
+// every CTA of that kernel has executed pdl_launch_dependents or exited.  It must call pdl_wait before it
+// touches global memory: the wait returns when the previous kernel has completed and its writes are
+// visible.  Both instructions do nothing in a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 // ----------------------------------------------------------------------------- small math
 __device__ __forceinline__ float ex2(float x) {
     float y;

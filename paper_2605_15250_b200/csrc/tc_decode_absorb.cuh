@@ -128,6 +128,8 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
         tmem_relinquish2();
     }
 
+    pdl_launch_dependents();
+    pdl_wait();  // barriers and TMEM are set up; everything below reads the caller's tensors
     // the plan of this pair: row block rb, and either one (sequence, split) piece or worker w's share
     const int pair = blockIdx.x >> 1;
     const int rb = pair % p.row_blocks;

@@ -111,6 +111,8 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
         tmem_relinquish();
     }
 
+    pdl_launch_dependents();
+    pdl_wait();  // barriers and TMEM are set up; everything below reads the caller's tensors
     // the plan of this CTA: group j, and either one (sequence, split) piece or worker w's share
     const int j = blockIdx.x % p.g;
     Walker walk;

@@ -191,8 +191,10 @@ inline gqla_status tc_combine_up_proj(const gqla_dims& d, gqla_dtype dtype, int3
             return GQLA_ERR_CUDA;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    kern<<<dim3((unsigned)m_tiles, (unsigned)d.g, 1), tc::CombineUpSmem::kThreads, tc::CombineUpSmem::kTotal, st>>>(p, tmB);
-    return cudaGetLastError() == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
+    return tc::launch_pdl(kern, dim3((unsigned)m_tiles, (unsigned)d.g, 1), dim3(tc::CombineUpSmem::kThreads),
+                          tc::CombineUpSmem::kTotal, st, p, tmB) == cudaSuccess
+               ? GQLA_OK
+               : GQLA_ERR_CUDA;
 }
 
 inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S,
@@ -231,8 +233,10 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
     auto kern = tc::decode_absorb_tc_kernel<0>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AbsorbSmem::kTotal) != cudaSuccess)
         return GQLA_ERR_CUDA;
-    kern<<<(unsigned)(2 * pairs), tc::AbsorbSmem::kThreads, tc::AbsorbSmem::kTotal, st>>>(p, tmQ, tmC);
-    return cudaGetLastError() == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
+    return tc::launch_pdl(kern, dim3((unsigned)(2 * pairs)), dim3(tc::AbsorbSmem::kThreads), tc::AbsorbSmem::kTotal, st, p,
+                          tmQ, tmC) == cudaSuccess
+               ? GQLA_OK
+               : GQLA_ERR_CUDA;
 }
 
 // CTA pairs of the absorb kernel that can be resident at once on the current device (cached).
@@ -274,8 +278,7 @@ inline cudaError_t gqa_launch(const tc::GqaParams& p, const CUtensorMap& q, cons
     auto kern = tc::decode_gqa_tc_kernel<R>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::GqaSmem::kTotal);
     if (e != cudaSuccess) return e;
-    kern<<<grid, tc::GqaSmem::kThreads, tc::GqaSmem::kTotal, st>>>(p, q, k, r, v);
-    return cudaGetLastError();
+    return tc::launch_pdl(kern, dim3(grid), dim3(tc::GqaSmem::kThreads), tc::GqaSmem::kTotal, st, p, q, k, r, v);
 }
 
 inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S, const void* q,

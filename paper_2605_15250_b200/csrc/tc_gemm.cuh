@@ -50,6 +50,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const Abort ab{abort_flag, p.status};
+    pdl_launch_dependents();
 
     // tile coordinates
     // expand: linear grid, (plane, group) fastest so that the CTAs sharing a tile of cache rows run together
@@ -74,6 +75,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // set-up done; the inputs may come from the previous kernel of the stream
 
     const CUtensorMap* tmB = (MODE == kGemmExpand && grp >= p.g) ? &tmB1 : &tmB0;
     const int j = (MODE == kGemmExpand) ? grp % p.g : grp;
@@ -214,8 +216,7 @@ inline cudaError_t gemm_launch(const GemmParams& p, const CUtensorMap& a, const 
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    kern<<<grid, 192, L::kTotal, st>>>(p, a, b0, b1);
-    return cudaGetLastError();
+    return launch_pdl(kern, grid, dim3(192), L::kTotal, st, p, a, b0, b1);
 }
 
 }  // namespace tc
