@@ -42,16 +42,18 @@ struct GqaSmem {
     static constexpr int kVBytes = 2 * 16384;                // 128 tokens x 128
     static constexpr int kStageBytes = kKcBytes + kKrBytes + kVBytes;
     static constexpr int kStages = 2;
-    static constexpr int kMergePitch = 33;                   // floats per lane row of the 32-column merge buffer
+    // floats per lane row of the merge buffer: 32 output columns + the row's (m, l) + 2 spare; a pitch of
+    // 36 words keeps 16-byte accesses of a quarter warp on distinct banks
+    static constexpr int kMergePitch = 36;
     static constexpr int kMergeBytes = 128 * kMergePitch * 4;
     static constexpr int kOffMerge = kQBytes + kStages * kStageBytes;
     static constexpr int kTileBytes = kOffMerge + kMergeBytes;
     // q_full q_empty o_free kfull[2] vfull[2] kempty[2] vempty[2] s_full[2] p_ready[2] pv_done[2]
     static constexpr int kNumBars = 17;
     static constexpr int kThreads = 192;
-    // behind the barriers: tmem slot + abort flag (16 B), then sm_m[128] + sm_l[128] (also the plan scratch)
-    static constexpr int kTotal = kTileBytes + kNumBars * 8 + 16 + 2 * 128 * 4;
-    static_assert(2 * 128 >= kThreads + 4, "plan scratch must fit in sm_m + sm_l");
+    // behind the barriers: tmem slot + abort flag (16 B).  The merge buffer doubles as the plan scratch.
+    static constexpr int kTotal = kTileBytes + kNumBars * 8 + 16;
+    static_assert(kMergeBytes >= (kThreads + 4) * 4, "plan scratch must fit in the merge buffer");
     static_assert(kTotal <= 232448, "shared memory budget of one CTA");
 };
 
@@ -94,8 +96,6 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
     uint64_t* pv_done = bars + 15; // [2]: P.V of tile n arrives on pv_done[n & 1]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + L::kNumBars);
     volatile int32_t* abort_flag = reinterpret_cast<volatile int32_t*>(tmem_slot + 1);
-    float* sm_m = reinterpret_cast<float*>(tmem_slot + 4);
-    float* sm_l = sm_m + 128;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const Abort ab{abort_flag, p.status};
@@ -118,7 +118,7 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
     Walker walk;
     if (p.balanced) {
         const BalancedStart st = balanced_prepass(p.seqlens, p.B, p.S, blockIdx.x / p.g, p.W,
-                                                  reinterpret_cast<int32_t*>(sm_m), L::kThreads);
+                                                  reinterpret_cast<int32_t*>(merge), L::kThreads);
         walk.init_balanced(p.seqlens, p.B, p.S, blockIdx.x / p.g, p.W, st);
     } else {
         const int unit = blockIdx.x / p.g;
@@ -239,7 +239,7 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
         const int col0 = R < 32 ? q * 32 : f * R;  // first column of the warp's window (warp-uniform)
         const int sub = R < 32 ? lane / R : 0;     // which R-column sub-block of the window is this thread's
         auto owns = [&](int c) -> bool { return R >= 32 || (c / R) == sub; };
-        const int mcol = Lr & 31, mrow0 = Lr >> 5;  // merge: output column and first row of this thread
+        const int mcg = Lr & 7, mrow0 = Lr >> 3;  // merge: group of four output columns and first row of this thread
 
         {   // a thread only ever writes its own columns of P; everything else stays zero for good
             uint32_t z[32];
@@ -339,22 +339,23 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
             if (pc.n_tiles > 0 && ok)
                 ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[n_last & 1], (n_last >> 1) & 1, ab, 9));
             tc_fence_after();
-            sm_m[Lr] = m_used;
-            sm_l[Lr] = l;
+            merge[Lr * L::kMergePitch + 32] = m_used;
+            merge[Lr * L::kMergePitch + 33] = l;
             named_bar_sync(1, 128);
             float M = -INFINITY;
 #pragma unroll
-            for (int ff = 0; ff < F; ++ff) M = fmaxf(M, sm_m[ff * R + r]);
+            for (int ff = 0; ff < F; ++ff) M = fmaxf(M, merge[(ff * R + r) * L::kMergePitch + 32]);
             float Lt = 0.f;
 #pragma unroll
             for (int ff = 0; ff < F; ++ff) {
-                const float mf = sm_m[ff * R + r];
-                if (mf > -INFINITY) Lt += sm_l[ff * R + r] * ex2(mf - M);
+                const float mf = merge[(ff * R + r) * L::kMergePitch + 32];
+                if (mf > -INFINITY) Lt += merge[(ff * R + r) * L::kMergePitch + 33] * ex2(mf - M);
             }
             const bool live = ok && pc.n_tiles > 0 && Lt > 0.f;
             const float w = (live && m_used > -INFINITY) ? ex2(m_used - M) / Lt : 0.f;
             const int64_t out_row0 = ((slot0 + pc.k) * p.s_q) * p.h_q + (int64_t)j * p.hpg;
-            // 32 output columns at a time through the merge buffer: lane rows in, (row, column) sums out
+            // 32 output columns at a time through the merge buffer: lane rows in (16-byte stores), sums of the
+            // F replicas out (thread = four columns of every 16th row; 16-byte loads and global stores)
 #pragma unroll 1
             for (int c4 = 0; c4 < 4; ++c4) {
                 uint32_t o[32];
@@ -362,21 +363,28 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
                     tmem_ld32(lane_base + kColO + c4 * 32, o);
                     tmem_wait_ld();
                 }
+                float4* mrow = reinterpret_cast<float4*>(merge + Lr * L::kMergePitch);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) merge[Lr * L::kMergePitch + i] = w == 0.f ? 0.f : __uint_as_float(o[i]) * w;
+                for (int i = 0; i < 8; ++i)
+                    mrow[i] = w == 0.f ? make_float4(0.f, 0.f, 0.f, 0.f)
+                                       : make_float4(__uint_as_float(o[4 * i]) * w, __uint_as_float(o[4 * i + 1]) * w,
+                                                     __uint_as_float(o[4 * i + 2]) * w, __uint_as_float(o[4 * i + 3]) * w);
                 if (c4 == 3) {  // O has been read: the next piece's first P.V may overwrite it
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(o_free);
                 }
                 named_bar_sync(1, 128);
-                for (int rr = mrow0; rr < R; rr += 4) {
+                for (int rr = mrow0; rr < R; rr += 16) {
                     const int pp = rr / p.hpg_box, ii = rr % p.hpg_box;
                     if (ii >= p.hpg) continue;
-                    float acc = 0.f;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                    for (int ff = 0; ff < F; ++ff) acc += merge[(ff * R + rr) * L::kMergePitch + mcol];
-                    p.o_part[(out_row0 + (int64_t)pp * p.h_q + ii) * 128 + c4 * 32 + mcol] = acc;
+                    for (int ff = 0; ff < F; ++ff) {
+                        const float4 x = *reinterpret_cast<const float4*>(merge + (ff * R + rr) * L::kMergePitch + 4 * mcg);
+                        acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+                    }
+                    *reinterpret_cast<float4*>(p.o_part + (out_row0 + (int64_t)pp * p.h_q + ii) * 128 + c4 * 32 + 4 * mcg) = acc;
                 }
                 named_bar_sync(1, 128);
             }
