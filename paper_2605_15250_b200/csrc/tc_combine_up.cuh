@@ -151,9 +151,9 @@ combine_up_tc_kernel(const CombineUpParams p, const __grid_constant__ CUtensorMa
             uint8_t* a_lane = a_smem + (lane >> 4) * 8192;  // k-block (within a chunk) of this lane's 4 columns
 #pragma unroll 1
             for (int r0 = 0; r0 < 16; r0 += 4) {
-                // 4 rows x all K chunks at a time: every load of the pass is issued before any is used.  Loads
-                // are unconditional (a partial of an empty split may hold anything: it is masked after the
-                // load, not skipped).
+                // 4 rows x all K chunks at a time: every load of a split slot is issued before any is used.
+                // Within a fetched slot the loads are unconditional (the partial of a row for which the slot is
+                // empty may hold anything: it is masked after the load).
                 float4 acc[4][L::kMaxChunks];
                 const float* src[4];
                 float rM[4], rinv[4];
@@ -173,13 +173,19 @@ combine_up_tc_kernel(const CombineUpParams p, const __grid_constant__ CUtensorMa
                     float wk[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
+                        const int tr = q * 16 + r0 + u;
+                        wk[u] = rinv[u] == 0.f ? 0.f : expf(sm_lse[tr * L::kMaxS + k] - rM[u]) * rinv[u];
+                    }
+                    // a slot that is empty for all four rows (the usual case under the balanced plan, whose
+                    // rows of one pass belong to one sequence) is not fetched at all; warp-uniform branch
+                    if (wk[0] == 0.f && wk[1] == 0.f && wk[2] == 0.f && wk[3] == 0.f) continue;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
 #pragma unroll
                         for (int c = 0; c < L::kMaxChunks; ++c)
                             if (c < n_chunks)
                                 x[u][c] = *reinterpret_cast<const float4*>(src[u] + (int64_t)k * rows_per_seq * p.r_kv +
                                                                            c * L::kChunkK);
-                        const int tr = q * 16 + r0 + u;
-                        wk[u] = rinv[u] == 0.f ? 0.f : expf(sm_lse[tr * L::kMaxS + k] - rM[u]) * rinv[u];
                     }
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {

@@ -66,7 +66,9 @@ class GqlaDecoder:
         B.gqla_absorb_q(self.dims, q_c, q_r, self.w_uk, q_hat)
         B.gqla_decode_absorb(self.dims, q_hat, self.cache, self.seq_start, self.seqlens, self.scale, num_splits,
                              o_part, lse_part, self.status)
-        if fused_tail:
+        # with many slots per sequence the fused kernel (64 rows per CTA, one slot after the other) runs out of
+        # parallelism; the separate merge streams the partials with every thread of the GPU
+        if fused_tail and slots <= 4:
             B.gqla_combine_up_proj(self.dims, o_part, lse_part, self.w_uv, o, lse)
         else:
             B.gqla_combine_splits(o_part, lse_part, o_hat, lse)
