@@ -228,10 +228,6 @@ __device__ __forceinline__ uint64_t desc_mnmajor_sw128(uint32_t smem_addr, uint3
            ((uint64_t)(1024 >> 4) << 32);
 }
 
-// Descriptor of the same layout `bytes` further on (bytes a multiple of 16, no carry out of the 14-bit
-// address field as long as the operand stays inside shared memory): one 64-bit add instead of a rebuild.
-__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) { return desc + (uint64_t)(bytes >> 4); }
-
 // Instruction descriptor for kind::f16 with bf16 operands and fp32 accumulation:
 //   [4,6) D format (1 = f32)  [7,10) A format (1 = bf16)  [10,13) B format (1 = bf16)
 //   [15] A major (0 = K)  [16] B major (0 = K, 1 = MN)  [17,23) N >> 3  [24,29) M >> 4
@@ -309,15 +305,8 @@ __device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* m
         "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(x), "r"(y)
         : "memory");
 }
-__device__ __forceinline__ void umma_ss2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                         uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// Same MMA with the descriptors given as (low word, high word): the high word of a shared-memory
+// D[tmem] (+)= A[smem] * B[smem] across the CTA pair, issued by ONE thread of the leader.  The descriptors are
+// given as (low word, high word): the high word of a shared-memory
 // descriptor (SBO, version, swizzle) is a constant, so stepping through an operand is one 32-bit add.
 // The issuing thread's instruction count per MMA matters: one MMA of the shapes used here is only 32-64
 // cycles of tensor work.
