@@ -96,7 +96,12 @@ inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t
     p.h_q = d.h_q; p.g = d.g; p.hpg = d.h_q / d.g; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
     p.out0 = k_c; p.out1 = v; p.aux_in = cache; p.aux_out = k_r; p.aux_stride = cache_row_stride;
     p.status = nullptr;
-    cudaError_t e = tc::gemm_launch<tc::kGemmExpand, 128, true>(p, tmA, tmK, tmV, dim3((unsigned)(m_tiles * 2 * d.g)), st);
+    // 128 x 256 output tiles (two adjacent groups) when g is even: the 128-row latent tile is then re-read
+    // through L2 by g CTAs instead of 2g
+    cudaError_t e = (d.g % 2 == 0)
+                        ? tc::gemm_launch<tc::kGemmExpand, 256, true>(p, tmA, tmK, tmV, dim3((unsigned)(m_tiles * d.g)), st)
+                        : tc::gemm_launch<tc::kGemmExpand, 128, true>(p, tmA, tmK, tmV, dim3((unsigned)(m_tiles * 2 * d.g)),
+                                                                      st);
     return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
 }
 

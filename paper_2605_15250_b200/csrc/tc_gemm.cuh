@@ -54,8 +54,12 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
 
     // tile coordinates
     // expand: linear grid, (plane, group) fastest so that the CTAs sharing a tile of cache rows run together
-    const int m_tile = (MODE == kGemmExpand) ? (int)(blockIdx.x / (2 * p.g)) : (int)blockIdx.x;
-    const int grp = (MODE == kGemmExpand) ? (int)(blockIdx.x % (2 * p.g)) : (int)blockIdx.y;  // plane * g + j, or j
+    // (expand: a CTA covers BN / d_h adjacent groups of one plane; grp counts in units of that many groups)
+    constexpr int kGroupsPerCta = (MODE == kGemmExpand) ? BN / 128 : 1;
+    const int grp_slots = (MODE == kGemmExpand) ? 2 * p.g / kGroupsPerCta : 1;
+    const int m_tile = (MODE == kGemmExpand) ? (int)(blockIdx.x / grp_slots) : (int)blockIdx.x;
+    const int grp = (MODE == kGemmExpand) ? (int)(blockIdx.x % grp_slots) * kGroupsPerCta
+                                          : (int)blockIdx.y;  // plane * g + first group j, or j
     const int n_tile = (MODE == kGemmExpand) ? 0 : (int)blockIdx.z;
 
     if (threadIdx.x == 0) {
@@ -102,7 +106,13 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
                         "r"(m_tile * (128 / p.hpg))
                         : "memory");
                 }
-                if (B_MN) {
+                if (B_MN && MODE == kGemmExpand) {
+                    // rows = j * K + k, columns = d; one 64x64 box per 64 output columns, two per group
+#pragma unroll
+                    for (int nb = 0; nb < BN / 64; ++nb)
+                        tma_load_2d(b_dst + nb * 8192, tmB, (nb & 1) * 64, (j + (nb >> 1)) * p.k_blocks * 64 + kb * 64,
+                                    &full[s]);
+                } else if (B_MN) {
                     // rows = j * K + k, columns = output feature; one 64x64 box per 64 output columns
 #pragma unroll
                     for (int nb = 0; nb < BN / 64; ++nb)
