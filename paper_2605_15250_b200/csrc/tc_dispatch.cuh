@@ -7,6 +7,7 @@
 #include "tc_decode_absorb.cuh"
 #include "tc_decode_gqa.cuh"
 #include "tc_combine_up.cuh"
+#include "tc_expand.cuh"
 #include "tc_gemm.cuh"
 
 namespace gqla {
@@ -89,6 +90,26 @@ inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t
         const uint32_t box[2] = {64, 64};
         if (!tc::make_tmap_bf16(&tmK, w_uk, 2, dims, str, box)) return GQLA_ERR_CUDA;
         if (!tc::make_tmap_bf16(&tmV, w_uv, 2, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    // the canonical shape (r_kv = 512, even g) runs on CTA pairs that keep their latent rows resident
+    if (d.r_kv == 64 * tc::ExpandSmem::kKBlocks && d.g % 2 == 0 && (N + 255) / 256 * 2 <= 0x7fffffffLL) {
+        tc::ExpandParams ep{};
+        ep.n_rows = N; ep.g = d.g; ep.r_kv = d.r_kv; ep.d_r = d.d_r;
+        ep.k_c = k_c; ep.v = v; ep.cache = cache; ep.k_r = k_r; ep.cache_stride = cache_row_stride; ep.status = nullptr;
+        auto kern = tc::expand_tc_kernel;
+        static bool attr_set[64] = {};
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::ExpandSmem::kTotal) != cudaSuccess)
+                return GQLA_ERR_CUDA;
+            if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        }
+        const unsigned pairs = (unsigned)((N + 255) / 256);
+        return tc::launch_pdl(kern, dim3(2 * pairs), dim3(tc::ExpandSmem::kThreads), tc::ExpandSmem::kTotal, st, ep, tmA, tmK,
+                              tmV) == cudaSuccess
+                   ? GQLA_OK
+                   : GQLA_ERR_CUDA;
     }
     tc::GemmParams p{};
     p.k_blocks = d.r_kv / 64;
