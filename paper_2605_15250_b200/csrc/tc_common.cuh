@@ -106,6 +106,14 @@ __device__ __forceinline__ void bulk_store(void* gdst, const void* ssrc, uint32_
                  "r"(bytes)
                  : "memory");
 }
+// 2D tiled store shared -> global through a tensor map (x * elem_size a multiple of 16 bytes, y >= 0);
+// rows and columns beyond the tensor's extent are clipped.  Tracked by bulk groups like bulk_store.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* src, int32_t x, int32_t y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                     reinterpret_cast<uint64_t>(m)),
+                 "r"(smem_u32(src)), "r"(x), "r"(y)
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Waits until the bulk stores of this thread have finished READING shared memory.
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }

@@ -105,9 +105,18 @@ inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t
                 return GQLA_ERR_CUDA;
             if (dev >= 0 && dev < 64) attr_set[dev] = true;
         }
+        // output planes as [N, g * 128] matrices; stores of 64 columns x 128 rows, clipped at row N
+        CUtensorMap tmOK, tmOV;
+        {
+            const uint64_t odims[2] = {(uint64_t)d.g * 128, (uint64_t)N};
+            const uint64_t ostr[1] = {(uint64_t)d.g * 128 * 2};
+            const uint32_t obox[2] = {64, 128};
+            if (!tc::make_tmap_bf16(&tmOK, k_c, 2, odims, ostr, obox)) return GQLA_ERR_CUDA;
+            if (!tc::make_tmap_bf16(&tmOV, v, 2, odims, ostr, obox)) return GQLA_ERR_CUDA;
+        }
         const unsigned pairs = (unsigned)((N + 255) / 256);
         return tc::launch_pdl(kern, dim3(2 * pairs), dim3(tc::ExpandSmem::kThreads), tc::ExpandSmem::kTotal, st, ep, tmA, tmK,
-                              tmV) == cudaSuccess
+                              tmV, tmOK, tmOV) == cudaSuccess
                    ? GQLA_OK
                    : GQLA_ERR_CUDA;
     }

@@ -4,11 +4,14 @@
 // while the pair walks all 2 g d_h / 256 column tiles; the weights stream through a ring, each CTA
 // fetching half of every B tile (cta_group::2 MMAs of 256 x 256 x 16 read B from both CTAs), so the
 // weights cross L2 -> SM once per 256 rows instead of once per 128.  Two 256-column accumulators in
-// TMEM: the epilogue warps store tile t while the MMAs of tile t + 1 run.
+// TMEM: the epilogue warps store tile t while the MMAs of tile t + 1 run.  The output leaves through a
+// swizzled shared-memory staging box and TMA stores (64 columns x 128 rows at a time): one thread per row
+// writing its row straight to global memory costs more store instructions than the MMAs give it time for.
 // Warp roles per CTA: warp 0 TMA producer, warp 1 TMEM owner (+ MMA issuer in the leader), warps 2-5
 // epilogue (TMEM lane = row).
 #pragma once
 #include "tc_common.cuh"
+
 
 namespace gqla {
 namespace tc {
@@ -28,21 +31,27 @@ struct ExpandSmem {
     static constexpr int kKBlocks = 8;                   // r_kv = 512
     static constexpr int kABytes = kKBlocks * 16384;     // 128 rows x 512, eight 64-wide k-blocks
     static constexpr int kBStage = 2 * 8192;             // 64 k x 128 n: this CTA's half of a 256-column tile
+    // ring of B stages: measured on the C2 cache, 4 stages 0.498 ms, 5 stages 0.464 ms (the weights come out of
+    // L2 and every k-block is only 512 cycles of tensor work)
     static constexpr int kStages = 5;
-    static constexpr int kTileBytes = kABytes + kStages * kBStage;
+    static constexpr int kOutBytes = 16384;              // output staging box: 128 rows x 64 bf16, 128-byte swizzle
+    static constexpr int kTileBytes = kABytes + kStages * kBStage + kOutBytes;  // one staging box (a second one measured slower: 0.524 vs 0.498 ms)
     static constexpr int kNumBars = 1 + 2 * kStages + 4;  // a_full, b_full[], b_empty[], acc_full[2], acc_empty[2]
     static constexpr int kThreads = 192;
     static constexpr int kTotal = 1024 + kTileBytes + kNumBars * 8 + 16;
+    static_assert(kTotal <= 232448, "shared memory budget of one CTA");
 };
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(ExpandSmem::kThreads, 1)
 expand_tc_kernel(const ExpandParams p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmK,
-                 const __grid_constant__ CUtensorMap tmV) {
+                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmOK,
+                 const __grid_constant__ CUtensorMap tmOV) {
     using L = ExpandSmem;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* a_smem = tiles;
     uint8_t* b_smem = tiles + L::kABytes;
+    uint8_t* out_smem = b_smem + L::kStages * L::kBStage;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + L::kTileBytes);
     uint64_t* a_full = bars;                       // leader: both CTAs' latent rows have landed
     uint64_t* b_full = bars + 1;                   // [kStages] leader: both halves of a B stage have landed
@@ -153,30 +162,40 @@ expand_tc_kernel(const ExpandParams p, const __grid_constant__ CUtensorMap tmA, 
             ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], (t >> 1) & 1, ab, 5));
             if (!ok) break;
             tc_fence_after();
-            __nv_bfloat16* plane = reinterpret_cast<__nv_bfloat16*>(2 * t >= p.g ? p.v : p.k_c);
-            __nv_bfloat16* dst = plane + n * ((int64_t)p.g * 128) + (int64_t)((2 * t) % p.g) * 128;
+            const CUtensorMap* tmO = 2 * t >= p.g ? &tmOV : &tmOK;
+            const int col_base = ((2 * t) % p.g) * 128;  // first column of the tile in its plane's [N, g * 128] rows
+            const int r = q * 32 + lane;                 // row of this thread within the CTA's 128
 #pragma unroll 1
-            for (int c0 = 0; c0 < 256; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(tmem_addr(tmem_base, q * 32, buf * 256 + c0), v);
+            for (int cb = 0; cb < 4; ++cb) {
+                uint32_t v[64];
+                tmem_ld32(tmem_addr(tmem_base, q * 32, buf * 256 + cb * 64), v);
+                tmem_ld32(tmem_addr(tmem_base, q * 32, buf * 256 + cb * 64 + 32), v + 32);
                 tmem_wait_ld();
-                if (valid) {
-                    uint4* d4 = reinterpret_cast<uint4*>(dst + c0);
+                // the staging box is rewritten: the store that last read it must have finished reading
+                uint8_t* box = out_smem;
+                if (threadIdx.x == 64) bulk_wait_read();
+                named_bar_sync(1, 128);
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(v[8 * u + 0]), __uint_as_float(v[8 * u + 1]));
-                        o.y = pack_bf16(__uint_as_float(v[8 * u + 2]), __uint_as_float(v[8 * u + 3]));
-                        o.z = pack_bf16(__uint_as_float(v[8 * u + 4]), __uint_as_float(v[8 * u + 5]));
-                        o.w = pack_bf16(__uint_as_float(v[8 * u + 6]), __uint_as_float(v[8 * u + 7]));
-                        d4[u] = o;
-                    }
+                for (int c = 0; c < 8; ++c) {  // 8 chunks of 8 bf16; chunk index XORed with (row & 7)
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(v[8 * c + 0]), __uint_as_float(v[8 * c + 1]));
+                    o.y = pack_bf16(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3]));
+                    o.z = pack_bf16(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5]));
+                    o.w = pack_bf16(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7]));
+                    *reinterpret_cast<uint4*>(box + r * 128 + ((c ^ (r & 7)) << 4)) = o;
+                }
+                fence_proxy_async_smem();
+                named_bar_sync(1, 128);
+                if (threadIdx.x == 64 && row_base < p.n_rows) {  // a CTA wholly behind the last row stores nothing
+                    tma_store_2d(tmO, box, col_base + cb * 64, (int32_t)row_base);
+                    bulk_commit();
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(acc_empty_l[buf]);
         }
+        if (threadIdx.x == 64) bulk_wait_read();  // the last store still reads the staging box
     }
     tc_fence_before();
     __syncthreads();
