@@ -148,11 +148,13 @@ __host__ __device__ inline BalancedStart balanced_start_serial(const int32_t* se
 }
 
 #ifdef __CUDACC__
-// Cooperative evaluation by all `nthreads` threads of a CTA.  `scratch` is shared memory of at least
-// nthreads + 4 int32.  Same result as balanced_start_serial.  Contains __syncthreads.
+// Cooperative evaluation by all `nthreads` threads of a CTA (a multiple of 32, at most 1024).  `scratch` is
+// shared memory of at least 3 * 32 + 4 int32.  Same result as balanced_start_serial.  Contains __syncthreads.
+// Thread t owns the contiguous chunk [t * chunk, (t + 1) * chunk) of the sequences; chunk sums are scanned
+// with warp shuffles and one shared-memory hop across warps.
 __device__ inline BalancedStart balanced_prepass(const int32_t* seqlens, int32_t B, int32_t S, int32_t w, int32_t W,
                                                  int32_t* scratch, int nthreads) {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarps = nthreads >> 5;
     const int32_t chunk = (B + nthreads - 1) / nthreads;
     const int32_t lo = tid * chunk < B ? tid * chunk : B, hi = lo + chunk < B ? lo + chunk : B;
     int32_t sum = 0, mx = 0;
@@ -161,40 +163,55 @@ __device__ inline BalancedStart balanced_prepass(const int32_t* seqlens, int32_t
         sum += t;
         if (t > mx) mx = t;
     }
-    int32_t* csum = scratch;            // [nthreads] chunk sums
-    int32_t* res = scratch + nthreads;  // [0] max tiles, [1] b0, [2] off_b0
-    if (tid == 0) { res[0] = 0; res[1] = B; res[2] = 0; }
-    csum[tid] = sum;
-    __syncthreads();
-    atomicMax(&res[0], mx);
-    int64_t total = 0;
-    int32_t prefix = 0;
-    for (int i = 0; i < nthreads; ++i) {
-        const int32_t c = csum[i];
-        if (i < tid) prefix += c;
-        total += c;
+    // inclusive scan of the chunk sums and maximum within the warp
+    int32_t incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    int32_t* wsum = scratch;       // [32] warp totals
+    int32_t* wmax = scratch + 32;  // [32] warp maxima
+    int32_t* wfound = scratch + 64;  // [32] first matching sequence of each warp (B: none)
+    int32_t* res = scratch + 96;   // [0] off_b0
+    if (lane == 31) wsum[wid] = incl;
+    if (lane == 0) wmax[wid] = mx;
     __syncthreads();
+    int64_t total = 0;
+    int32_t base = 0, gmax = 0;
+    for (int i = 0; i < nwarps; ++i) {
+        const int32_t c = wsum[i];
+        if (i < wid) base += c;
+        total += c;
+        gmax = max(gmax, wmax[i]);
+    }
     BalancedStart st;
-    st.share = balanced_share(total, res[0], S, W);
+    st.share = balanced_share(total, gmax, S, W);
     const int64_t mb = (int64_t)w * st.share;
     st.my_begin = (int32_t)(mb < total ? mb : total);
     const int64_t me = (int64_t)st.my_begin + st.share;
     st.my_end = (int32_t)(me < total ? me : total);
     st.total = (int32_t)total;
     // first sequence whose tiles (an empty one counts as a point) end beyond my_begin
-    int32_t off = prefix, found = B, found_off = 0;
+    int32_t off = base + incl - sum, found = B, found_off = 0;
     for (int32_t i = lo; i < hi; ++i) {
         const int32_t t = tiles_of(seqlens[i]);
         if (off + (t > 0 ? t : 1) > st.my_begin) { found = i; found_off = off; break; }
         off += t;
     }
-    if (found < B) atomicMin(&res[1], found);
+    int32_t wf = found;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wf = min(wf, __shfl_xor_sync(0xffffffffu, wf, o));
+    if (lane == 0) wfound[wid] = wf;
     __syncthreads();
-    if (found < B && res[1] == found) res[2] = found_off;
+    int32_t b0 = B;
+    for (int i = 0; i < nwarps; ++i) b0 = min(b0, wfound[i]);
+    if (found < B && found == b0) res[0] = found_off;
     __syncthreads();
-    st.b0 = res[1];
-    st.off_b0 = st.b0 < B ? res[2] : (int32_t)total;
+    st.b0 = b0;
+    st.off_b0 = b0 < B ? res[0] : (int32_t)total;
     __syncthreads();  // scratch may be reused by the caller
     return st;
 }
