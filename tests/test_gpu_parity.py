@@ -38,7 +38,7 @@ def _wl(name, batch, s_q, seed, dtype="bf16", **dims):
 
 
 def test_c0_tiny_fp32(policy):
-    """BASELINE config 0: B=1, h_q=8, g=2, d_h=16, r_kv=32, d_r=8, T=64, fp32."""
+    """Workload C0 (tiny check): B=1, h_q=8, g=2, d_h=16, r_kv=32, d_r=8, T=64, fp32."""
     from tests.parity_util import end_to_end, stagewise
     w = synth.WORKLOADS["C0"]
     errs = stagewise(w, None, 1)
@@ -283,7 +283,7 @@ def test_determinism_run_to_run():
     assert torch.equal(a1, a2)
 
 
-# ------------------------------------------------------------------ BASELINE configs at full size
+# ------------------------------------------------------------------ workloads C1-C4 at full size
 
 
 def test_c1_full_absorb():

@@ -175,7 +175,7 @@ def test_contractions_against_einsum_with_repeated_weights():
 
 
 def test_c0_three_way_agreement():
-    """BASELINE config 0: both paths against each other and against brute force."""
+    """Workload C0 (tiny check): both paths against each other and against brute force."""
     w = synth.WORKLOADS["C0"]
     x = synth.make_inputs(w)
     d = O.Dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)
