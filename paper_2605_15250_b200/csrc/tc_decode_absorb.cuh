@@ -15,17 +15,18 @@
 // operand shape comes out of L2 ([64 rows x 64 columns] 8 KB boxes, 128-byte swizzle).
 //
 // Staging: two rings per CTA, one of K groups (three 8 KB boxes = 192 columns of 64 rows) and one of
-// V groups (two box pairs = one token half of a tile), each one tile deep, filled by one producer
-// thread that polls both rings so that neither blocks the other; the loads of tile t+1 are in flight
-// while the MMAs of tile t run, and the K loads of the next piece while this piece is stored.
+// V groups (two box pairs = one token half of a tile), each one tile deep, each filled by a producer
+// thread of its own (a thread issues a tensor load only every few hundred cycles, and a tile needs 17);
+// the loads of tile t+1 are in flight while the MMAs of tile t run, and the K loads of the next piece
+// while this piece is stored.
 // Barriers are per group, not per box: every barrier operation of the issuing threads costs on the
 // order of 100 cycles next to tensor-core operand traffic, and one MMA of this shape is only 32-64
 // cycles of tensor work.
 //
-// Warp roles per CTA: warp 0 TMA producer, warp 1 TMEM owner (+ MMA issuer in the leader CTA),
-// warps 2-9 softmax.  A softmax thread owns one TMEM lane = (row, token half) and one half of that
-// lane's 64 score columns, so a row's 128 scores of a tile sit in four threads of four different
-// warps; they share the tile maximum through shared memory and keep separate partial sums.
+// Warp roles per CTA: warp 0 TMA producer of Q and K, warp 1 TMEM owner (+ MMA issuer in the leader CTA),
+// warps 2-9 softmax, warp 10 TMA producer of V.  A softmax thread owns one TMEM lane = (row, token half)
+// and one half of that lane's 64 score columns, so a row's 128 scores of a tile sit in four threads of
+// four different warps; they share the tile maximum through shared memory and keep separate partial sums.
 #pragma once
 #include "common.cuh"
 #include "sched.cuh"
@@ -61,7 +62,8 @@ struct AbsorbSmem {
     // pv_done[2] xch[2] fin epi
     static constexpr int kNumBars = 2 * kNK + 2 * kNV + 14;
     static constexpr int kSoftmaxWarps = 8;
-    static constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
+    static constexpr int kVProducerWarp = 2 + kSoftmaxWarps;  // behind the softmax warps
+    static constexpr int kThreads = 96 + 32 * kSoftmaxWarps;
     // output staging for the epilogue (P and the V ring, idle once the last P.V of a piece has completed):
     // 64 rows x 256 fp32 (the columns of one MMA m) per pass, padded pitch
     static constexpr int kOutPitch = 256 * 4 + 16;
@@ -152,14 +154,14 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
     int pi = 0;  // non-empty pieces walked so far (phase of the per-piece barriers)
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        // ------------------------------------------------------------------ TMA producer of Q and the K ring
+        // (both CTAs).  Every "full" barrier lives in the leader and counts the bytes of BOTH CTAs.
         if (elect_one()) {
             tma_prefetch_desc(&tmQ);
             tma_prefetch_desc(&tmC);
-            // every "full" barrier lives in the leader and counts the bytes of BOTH CTAs
             const uint32_t q_full_l = mapa(smem_u32(q_full), 0);
-            int ks = 0, vs = 0;           // ring slots, running across pieces
-            uint32_t kph = 1, vph = 1;    // parity that means "slot is free"
+            int ks = 0;
+            uint32_t kph = 1;  // parity that means "slot is free"
             bool ok = true;
             while (ok && walk.next(pc)) {
                 if (pc.n_tiles == 0) continue;
@@ -169,32 +171,42 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
                 for (int kb = 0; kb < 9; ++kb)
                     tma_load_2d_pair(tiles + kb * L::kBox, &tmQ, kb * 64, pc.b * p.rows_total + rho0, q_full_l);
                 const int64_t row0 = p.seq_start[pc.b] + pc.tok_begin;
-                // K groups in the order (tile, column third); V groups in the order (tile, token half).
-                // Both rings are polled with a non-blocking probe: a full ring never keeps the other one
-                // from being refilled.
-                const int total_k = 3 * pc.n_tiles, total_v = 2 * pc.n_tiles;
-                int ik = 0, kt = 0, kg = 0;  // K: index, tile, column third
-                int iv = 0, vt = 0, vh = 0;  // V: index, tile, token half
-                // the V ring doubles as the output staging of the previous piece
-                bool staging_free = pi == 0;
-                uint32_t idle = 0;
-                while (ik < total_k || iv < total_v) {
-                    bool progressed = false;
-                    if (ik < total_k && mbar_test_wait(&kempty[ks], kph)) {
+                // K groups in the order (tile, column third)
+                for (int kt = 0; kt < pc.n_tiles && ok; ++kt) {
+                    const int32_t row = (int32_t)(row0 + (int64_t)kt * 128 + cta * 64);
+#pragma unroll 1
+                    for (int kg = 0; kg < 3; ++kg) {
+                        if (!(ok = mbar_wait(&kempty[ks], kph, ab, 1))) break;
                         if (cta == 0) mbar_expect_tx(&kfull[ks], 2 * L::kKGroup);
-                        const int32_t row = (int32_t)(row0 + (int64_t)kt * 128 + cta * 64);
                         const uint32_t bar = mapa(smem_u32(&kfull[ks]), 0);
                         uint8_t* dst = tiles + L::kOffK + ks * L::kKGroup;
 #pragma unroll
                         for (int i = 0; i < 3; ++i) tma_load_2d_pair(dst + i * L::kBox, &tmC, (3 * kg + i) * 64, row, bar);
-                        ++ik;
                         if (++ks == L::kNK) { ks = 0; kph ^= 1; }
-                        if (++kg == 3) { kg = 0; ++kt; }
-                        progressed = true;
                     }
-                    if (!staging_free && mbar_test_wait(epi_done, (pi - 1) & 1)) staging_free = true;
-                    // the V boxes of a tile are re-reads of its K boxes: issue them after those, so they hit L2
-                    if (iv < total_v && kt > vt && staging_free && mbar_test_wait(&vempty[vs], vph)) {
+                }
+                ++pi;
+            }
+        }
+    } else if (warp == L::kVProducerWarp) {
+        // ------------------------------------------------------------------ TMA producer of the V ring (both
+        // CTAs).  A thread issues a tensor load only every few hundred cycles, and a tile needs 17 of them:
+        // the two rings are fed by two threads.  V groups in the order (tile, token half); a V slot is free
+        // only after P.V of the previous tile, i.e. after Qh Kh^T of this tile has read the same cache rows
+        // as K boxes, so the V boxes come out of L2.
+        if (elect_one()) {
+            int vs = 0;
+            uint32_t vph = 1;
+            bool ok = true;
+            while (ok && walk.next(pc)) {
+                if (pc.n_tiles == 0) continue;
+                // the V ring doubles as the output staging of the previous piece
+                if (pi > 0 && !(ok = mbar_wait(epi_done, (pi - 1) & 1, ab, 16))) break;
+                const int64_t row0 = p.seq_start[pc.b] + pc.tok_begin;
+                for (int vt = 0; vt < pc.n_tiles && ok; ++vt) {
+#pragma unroll 1
+                    for (int vh = 0; vh < 2; ++vh) {
+                        if (!(ok = mbar_wait(&vempty[vs], vph, ab, 2))) break;
                         if (cta == 0) mbar_expect_tx(&vfull[vs], 2 * L::kVGroup);
                         const int32_t row = (int32_t)(row0 + (int64_t)vt * 128 + vh * 64);
                         const uint32_t bar = mapa(smem_u32(&vfull[vs]), 0);
@@ -204,17 +216,7 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
                         for (int mi = 0; mi < 4; ++mi)
                             tma_load_2d_pair(dst + mi * L::kBox, &tmC, 256 * (mi >> 1) + 128 * (int)cta + 64 * (mi & 1), row,
                                              bar);
-                        ++iv;
                         if (++vs == L::kNV) { vs = 0; vph ^= 1; }
-                        if (++vh == 2) { vh = 0; ++vt; }
-                        progressed = true;
-                    }
-                    if (progressed) {
-                        idle = 0;
-                    } else {
-                        ++idle;
-                        if ((idle & 63u) == 63u && ab.raised()) { ok = false; break; }
-                        if (idle > kWaitSpins) { ab.raise(1); ok = false; break; }
                     }
                 }
                 ++pi;
