@@ -5,7 +5,9 @@
 //   S = Q K^T   Q: the group's h_q/g heads x s_q queries (R rows), K = [K_C[:, j] ; k_R]  (192 wide)
 //   O = P V     P = exp2(S * scale*log2e - m),  V = V[:, j]                                (128 wide)
 //
-// The MMA tile is 128 rows, the group only has R = (h_q/g)*s_q <= 128 of them, so the R query rows
+// The MMA tile is 128 rows, the group only has (h_q/g)*s_q <= 128 of them.  Heads per group and query
+// positions are each padded to a power of two (R rows in all; padding rows hold zeros or the next
+// sequence's queries and are dropped at the store), and the R query rows
 // are replicated F = 128/R times down the tile and replica f only keeps the scores of tokens
 // [f*R, (f+1)*R) of each 128-token tile (its other probabilities are zero).  Every TMEM lane thus
 // runs an independent online softmax over a disjoint token subset -- no cross-thread reduction in
@@ -234,7 +236,7 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
         const int f = Lr / R;                // replica: token sub-block of every tile
         const int pq = r / p.hpg_box;        // query position within the step
         const int il = r % p.hpg_box;        // head within the group
-        const bool row_valid = il < p.hpg;
+        const bool row_valid = il < p.hpg && pq < p.s_q;  // padding rows are computed and dropped
         const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
         const int col0 = R < 32 ? q * 32 : f * R;  // first column of the warp's window (warp-uniform)
         const int sub = R < 32 ? lane / R : 0;     // which R-column sub-block of the window is this thread's
@@ -377,7 +379,7 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
                 named_bar_sync(1, 128);
                 for (int rr = mrow0; rr < R; rr += 16) {
                     const int pp = rr / p.hpg_box, ii = rr % p.hpg_box;
-                    if (ii >= p.hpg) continue;
+                    if (ii >= p.hpg || pp >= p.s_q) continue;
                     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                     for (int ff = 0; ff < F; ++ff) {

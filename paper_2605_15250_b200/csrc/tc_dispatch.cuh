@@ -22,22 +22,29 @@ inline bool tc_gemm_covers(const gqla_dims& d, gqla_dtype dtype) {
            hpg <= 128 && 128 % hpg == 0;
 }
 
-// path: 0 = absorb, 1 = GQA
-inline int gqa_rows(const gqla_dims& d, int32_t s_q, int* hpg_box) {
-    const int hpg = d.h_q / d.g;
-    const int hb = hpg * s_q >= 8 ? hpg : 8 / s_q;
+inline int next_pow2(int x) {
+    int p = 1;
+    while (p < x) p <<= 1;
+    return p;
+}
+// Rows of the GQA kernel's query block: heads per group and query positions are each padded to a power
+// of two (the padding rows are computed and dropped), at least 8 rows in all.
+inline int gqa_rows(const gqla_dims& d, int32_t s_q, int* hpg_box, int* sq_box) {
+    const int sb = next_pow2(s_q);
+    int hb = next_pow2(d.h_q / d.g);
+    if (hb * sb < 8) hb = 8 / sb;
     if (hpg_box != nullptr) *hpg_box = hb;
-    return hb * s_q;
+    if (sq_box != nullptr) *sq_box = sb;
+    return hb * sb;
 }
 inline bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 
 inline bool tc_covers(const gqla_dims& d, gqla_dtype dtype, int32_t s_q, int32_t path) {
     if (dtype != GQLA_BF16) return false;
     if (path == 1) {
-        // the group's R = (h_q/g) * s_q rows are replicated 128/R times down the MMA tile: R must divide 128
-        if (d.d_h != 128 || d.d_r != 64 || s_q < 1 || s_q > 8 || !is_pow2(s_q)) return false;
-        const int R = gqa_rows(d, s_q, nullptr);
-        return is_pow2(d.h_q / d.g) && R >= 8 && R <= 128;
+        // the group's (h_q/g) * s_q rows, padded to R, are replicated 128/R times down the MMA tile
+        if (d.d_h != 128 || d.d_r != 64 || s_q < 1 || s_q > 8) return false;
+        return gqa_rows(d, s_q, nullptr, nullptr) <= 128;
     }
     // absorb path: the pair kernel is specialised for the 512 + 64 latent row
     return d.r_kv == 512 && d.d_r == 64 && s_q >= 1 && s_q <= 8;
@@ -329,14 +336,14 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
     const int64_t units = balanced ? (int64_t)workers * d.g : (int64_t)B * S * d.g;
     if (units > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     const int hpg = d.h_q / d.g;
-    int hpg_box = 0;
-    const int R = gqa_rows(d, s_q, &hpg_box);
+    int hpg_box = 0, sq_box = 0;
+    const int R = gqa_rows(d, s_q, &hpg_box, &sq_box);
     CUtensorMap tmQ, tmK, tmR, tmV;
     {
         const int feat = d.d_h + d.d_r;
         const uint64_t dims[4] = {(uint64_t)feat, (uint64_t)hpg, (uint64_t)d.g, (uint64_t)B * s_q};
         const uint64_t str[3] = {(uint64_t)feat * 2, (uint64_t)hpg * feat * 2, (uint64_t)d.h_q * feat * 2};
-        const uint32_t box[4] = {64, (uint32_t)hpg_box, 1, (uint32_t)s_q};
+        const uint32_t box[4] = {64, (uint32_t)hpg_box, 1, (uint32_t)sq_box};  // beyond a dimension: zero fill
         if (!tc::make_tmap_bf16(&tmQ, q, 4, dims, str, box)) return GQLA_ERR_CUDA;
     }
     {

@@ -196,27 +196,32 @@ def test_absorb_balanced_plan_llama(s_q):
     _balanced_absorb_case(w, synth.make_seqlens(w.with_(seqlen_range=(0, 1500))), 3)
 
 
-@pytest.mark.parametrize("h_q,g", [(128, 4), (64, 8), (64, 4), (16, 8)])
+@pytest.mark.parametrize("h_q,g", [(128, 4), (64, 8), (64, 4), (16, 8), (28, 4), (20, 4)])
 @pytest.mark.parametrize("s_q", [1, 2])
 def test_shape_variants_of_the_paper(h_q, g, s_q):
     """Operating points the paper discusses besides the canonical one: g = 4 (cache 2176 B/token, Table
-    "roofline"), h_q = 64 (Sec. 4.2), and few heads per group; fixed and balanced plans."""
+    "roofline"), h_q = 64 (Sec. 4.2), few heads per group, and head counts whose heads per group are not a
+    power of two (h_q = 28 at g = 4, the Qwen2.5-7B setup of Sec. 5; h_q = 20); fixed and balanced plans.
+    Both decode paths stay on the tensor-core kernels."""
     from tests.parity_util import end_to_end, stagewise
+    dims = B.make_dims(h_q, g, 128, 512, 64)
+    assert B.kernel_for(dims, torch.bfloat16, s_q, "absorb") == "tcgen05"
+    assert B.kernel_for(dims, torch.bfloat16, s_q, "gqa") == "tcgen05"
     w = _wl("variant", 5, s_q, 131, h_q=h_q, g=g, d_h=128, r_kv=512, d_r=64)
     seqlens = np.array([700, 0, 129, 2050, 64], dtype=np.int32)
     stagewise(w, seqlens, 3, 4.0)
     end_to_end(w, seqlens, -3, q_gain=4.0)
 
 
-@pytest.mark.parametrize("s_q", [3, 4])
+@pytest.mark.parametrize("s_q", [3, 4, 5, 8])
 def test_speculative_query_counts(s_q):
-    """s_q >= 3 (speculative decoding, Sec. 4.2): the absorb path stays on the tensor-core kernel (more
-    row blocks); the GQA path does for s_q = 4 (its rows still divide the 128-row tile) and falls back to
-    the generic kernel for s_q = 3; the causal mask covers all s_q positions."""
+    """s_q >= 3 (speculative decoding, Sec. 4.2): both paths stay on the tensor-core kernels (the absorb
+    path with more row blocks, the GQA path with s_q = 3 padded to four query positions per head); the
+    causal mask covers all s_q positions."""
     from tests.parity_util import end_to_end, stagewise
     w = _wl("spec", 4, s_q, 132, **CANON)
     assert B.kernel_for(B.make_dims(**CANON), torch.bfloat16, s_q, "absorb") == "tcgen05"
-    assert B.kernel_for(B.make_dims(**CANON), torch.bfloat16, s_q, "gqa") == ("tcgen05" if s_q == 4 else "generic")
+    assert B.kernel_for(B.make_dims(**CANON), torch.bfloat16, s_q, "gqa") == "tcgen05"
     seqlens = np.array([300, 2, 1029, 64], dtype=np.int32)
     stagewise(w, seqlens, 2, 4.0)
     end_to_end(w, seqlens, 2, q_gain=4.0)
