@@ -191,8 +191,9 @@ int32_t gqla_balanced_workers(const gqla_dims* dims, gqla_dtype dtype, int32_t s
 int32_t gqla_visible_limit(int32_t seqlen, int32_t s_q, int32_t p);
 /* 0-indexed group of 0-indexed head: the paper's j(i) = ceil(i/(h_q/g)); -1 on bad input. */
 int32_t gqla_group_of_head(const gqla_dims* dims, int32_t head);
-/* Name of the kernel family the current policy selects for a decode call
- * ("tcgen05" or "generic"); path: 0 = absorb, 1 = GQA. */
+/* Name of the kernel family the current policy selects ("tcgen05" or "generic") for a decode call
+ * (path: 0 = absorb, 1 = GQA) or for the grouped projections gqla_absorb_q, gqla_up_proj and
+ * gqla_combine_up_proj (path: 2; s_q is ignored). */
 const char* gqla_kernel_for(const gqla_dims* dims, gqla_dtype dtype, int32_t s_q, int32_t path);
 const char* gqla_status_str(gqla_status s);
 

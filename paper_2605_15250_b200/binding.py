@@ -123,7 +123,7 @@ def get_policy() -> int:
 
 def kernel_for(dims: GqlaDims, dtype: torch.dtype, s_q: int, path: str) -> str:
     code = GQLA_BF16 if dtype == torch.bfloat16 else GQLA_F32
-    return lib().gqla_kernel_for(ctypes.byref(dims), code, s_q, 0 if path == "absorb" else 1).decode()
+    return lib().gqla_kernel_for(ctypes.byref(dims), code, s_q, {"absorb": 0, "gqa": 1, "projections": 2}[path]).decode()
 
 
 # ------------------------------------------------------------------ the six calls

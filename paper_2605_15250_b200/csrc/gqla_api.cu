@@ -121,8 +121,9 @@ int32_t gqla_group_of_head(const gqla_dims* d, int32_t head) {
 
 const char* gqla_kernel_for(const gqla_dims* d, gqla_dtype dtype, int32_t s_q, int32_t path) {
     if (check_dims(d) != GQLA_OK) return "invalid";
-    if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, path)) return "tcgen05";
-    return "generic";
+    if (g_policy.load() != GQLA_POLICY_AUTO) return "generic";
+    if (path == 2) return tc_gemm_covers(*d, dtype) ? "tcgen05" : "generic";
+    return tc_covers(*d, dtype, s_q, path) ? "tcgen05" : "generic";
 }
 
 gqla_status gqla_absorb_q(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, const void* q_c,

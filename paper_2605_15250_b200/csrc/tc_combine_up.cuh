@@ -16,6 +16,7 @@ namespace tc {
 
 struct CombineUpParams {
     int32_t S, s_q, h_q, g, hpg, r_kv;
+    int32_t hpb;            // heads per group padded to a power of two (head slots of a tile)
     int64_t positions;      // B * s_q
     const float* o_part;    // [B, S, s_q*h_q, r_kv]
     const float* lse_part;  // [B, S, s_q*h_q]
@@ -112,11 +113,12 @@ combine_up_tc_kernel(const CombineUpParams p, const __grid_constant__ CUtensorMa
     } else {
         // ------------------------------------------------------------------ builders, then epilogue
         const int q = warp & 3;  // TMEM lane quadrant of this warp; it holds tile rows [16q, 16q + 16)
-        // global row of tile row tr: position m_tile * (64/hpg) + tr / hpg, head j * hpg + tr % hpg
+        // global row of tile row tr: position m_tile * (64/hpb) + tr / hpb, head j * hpg + tr % hpb (head
+        // slots beyond the group's hpg heads stay empty)
         auto row_of = [&](int tr, int64_t* part_row, int64_t* out_row) -> bool {
-            const int64_t pos = (int64_t)m_tile * (L::kRows / p.hpg) + tr / p.hpg;
-            if (pos >= p.positions) return false;
-            const int i = j * p.hpg + tr % p.hpg;
+            const int64_t pos = (int64_t)m_tile * (L::kRows / p.hpb) + tr / p.hpb;
+            if (pos >= p.positions || tr % p.hpb >= p.hpg) return false;
+            const int i = j * p.hpg + tr % p.hpb;
             const int64_t b = pos / p.s_q;
             const int pq = (int)(pos % p.s_q);
             *part_row = b * p.S * rows_per_seq + (int64_t)pq * p.h_q + i;  // split 0; + k * rows_per_seq

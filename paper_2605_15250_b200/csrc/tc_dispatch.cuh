@@ -13,20 +13,19 @@
 namespace gqla {
 
 inline bool stride_ok(int64_t elems) { return (elems * 2) % 16 == 0; }
-
-// Shapes the grouped tcgen05 GEMMs cover: bf16, d_h = 128, r_kv a multiple of 256, d_r a multiple
-// of 8, heads-per-group dividing 128.
-inline bool tc_gemm_covers(const gqla_dims& d, gqla_dtype dtype) {
-    const int hpg = d.h_q / d.g;
-    return dtype == GQLA_BF16 && d.d_h == 128 && d.r_kv % 256 == 0 && d.r_kv <= 4096 && d.d_r % 8 == 0 &&
-           hpg <= 128 && 128 % hpg == 0;
-}
-
 inline int next_pow2(int x) {
     int p = 1;
     while (p < x) p <<= 1;
     return p;
 }
+
+// Shapes the grouped tcgen05 GEMMs cover: bf16, d_h = 128, r_kv a multiple of 256, d_r a multiple
+// of 8, at most 128 heads per group (padded to a power of two of head slots per query position).
+inline bool tc_gemm_covers(const gqla_dims& d, gqla_dtype dtype) {
+    const int hpg = d.h_q / d.g;
+    return dtype == GQLA_BF16 && d.d_h == 128 && d.r_kv % 256 == 0 && d.r_kv <= 4096 && d.d_r % 8 == 0 && hpg <= 128;
+}
+
 // Rows of the GQA kernel's query block: heads per group and query positions are each padded to a power
 // of two (the padding rows are computed and dropped), at least 8 rows in all.
 inline int gqa_rows(const gqla_dims& d, int32_t s_q, int* hpg_box, int* sq_box) {
@@ -144,19 +143,19 @@ inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t
 
 // 4-D view of a [B*s_q, h_q, feat] activation: (feat, head-in-group, group, position).
 inline bool make_grouped_act_map(CUtensorMap* m, const void* base, const gqla_dims& d, int feat, int64_t positions) {
-    const int hpg = d.h_q / d.g;
+    const int hpg = d.h_q / d.g, hpb = next_pow2(hpg);
     const uint64_t dims[4] = {(uint64_t)feat, (uint64_t)hpg, (uint64_t)d.g, (uint64_t)positions};
     const uint64_t str[3] = {(uint64_t)feat * 2, (uint64_t)hpg * feat * 2, (uint64_t)d.h_q * feat * 2};
-    const uint32_t box[4] = {64, (uint32_t)hpg, 1, (uint32_t)(128 / hpg)};
+    const uint32_t box[4] = {64, (uint32_t)hpb, 1, (uint32_t)(128 / hpb)};  // beyond the hpg heads: zero fill
     return tc::make_tmap_bf16(m, base, 4, dims, str, box);
 }
 
 inline gqla_status tc_absorb_q(const gqla_dims& d, gqla_dtype dtype, int32_t B, int32_t s_q, const void* q_c,
                                const void* q_r, const void* w_uk, void* q_hat, cudaStream_t st) {
     if (!tc_gemm_covers(d, dtype)) return GQLA_ERR_UNSUPPORTED;
-    const int hpg = d.h_q / d.g;
+    const int hpg = d.h_q / d.g, hpb = next_pow2(hpg);
     const int64_t positions = (int64_t)B * s_q;
-    const int64_t m_tiles = (positions + 128 / hpg - 1) / (128 / hpg);
+    const int64_t m_tiles = (positions + 128 / hpb - 1) / (128 / hpb);
     if (m_tiles > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     CUtensorMap tmA, tmB;
     if (!make_grouped_act_map(&tmA, q_c, d, d.d_h, positions)) return GQLA_ERR_CUDA;
@@ -170,7 +169,7 @@ inline gqla_status tc_absorb_q(const gqla_dims& d, gqla_dtype dtype, int32_t B, 
     tc::GemmParams p{};
     p.k_blocks = d.d_h / 64;
     p.m_total = positions;
-    p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
+    p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpb = hpb; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
     p.out0 = q_hat; p.aux_in = q_r;
     cudaError_t e = tc::gemm_launch<tc::kGemmAbsorbQ, 256, false>(
         p, tmA, tmB, tmB, dim3((unsigned)m_tiles, (unsigned)d.g, (unsigned)(d.r_kv / 256)), st);
@@ -180,9 +179,9 @@ inline gqla_status tc_absorb_q(const gqla_dims& d, gqla_dtype dtype, int32_t B, 
 inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, int32_t s_q, const void* o_hat,
                               const void* w_uv, void* o, cudaStream_t st) {
     if (!tc_gemm_covers(d, dtype)) return GQLA_ERR_UNSUPPORTED;
-    const int hpg = d.h_q / d.g;
+    const int hpg = d.h_q / d.g, hpb = next_pow2(hpg);
     const int64_t positions = (int64_t)B * s_q;
-    const int64_t m_tiles = (positions + 128 / hpg - 1) / (128 / hpg);
+    const int64_t m_tiles = (positions + 128 / hpb - 1) / (128 / hpb);
     if (m_tiles > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     CUtensorMap tmA, tmB;
     if (!make_grouped_act_map(&tmA, o_hat, d, d.r_kv, positions)) return GQLA_ERR_CUDA;
@@ -196,7 +195,7 @@ inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, i
     tc::GemmParams p{};
     p.k_blocks = d.r_kv / 64;
     p.m_total = positions;
-    p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
+    p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpb = hpb; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
     p.out0 = o;
     cudaError_t e =
         tc::gemm_launch<tc::kGemmUpProj, 128, true>(p, tmA, tmB, tmB, dim3((unsigned)m_tiles, (unsigned)d.g, 1), st);
@@ -207,12 +206,12 @@ inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, i
 inline gqla_status tc_combine_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, int32_t s_q, int32_t S,
                                       const float* o_part, const float* lse_part, const void* w_uv, void* o, float* lse,
                                       cudaStream_t st) {
-    const int hpg = d.h_q / d.g;
-    if (!tc_gemm_covers(d, dtype) || S > tc::CombineUpSmem::kMaxS || hpg > 64 ||
+    const int hpg = d.h_q / d.g, hpb = next_pow2(hpg);
+    if (!tc_gemm_covers(d, dtype) || S > tc::CombineUpSmem::kMaxS || hpb > 64 ||
         d.r_kv > tc::CombineUpSmem::kMaxChunks * tc::CombineUpSmem::kChunkK)
         return GQLA_ERR_UNSUPPORTED;
     const int64_t positions = (int64_t)B * s_q;
-    const int64_t m_tiles = (positions + 64 / hpg - 1) / (64 / hpg);
+    const int64_t m_tiles = (positions + 64 / hpb - 1) / (64 / hpb);
     if (m_tiles > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     CUtensorMap tmB;
     {
@@ -222,7 +221,7 @@ inline gqla_status tc_combine_up_proj(const gqla_dims& d, gqla_dtype dtype, int3
         if (!tc::make_tmap_bf16(&tmB, w_uv, 2, dims, str, box)) return GQLA_ERR_CUDA;
     }
     tc::CombineUpParams p{};
-    p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.r_kv = d.r_kv;
+    p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpb = hpb; p.r_kv = d.r_kv;
     p.positions = positions; p.o_part = o_part; p.lse_part = lse_part; p.out = o; p.lse = lse; p.status = nullptr;
     auto kern = tc::combine_up_tc_kernel;
     static bool attr_set[64] = {};

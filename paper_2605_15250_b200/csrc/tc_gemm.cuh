@@ -17,6 +17,7 @@ struct GemmParams {
     int32_t k_blocks;   // K / 64
     int64_t m_total;    // expand: cache rows N;  others: B * s_q (query positions)
     int32_t h_q, g, hpg, d_h, r_kv, d_r;
+    int32_t hpb;        // heads per group padded to a power of two: a tile is 128/hpb positions x hpb head slots
     void* out0;         // expand: k_c;  absorb_q: q_hat;  up_proj: o
     void* out1;         // expand: v
     const void* aux_in; // absorb_q: q_r (copied into q_hat's tail);  expand: cache (for the k_R copy)
@@ -98,12 +99,13 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
                 if (MODE == kGemmExpand) {
                     tma_load_2d(a_dst, &tmA, kb * 64, m_tile * 128, &full[s]);
                 } else {
-                    // 4-D view (feature, head-in-group, group, query position): 128/hpg positions x hpg heads
+                    // 4-D view (feature, head-in-group, group, query position): 128/hpb positions x hpb head
+                    // slots (slots beyond the group's hpg heads read zeros and are not stored)
                     asm volatile(
                         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], "
                         "[%1, {%3, %4, %5, %6}], [%2];" ::"r"(smem_u32(a_dst)),
                         "l"(reinterpret_cast<uint64_t>(&tmA)), "r"(smem_u32(&full[s])), "r"(kb * 64), "r"(0), "r"(j),
-                        "r"(m_tile * (128 / p.hpg))
+                        "r"(m_tile * (128 / p.hpb))
                         : "memory");
                 }
                 if (B_MN && MODE == kGemmExpand) {
@@ -167,9 +169,10 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
                 }
             }
         } else {
-            const int64_t bp = (int64_t)m_tile * (128 / p.hpg) + row / p.hpg;
-            const int i = j * p.hpg + row % p.hpg;
-            if (bp < p.m_total) {
+            const int64_t bp = (int64_t)m_tile * (128 / p.hpb) + row / p.hpb;
+            const int il = row % p.hpb;
+            const int i = j * p.hpg + il;
+            if (bp < p.m_total && il < p.hpg) {
                 const int64_t r = bp * p.h_q + i;
                 if (MODE == kGemmAbsorbQ) {
                     __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out0) + r * (p.r_kv + p.d_r);

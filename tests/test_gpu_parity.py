@@ -207,6 +207,7 @@ def test_shape_variants_of_the_paper(h_q, g, s_q):
     dims = B.make_dims(h_q, g, 128, 512, 64)
     assert B.kernel_for(dims, torch.bfloat16, s_q, "absorb") == "tcgen05"
     assert B.kernel_for(dims, torch.bfloat16, s_q, "gqa") == "tcgen05"
+    assert B.kernel_for(dims, torch.bfloat16, s_q, "projections") == "tcgen05"
     w = _wl("variant", 5, s_q, 131, h_q=h_q, g=g, d_h=128, r_kv=512, d_r=64)
     seqlens = np.array([700, 0, 129, 2050, 64], dtype=np.int32)
     stagewise(w, seqlens, 3, 4.0)
