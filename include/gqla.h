@@ -117,6 +117,16 @@ gqla_status gqla_expand_cache(const gqla_dims* dims, gqla_dtype dtype, int64_t N
                               int64_t cache_row_stride, const void* w_uk, const void* w_uv, void* k_c, void* v,
                               void* k_r, void* stream);
 
+/* Sec. 3.1 again, for the rows a decode step appends: the expansion is a per-token linear map, so a
+ * cache that was expanded once stays current if every step expands only its new rows.  For each
+ * sequence b and p < s_q with seqlens[b] - s_q + p >= 0, row n = seq_start[b] + seqlens[b] - s_q + p of
+ * k_c, v (and k_r unless NULL) is computed from row n of the latent cache; seqlens already counts the
+ * new tokens, whose latent rows the caller has written.  No other row is touched.  Layouts as for
+ * gqla_expand_cache; seq_start int64 [B] and seqlens int32 [B] are device arrays. */
+gqla_status gqla_append_expand(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, const void* cache,
+                               int64_t cache_row_stride, const int64_t* seq_start, const int32_t* seqlens,
+                               const void* w_uk, const void* w_uv, void* k_c, void* v, void* k_r, void* stream);
+
 /* Eq. (mha): split-KV attention of each head over its group's K_C, V plus the shared k^R.
  *   q [B, s_q, h_q, d_h+d_r] (= [q^C ; q^R]);  k_c, v [N, g, d_h];  k_r [N, .] with row stride
  *   k_r_row_stride (elements; d_r for a dense plane, r_kv+d_r when aliasing the latent cache);

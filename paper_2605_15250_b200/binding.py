@@ -37,6 +37,8 @@ _PROTOTYPES = {
     "gqla_absorb_q": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_decode_absorb": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
                                      c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_append_expand": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_int64, c_void_p, c_void_p, c_void_p,
+                                     c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_expand_cache": (c_int32, [c_void_p, c_int32, c_int64, c_void_p, c_int64, c_void_p, c_void_p, c_void_p,
                                     c_void_p, c_void_p, c_void_p]),
     "gqla_decode_gqa": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
@@ -160,6 +162,18 @@ def gqla_expand_cache(dims: GqlaDims, cache: torch.Tensor, w_uk: torch.Tensor, w
     _check(lib().gqla_expand_cache(ctypes.byref(dims), _dtype_code(cache), cache.shape[0], _ptr(cache),
                                    cache.stride(0), _ptr(w_uk), _ptr(w_uv), _ptr(k_c), _ptr(v), _ptr(k_r),
                                    _stream()), "gqla_expand_cache")
+
+
+def gqla_append_expand(dims: GqlaDims, s_q: int, cache: torch.Tensor, seq_start: torch.Tensor, seqlens: torch.Tensor,
+                       w_uk: torch.Tensor, w_uv: torch.Tensor, k_c: torch.Tensor, v: torch.Tensor,
+                       k_r: torch.Tensor | None) -> None:
+    """Expands only the s_q rows each sequence appended in this step (Sec. 3.1, per-token map)."""
+    _contig(w_uk, w_uv, k_c, v, k_r, seq_start, seqlens)
+    assert cache.dim() == 2 and cache.stride(1) == 1
+    assert seq_start.dtype == torch.int64 and seqlens.dtype == torch.int32
+    _check(lib().gqla_append_expand(ctypes.byref(dims), _dtype_code(cache), seqlens.shape[0], s_q, _ptr(cache),
+                                    cache.stride(0), _ptr(seq_start), _ptr(seqlens), _ptr(w_uk), _ptr(w_uv), _ptr(k_c),
+                                    _ptr(v), _ptr(k_r), _stream()), "gqla_append_expand")
 
 
 def gqla_decode_gqa(dims: GqlaDims, q: torch.Tensor, k_c: torch.Tensor, v: torch.Tensor, k_r: torch.Tensor,

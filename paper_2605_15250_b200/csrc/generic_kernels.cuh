@@ -320,4 +320,74 @@ __global__ void __launch_bounds__(256) expand_cache_generic_kernel(int64_t N, in
         }
 }
 
+// The same expansion for the rows appended by the current decode step only: the last s_q rows of every
+// sequence (positions seqlens[b] - s_q + p >= 0).  One block stages kExpandRows such rows and computes one
+// (plane, group) slice of them, so a weight slice is read once per block.  Thread (d, q) sums a quarter
+// of the latent index for output column d of all staged rows (the weight loads of a warp are coalesced
+// and several are in flight); the four quarters meet in shared memory.
+constexpr int kAppendThreads = 512, kAppendKSplit = 4, kAppendCols = kAppendThreads / kAppendKSplit;
+template <typename T>
+__global__ void __launch_bounds__(kAppendThreads)
+append_expand_kernel(int32_t B, int32_t s_q, int32_t g, int32_t d_h, int32_t r_kv, int32_t d_r,
+                     const T* __restrict__ cache, int64_t cache_stride, const int64_t* __restrict__ seq_start,
+                     const int32_t* __restrict__ seqlens, const T* __restrict__ w_uk, const T* __restrict__ w_uv,
+                     T* __restrict__ k_c, T* __restrict__ v, T* __restrict__ k_r) {
+    extern __shared__ float cs[];                 // [kExpandRows][r_kv] latent rows
+    float* red = cs + kExpandRows * r_kv;         // [kAppendKSplit][kExpandRows][kAppendCols] partial sums
+    __shared__ int64_t rows[kExpandRows];
+    const int64_t u0 = (int64_t)blockIdx.x * kExpandRows;  // first (sequence, new token) unit of this block
+    if (threadIdx.x < kExpandRows) {
+        const int64_t u = u0 + threadIdx.x;
+        int64_t n = -1;
+        if (u < (int64_t)B * s_q) {
+            const int32_t b = (int32_t)(u / s_q), pq = (int32_t)(u % s_q);
+            const int32_t pos = seqlens[b] - s_q + pq;
+            if (pos >= 0) n = seq_start[b] + pos;
+        }
+        rows[threadIdx.x] = n;
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < kExpandRows * r_kv; t += blockDim.x) {
+        const int rr = t / r_kv, c = t % r_kv;
+        cs[t] = rows[rr] >= 0 ? ldf(cache + rows[rr] * cache_stride + c) : 0.f;
+    }
+    __syncthreads();
+    const int plane = blockIdx.y / g, j = blockIdx.y % g;
+    const T* w = (plane == 0 ? w_uk : w_uv) + (int64_t)j * r_kv * d_h;
+    T* out = plane == 0 ? k_c : v;
+    const int dl = threadIdx.x % kAppendCols, kq = threadIdx.x / kAppendCols;
+    const int r_lo = (int)((int64_t)r_kv * kq / kAppendKSplit), r_hi = (int)((int64_t)r_kv * (kq + 1) / kAppendKSplit);
+    for (int d0 = 0; d0 < d_h; d0 += kAppendCols) {
+        const int d = d0 + dl;
+        float acc[kExpandRows];
+#pragma unroll
+        for (int rr = 0; rr < kExpandRows; ++rr) acc[rr] = 0.f;
+        if (d < d_h) {
+#pragma unroll 8
+            for (int r = r_lo; r < r_hi; ++r) {
+                const float a = ldf(w + (int64_t)r * d_h + d);
+#pragma unroll
+                for (int rr = 0; rr < kExpandRows; ++rr) acc[rr] = fmaf(a, cs[rr * r_kv + r], acc[rr]);
+            }
+        }
+#pragma unroll
+        for (int rr = 0; rr < kExpandRows; ++rr) red[(kq * kExpandRows + rr) * kAppendCols + dl] = acc[rr];
+        __syncthreads();
+        // thread (dl, kq) finishes rows kq and kq + kAppendKSplit
+        if (d < d_h)
+            for (int rr = kq; rr < kExpandRows; rr += kAppendKSplit) {
+                float sum = 0.f;
+#pragma unroll
+                for (int q = 0; q < kAppendKSplit; ++q) sum += red[(q * kExpandRows + rr) * kAppendCols + dl];
+                if (rows[rr] >= 0) stf(out + (rows[rr] * g + j) * d_h + d, sum);
+            }
+        __syncthreads();
+    }
+    if (k_r != nullptr && blockIdx.y == 0)
+        for (int t = threadIdx.x; t < kExpandRows * d_r; t += blockDim.x) {
+            const int rr = t / d_r, c = t % d_r;
+            if (rows[rr] >= 0) k_r[rows[rr] * d_r + c] = cache[rows[rr] * cache_stride + r_kv + c];
+        }
+}
+
 }  // namespace gqla

@@ -249,6 +249,43 @@ gqla_status gqla_expand_cache(const gqla_dims* d, gqla_dtype dtype, int64_t N, c
     return launch_status();
 }
 
+gqla_status gqla_append_expand(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, const void* cache,
+                               int64_t cache_row_stride, const int64_t* seq_start, const int32_t* seqlens,
+                               const void* w_uk, const void* w_uv, void* k_c, void* v, void* k_r, void* stream) {
+    gqla_status s;
+    if ((s = check_dims(d)) != GQLA_OK) return s;
+    if ((s = check_dtype(dtype)) != GQLA_OK) return s;
+    if (B < 0 || s_q < 1 || cache_row_stride < d->r_kv + d->d_r) return GQLA_ERR_SHAPE;
+    if (B == 0) return GQLA_OK;
+    if (cache == nullptr || seq_start == nullptr || seqlens == nullptr || w_uk == nullptr || w_uv == nullptr ||
+        k_c == nullptr || v == nullptr)
+        return GQLA_ERR_NULL;
+    if (!aligned16(cache) || !aligned16(w_uk) || !aligned16(w_uv) || !aligned16(k_c) || !aligned16(v) ||
+        !aligned16(k_r))
+        return GQLA_ERR_ALIGN;
+    if (g_policy.load() == GQLA_POLICY_AUTO) {
+        s = tc_append_expand(*d, dtype, B, s_q, cache, cache_row_stride, seq_start, seqlens, w_uk, w_uv, k_c, v, k_r,
+                             (cudaStream_t)stream);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
+    const size_t smem = ((size_t)kExpandRows * d->r_kv + (size_t)kAppendKSplit * kExpandRows * kAppendCols) * sizeof(float);
+    if (smem > 48 * 1024 || 2 * d->g > 65535) return GQLA_ERR_UNSUPPORTED;
+    const int64_t blocks = ((int64_t)B * s_q + kExpandRows - 1) / kExpandRows;
+    if (blocks > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    const dim3 grid((unsigned)blocks, (unsigned)(2 * d->g));
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == GQLA_BF16)
+        append_expand_kernel<__nv_bfloat16><<<grid, kAppendThreads, smem, st>>>(
+            B, s_q, d->g, d->d_h, d->r_kv, d->d_r, (const __nv_bfloat16*)cache, cache_row_stride, seq_start, seqlens,
+            (const __nv_bfloat16*)w_uk, (const __nv_bfloat16*)w_uv, (__nv_bfloat16*)k_c, (__nv_bfloat16*)v,
+            (__nv_bfloat16*)k_r);
+    else
+        append_expand_kernel<float><<<grid, kAppendThreads, smem, st>>>(B, s_q, d->g, d->d_h, d->r_kv, d->d_r, (const float*)cache,
+                                                             cache_row_stride, seq_start, seqlens, (const float*)w_uk,
+                                                             (const float*)w_uv, (float*)k_c, (float*)v, (float*)k_r);
+    return launch_status();
+}
+
 static gqla_status check_decode_common(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, int32_t S,
                                        const int64_t* seq_start, const int32_t* seqlens, const float* o_part,
                                        const float* lse_part) {

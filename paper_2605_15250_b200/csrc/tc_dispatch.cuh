@@ -6,6 +6,7 @@
 #include "common.cuh"
 #include "tc_decode_absorb.cuh"
 #include "tc_decode_gqa.cuh"
+#include "tc_append.cuh"
 #include "tc_combine_up.cuh"
 #include "tc_expand.cuh"
 #include "tc_gemm.cuh"
@@ -200,6 +201,45 @@ inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, i
     cudaError_t e =
         tc::gemm_launch<tc::kGemmUpProj, 128, true>(p, tmA, tmB, tmB, dim3((unsigned)m_tiles, (unsigned)d.g, 1), st);
     return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
+}
+
+// Expansion of the step's new rows; covers bf16, d_h = 128, r_kv a multiple of 128 up to 512, d_r a multiple of 8.
+inline gqla_status tc_append_expand(const gqla_dims& d, gqla_dtype dtype, int32_t B, int32_t s_q, const void* cache,
+                                    int64_t cache_row_stride, const int64_t* seq_start, const int32_t* seqlens,
+                                    const void* w_uk, const void* w_uv, void* k_c, void* v, void* k_r, cudaStream_t st) {
+    if (dtype != GQLA_BF16 || d.d_h != 128 || d.r_kv % tc::AppendSmem::kChunkK != 0 ||
+        d.r_kv > tc::AppendSmem::kMaxChunks * tc::AppendSmem::kChunkK || d.d_r % 8 != 0 || d.d_r > 256 ||
+        !stride_ok(cache_row_stride) || 2 * d.g > 65535)
+        return GQLA_ERR_UNSUPPORTED;
+    const int64_t m_tiles = ((int64_t)B * s_q + tc::AppendSmem::kRows - 1) / tc::AppendSmem::kRows;
+    if (m_tiles > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
+    CUtensorMap tmK, tmV;
+    {
+        // W[j] as an MN-major B operand: rows = (j, r) (contraction), columns = d (output)
+        const uint64_t dims[2] = {(uint64_t)d.d_h, (uint64_t)d.g * d.r_kv};
+        const uint64_t str[1] = {(uint64_t)d.d_h * 2};
+        const uint32_t box[2] = {64, 64};
+        if (!tc::make_tmap_bf16(&tmK, w_uk, 2, dims, str, box)) return GQLA_ERR_CUDA;
+        if (!tc::make_tmap_bf16(&tmV, w_uv, 2, dims, str, box)) return GQLA_ERR_CUDA;
+    }
+    tc::AppendParams p{};
+    p.B = B; p.s_q = s_q; p.g = d.g; p.r_kv = d.r_kv; p.d_r = d.d_r;
+    p.cache = (const __nv_bfloat16*)cache; p.cache_stride = cache_row_stride;
+    p.seq_start = seq_start; p.seqlens = seqlens;
+    p.k_c = (__nv_bfloat16*)k_c; p.v = (__nv_bfloat16*)v; p.k_r = (__nv_bfloat16*)k_r; p.status = nullptr;
+    auto kern = tc::append_expand_tc_kernel;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AppendSmem::kTotal) != cudaSuccess)
+            return GQLA_ERR_CUDA;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    return tc::launch_pdl(kern, dim3((unsigned)m_tiles, (unsigned)(2 * d.g), 1), dim3(tc::AppendSmem::kThreads),
+                          tc::AppendSmem::kTotal, st, p, tmK, tmV) == cudaSuccess
+               ? GQLA_OK
+               : GQLA_ERR_CUDA;
 }
 
 // Fused split merge + up-projection; covers what tc_up_proj covers with d_h = 128 and r_kv % 128 == 0.

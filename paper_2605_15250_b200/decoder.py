@@ -51,6 +51,13 @@ class GqlaDecoder:
             self.k_r = torch.empty((N, self.d_r), dtype=self.dtype, device=self.device)
             B.gqla_expand_cache(self.dims, self.cache, self.w_uk, self.w_uv, self.k_c, self.v, self.k_r)
 
+    def append_expand(self, s_q: int) -> None:
+        """After a step has written s_q new latent rows per sequence (and raised seqlens): expands just
+        those rows into K_C, V (and k_R unless it aliases the latent cache)."""
+        alias = self.k_r.data_ptr() == self.cache[:, self.r_kv:].data_ptr()
+        B.gqla_append_expand(self.dims, s_q, self.cache, self.seq_start, self.seqlens, self.w_uk, self.w_uv, self.k_c,
+                             self.v, None if alias else self.k_r)
+
     # ---- absorb path ----
     def absorb_step(self, q_c: torch.Tensor, q_r: torch.Tensor, num_splits: int = 1, want_lse: bool = False,
                     fused_tail: bool = True):

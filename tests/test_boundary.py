@@ -112,6 +112,11 @@ def test_argument_errors_return_before_launch():
     assert L.gqla_expand_cache(r(d), 0, 10, p, 575, p, p, p, p, p, None) == 2  # stride < r_kv + d_r
     assert L.gqla_expand_cache(r(d), 0, 10, p, 576, p, p, None, p, p, None) == 1
     assert L.gqla_expand_cache(r(d), 0, 0, None, 576, None, None, None, None, None, None) == 0
+    assert L.gqla_append_expand(r(d), 0, 4, 0, p, 576, p, p, p, p, p, p, p, None) == 2  # s_q < 1
+    assert L.gqla_append_expand(r(d), 0, 4, 1, p, 575, p, p, p, p, p, p, p, None) == 2  # stride < r_kv + d_r
+    assert L.gqla_append_expand(r(d), 0, 4, 1, p, 576, p, None, p, p, p, p, p, None) == 1
+    assert L.gqla_append_expand(r(d), 0, 4, 1, p, 576, p, p, p, p, odd, p, p, None) == 3
+    assert L.gqla_append_expand(r(d), 0, 0, 1, None, 576, None, None, None, None, None, None, None, None) == 0
     assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 0, p, p, 576, 10, p, p, p, p, None, None) == 2  # splits < 1
     assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, p, p, 576, 10, None, p, p, p, None, None) == 1
     assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, p, p, 100, 10, p, p, p, p, None, None) == 2

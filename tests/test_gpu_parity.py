@@ -214,6 +214,87 @@ def test_shape_variants_of_the_paper(h_q, g, s_q):
     end_to_end(w, seqlens, -3, q_gain=4.0)
 
 
+@pytest.mark.parametrize("dims,dtype", [(CANON, "bf16"), (LLAMA, "bf16"),
+                                        (dict(h_q=6, g=2, d_h=20, r_kv=36, d_r=12), "f32")])
+@pytest.mark.parametrize("s_q", [1, 2, 3])
+@pytest.mark.parametrize("copy_k_r", [False, True])
+def test_append_expand_touches_only_the_new_rows(dims, dtype, s_q, copy_k_r):
+    """The expansion of Sec. 3.1 is a per-token map: after a step only the s_q rows each sequence appended
+    need expanding.  The new rows must equal the oracle's expansion of those rows, k_R bit for bit, and every
+    other row of the planes must keep the sentinel it held (also for sequences shorter than s_q)."""
+    from tests.parity_util import assert_close, dims_of
+    from oracle import gqla_oracle as O
+    w = _wl("append", 7, s_q, 140, dtype=dtype, **dims)
+    seqlens = np.array([700, 0, 1, 129, 2050, 2, 64], dtype=np.int32)
+    x = synth.make_inputs(w, seqlens=seqlens)
+    od, bd = dims_of(w)
+    dt = x["cache"].dtype
+    N = x["cache"].shape[0]
+    sentinel = 7.0
+    k_c = torch.full((N, w.g, w.d_h), sentinel, dtype=dt, device="cuda")
+    v = torch.full((N, w.g, w.d_h), sentinel, dtype=dt, device="cuda")
+    k_r = torch.full((N, w.d_r), sentinel, dtype=dt, device="cuda") if copy_k_r else None
+    B.gqla_append_expand(bd, s_q, x["cache"].cuda(), x["seq_start"].cuda(), x["seqlens"].cuda(), x["w_uk"].cuda(),
+                         x["w_uv"].cuda(), k_c, v, k_r)
+    torch.cuda.synchronize()
+    f = {k: synth.to_f64(x[k]) for k in ("cache", "w_uk", "w_uv")}
+    kc_ref, v_ref, kr_ref = O.expand_cache(od, f["cache"], f["w_uk"], f["w_uv"])
+    new = np.zeros(N, dtype=bool)
+    for b, T in enumerate(seqlens):
+        for pos in range(max(0, int(T) - s_q), int(T)):
+            new[int(x["seq_start"][b]) + pos] = True
+    assert new.sum() == sum(min(int(T), s_q) for T in seqlens)
+    kc_got, v_got = k_c.float().cpu().numpy(), v.float().cpu().numpy()
+    assert_close(kc_got[new], kc_ref[new], "append k_c")
+    assert_close(v_got[new], v_ref[new], "append v")
+    assert np.all(kc_got[~new] == sentinel) and np.all(v_got[~new] == sentinel), "rows outside the step were written"
+    if copy_k_r:
+        kr_got = k_r.float().cpu().numpy()
+        assert np.array_equal(kr_got[new], kr_ref[new]), "k_R of the new rows must be a bit-exact copy"
+        assert np.all(kr_got[~new] == sentinel)
+
+
+def test_append_expand_keeps_an_expanded_cache_current():
+    """A decode loop on the GQA path: expand once, then per step append s_q latent rows per sequence and
+    expand only those.  Attention over the incrementally kept planes must agree with the oracle's GQA path
+    on the grown cache."""
+    from tests.parity_util import assert_close, dims_of
+    from oracle import gqla_oracle as O
+    from paper_2605_15250_b200.decoder import GqlaDecoder
+    s_q = 2
+    w = _wl("loop", 3, s_q, 141, **CANON)
+    final = np.array([260, 131, 7], dtype=np.int32)
+    x = synth.make_inputs(w, seqlens=final, q_gain=4.0)
+    od, bd = dims_of(w)
+    dev = torch.device("cuda", 0)
+    steps = 3
+    # the cache starts steps * s_q rows short; each step reveals s_q more rows per sequence
+    start = np.maximum(final - steps * s_q, 0).astype(np.int32)
+    dec = GqlaDecoder(w.h_q, w.g, w.d_h, w.r_kv, w.d_r, x["w_uk"].to(dev), x["w_uv"].to(dev), x["cache"].to(dev),
+                      x["seq_start"].to(dev), torch.from_numpy(start).to(dev), w.scale)
+    dec.expand_cache()
+    # rows beyond the start lengths are wiped, so that stale values cannot pass for appended ones
+    keep = np.zeros(x["cache"].shape[0], dtype=bool)
+    for b, T in enumerate(start):
+        keep[int(x["seq_start"][b]):int(x["seq_start"][b]) + int(T)] = True
+    wipe = torch.from_numpy(~keep).to(dev)
+    dec.k_c[wipe] = 0
+    dec.v[wipe] = 0
+    cur = start.copy()
+    for _ in range(steps):
+        cur = np.minimum(cur + s_q, final).astype(np.int32)
+        dec.seqlens.copy_(torch.from_numpy(cur))
+        dec.append_expand(s_q)
+    q = torch.cat([x["q_c"], x["q_r"]], -1).contiguous().to(dev)
+    o = dec.gqa_step(q, 2)
+    torch.cuda.synchronize()
+    dec.check_status()
+    f = {k: synth.to_f64(x[k]) for k in ("q_c", "q_r", "cache", "w_uk", "w_uv")}
+    o_ref = O.gqa_path(od, f["q_c"], f["q_r"], f["w_uk"], f["w_uv"], f["cache"], x["seq_start"].numpy(), final, s_q,
+                       w.scale)
+    assert_close(o.float().cpu().numpy(), o_ref, "gqa path after incremental expansion")
+
+
 @pytest.mark.parametrize("s_q", [3, 4, 5, 8])
 def test_speculative_query_counts(s_q):
     """s_q >= 3 (speculative decoding, Sec. 4.2): both paths stay on the tensor-core kernels (the absorb
