@@ -214,6 +214,23 @@ def test_shape_variants_of_the_paper(h_q, g, s_q):
     end_to_end(w, seqlens, -3, q_gain=4.0)
 
 
+@pytest.mark.parametrize("hpg,g,s_q", [(1, 8, 1), (1, 4, 8), (3, 2, 1), (3, 4, 5), (5, 4, 3), (6, 2, 2), (7, 4, 4), (9, 1, 6),
+                                       (12, 2, 7), (24, 4, 2), (32, 2, 3), (64, 1, 2), (128, 1, 1)])
+def test_heads_per_group_and_query_counts_off_the_powers_of_two(hpg, g, s_q):
+    """Heads per group and query positions are padded to powers of two inside the tensor-core kernels
+    (padding rows read zeros or a neighbour's queries and are dropped at the store).  Every combination
+    here has padding on one or both axes, or sits at an edge (one head per group, 128 rows per group);
+    both paths, fixed and balanced plans, against the oracle."""
+    from tests.parity_util import end_to_end
+    dims = B.make_dims(hpg * g, g, 128, 512, 64)
+    for path in ("absorb", "gqa", "projections"):
+        assert B.kernel_for(dims, torch.bfloat16, s_q, path) == "tcgen05", path
+    w = _wl("pad", 4, s_q, 150 + hpg + s_q, h_q=hpg * g, g=g, d_h=128, r_kv=512, d_r=64)
+    seqlens = np.array([300, max(s_q - 1, 0), 129, 517], dtype=np.int32)
+    end_to_end(w, seqlens, 2, q_gain=4.0)
+    end_to_end(w, seqlens, -3, q_gain=4.0)
+
+
 @pytest.mark.parametrize("dims,dtype", [(CANON, "bf16"), (LLAMA, "bf16"),
                                         (dict(h_q=6, g=2, d_h=20, r_kv=36, d_r=12), "f32")])
 @pytest.mark.parametrize("s_q", [1, 2, 3])
