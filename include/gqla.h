@@ -161,6 +161,27 @@ gqla_status gqla_decode_gqa_noalloc(const gqla_dims* dims, gqla_dtype dtype, int
                                     const int64_t* seq_start, const int32_t* seqlens, void* out, float* lse,
                                     int32_t* status_word, void* stream);
 
+/* The two decode calls over a PAGED cache (paging is not in the paper, which names KV paging among the effects
+ * its model omits, Sec. 5.1 "Limitations"; it changes where a row is fetched from and nothing else).  The cache
+ * (or, on the GQA path, each of k_c, v, k_r) is cut into pages of page_size rows; row t of sequence b is row
+ *   block_table[b * max_pages + t / page_size] * page_size + t % page_size
+ * with block_table an int32 [B, max_pages] device array whose entries below ceil(seqlens[b] / page_size)
+ * must name pages inside the cache (page * page_size + page_size <= cache_rows / n_rows); later entries
+ * are never read.  Everything else is as for gqla_decode_absorb / gqla_decode_gqa, and the outputs are
+ * the same as for the packed cache holding the same rows.  The tensor-core kernels take page sizes that
+ * are multiples of 128 rows with num_splits == 1 or the balanced plan (num_splits <= -2); other
+ * combinations run on the generic kernels. */
+gqla_status gqla_decode_absorb_paged(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                                     int32_t num_splits, const void* q_hat, const void* cache,
+                                     int64_t cache_row_stride, int64_t cache_rows, const int32_t* block_table,
+                                     int32_t max_pages, int32_t page_size, const int32_t* seqlens, float* o_part,
+                                     float* lse_part, int32_t* status_word, void* stream);
+gqla_status gqla_decode_gqa_paged(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                                  int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
+                                  int64_t k_r_row_stride, int64_t n_rows, const int32_t* block_table,
+                                  int32_t max_pages, int32_t page_size, const int32_t* seqlens, float* o_part,
+                                  float* lse_part, int32_t* status_word, void* stream);
+
 /* Log-sum-exp merge of split partials (split-KV is not in the paper; it is the flash-decoding
  * reduction of the same softmax):  M = max_k lse_k, w_k = exp(lse_k - M),
  *   out = sum_k w_k o_k / sum_k w_k,   lse = M + ln sum_k w_k;  all splits empty -> out = 0, lse = -inf.

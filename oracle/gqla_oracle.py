@@ -280,6 +280,21 @@ def decode_gqa_partials(dims: Dims, q, k_c, v, k_r, seq_start, seqlens, s_q, sca
     return _decode(dims, q_rows_of, K_of, V_of, dims.d_h, B, s_q, seq_start, seqlens, scale, num_splits, plans)
 
 
+def unpage(paged: np.ndarray, block_table: np.ndarray, page_size: int, seqlens: np.ndarray):
+    """Paged cache -> packed cache (paging is storage only; the paper's model leaves it out, Sec. 5.1).
+
+    Row t of sequence b lives in row block_table[b, t // page_size] * page_size + t % page_size of
+    `paged` [n_pages * page_size, ...].  Returns (packed rows of all sequences in order, seq_start), so
+    that every function above applies unchanged."""
+    rows, seq_start, n = [], np.zeros(len(seqlens), dtype=np.int64), 0
+    for b, T in enumerate(seqlens):
+        seq_start[b] = n
+        for t in range(int(T)):
+            rows.append(int(block_table[b, t // page_size]) * page_size + t % page_size)
+        n += int(T)
+    return paged[np.array(rows, dtype=np.int64)], seq_start
+
+
 def combine_splits(o_part: np.ndarray, lse_part: np.ndarray):
     """Log-sum-exp merge of per-split partials (split axis = 1).
 

@@ -37,6 +37,12 @@ _PROTOTYPES = {
     "gqla_absorb_q": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_decode_absorb": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
                                      c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_decode_absorb_paged": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
+                                           c_int64, c_int64, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
+                                           c_void_p, c_void_p]),
+    "gqla_decode_gqa_paged": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
+                                        c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_int32, c_int32, c_void_p,
+                                        c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_append_expand": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_int64, c_void_p, c_void_p, c_void_p,
                                      c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_expand_cache": (c_int32, [c_void_p, c_int32, c_int64, c_void_p, c_int64, c_void_p, c_void_p, c_void_p,
@@ -162,6 +168,37 @@ def gqla_expand_cache(dims: GqlaDims, cache: torch.Tensor, w_uk: torch.Tensor, w
     _check(lib().gqla_expand_cache(ctypes.byref(dims), _dtype_code(cache), cache.shape[0], _ptr(cache),
                                    cache.stride(0), _ptr(w_uk), _ptr(w_uv), _ptr(k_c), _ptr(v), _ptr(k_r),
                                    _stream()), "gqla_expand_cache")
+
+
+def gqla_decode_absorb_paged(dims: GqlaDims, q_hat: torch.Tensor, cache: torch.Tensor, block_table: torch.Tensor,
+                             page_size: int, seqlens: torch.Tensor, scale: float, num_splits: int, o_part: torch.Tensor,
+                             lse_part: torch.Tensor, status_word: torch.Tensor | None = None) -> None:
+    """gqla_decode_absorb over a paged cache: block_table int32 [B, max_pages] of page numbers."""
+    _contig(q_hat, block_table, seqlens, o_part, lse_part)
+    assert cache.dim() == 2 and cache.stride(1) == 1
+    assert block_table.dtype == torch.int32 and block_table.dim() == 2 and seqlens.dtype == torch.int32
+    assert o_part.dtype == torch.float32 and lse_part.dtype == torch.float32
+    B, s_q = q_hat.shape[0], q_hat.shape[1]
+    _check(lib().gqla_decode_absorb_paged(ctypes.byref(dims), _dtype_code(q_hat), B, s_q, scale, num_splits, _ptr(q_hat),
+                                          _ptr(cache), cache.stride(0), cache.shape[0], _ptr(block_table),
+                                          block_table.shape[1], page_size, _ptr(seqlens), _ptr(o_part), _ptr(lse_part),
+                                          _ptr(status_word), _stream()), "gqla_decode_absorb_paged")
+
+
+def gqla_decode_gqa_paged(dims: GqlaDims, q: torch.Tensor, k_c: torch.Tensor, v: torch.Tensor, k_r: torch.Tensor,
+                          block_table: torch.Tensor, page_size: int, seqlens: torch.Tensor, scale: float,
+                          num_splits: int, o_part: torch.Tensor, lse_part: torch.Tensor,
+                          status_word: torch.Tensor | None = None) -> None:
+    """gqla_decode_gqa over paged K_C, V, k_R planes: block_table int32 [B, max_pages] of page numbers."""
+    _contig(q, k_c, v, block_table, seqlens, o_part, lse_part)
+    assert k_r.dim() == 2 and k_r.stride(1) == 1
+    assert block_table.dtype == torch.int32 and block_table.dim() == 2 and seqlens.dtype == torch.int32
+    assert o_part.dtype == torch.float32 and lse_part.dtype == torch.float32
+    B, s_q = q.shape[0], q.shape[1]
+    _check(lib().gqla_decode_gqa_paged(ctypes.byref(dims), _dtype_code(q), B, s_q, scale, num_splits, _ptr(q), _ptr(k_c),
+                                       _ptr(v), _ptr(k_r), k_r.stride(0), k_c.shape[0], _ptr(block_table),
+                                       block_table.shape[1], page_size, _ptr(seqlens), _ptr(o_part), _ptr(lse_part),
+                                       _ptr(status_word), _stream()), "gqla_decode_gqa_paged")
 
 
 def gqla_append_expand(dims: GqlaDims, s_q: int, cache: torch.Tensor, seq_start: torch.Tensor, seqlens: torch.Tensor,

@@ -23,6 +23,20 @@ __host__ __device__ inline int32_t visible_limit(int32_t T, int32_t s_q, int32_t
     return lim > 0 ? lim : 0;
 }
 
+// Where the cache rows of a sequence live.  Packed: row t of sequence b is seq_start[b] + t.  Paged: the
+// cache is cut into pages of page_size rows and block_table[b * max_pages + t / page_size] names the page of
+// row t (paging is not in the paper; it only changes where a row is fetched from).
+struct RowMap {
+    const int64_t* seq_start;    // packed layout (null when paged)
+    const int32_t* block_table;  // paged layout (null when packed)
+    int32_t max_pages, page_size;
+    __host__ __device__ bool paged() const { return block_table != nullptr; }
+    __device__ __forceinline__ int64_t row(int32_t b, int32_t t) const {
+        if (block_table == nullptr) return seq_start[b] + t;
+        return (int64_t)block_table[(int64_t)b * max_pages + t / page_size] * page_size + t % page_size;
+    }
+};
+
 __device__ __forceinline__ float ldf(const float* p) { return *p; }
 __device__ __forceinline__ float ldf(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 __device__ __forceinline__ void stf(float* p, float v) { *p = v; }

@@ -14,7 +14,7 @@ struct DecodeArgs {
     const void* v;       // values; row stride v_stride, + group * v_gstride
     int64_t kA_stride, kA_gstride, kB_stride, v_stride, v_gstride;
     int32_t dA, dB, dv;
-    const int64_t* seq_start;
+    RowMap rows;
     const int32_t* seqlens;
     int32_t B, S, s_q, h_q, hpg;
     float scale;
@@ -45,7 +45,6 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a) {
     if (end > lim) end = lim;
 
     const E* q = (const E*)a.q + ((int64_t)(b * a.s_q + p) * a.h_q + i) * (a.dA + a.dB);
-    const int64_t r0 = a.seq_start[b];
     const E* kA = (const E*)a.kA + (int64_t)j * a.kA_gstride;
     const E* kB = (const E*)a.kB;
     const E* vv = (const E*)a.v + (int64_t)j * a.v_gstride;
@@ -56,11 +55,12 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a) {
     float m = -INFINITY, l = 0.f;
 
     for (int32_t s = begin; s < end; ++s) {
-        const E* ka = kA + (r0 + s) * a.kA_stride;
+        const int64_t n = a.rows.row(b, s);
+        const E* ka = kA + n * a.kA_stride;
         float dot = 0.f;
         for (int d = lane; d < a.dA; d += 32) dot = fmaf(ldf(q + d), ldf(ka + d), dot);
         if (a.dB > 0) {
-            const E* kb = kB + (r0 + s) * a.kB_stride;
+            const E* kb = kB + n * a.kB_stride;
             for (int d = lane; d < a.dB; d += 32) dot = fmaf(ldf(q + a.dA + d), ldf(kb + d), dot);
         }
         const float x = warp_sum(dot) * a.scale;
@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a) {
         const float corr = expf(m - m_new);  // exp(-inf) = 0 on the first row
         const float e = expf(x - m_new);
         l = l * corr + e;
-        const E* vr = vv + (r0 + s) * a.v_stride;
+        const E* vr = vv + n * a.v_stride;
 #pragma unroll
         for (int c = 0; c < kGenericMaxV; ++c) {
             const int d = lane + 32 * c;

@@ -287,23 +287,31 @@ gqla_status gqla_append_expand(const gqla_dims* d, gqla_dtype dtype, int32_t B, 
 }
 
 static gqla_status check_decode_common(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, int32_t S,
-                                       const int64_t* seq_start, const int32_t* seqlens, const float* o_part,
+                                       const RowMap& rows, const int32_t* seqlens, const float* o_part,
                                        const float* lse_part) {
     gqla_status s;
     if ((s = check_dims(d)) != GQLA_OK) return s;
     if ((s = check_dtype(dtype)) != GQLA_OK) return s;
     if (B < 0 || s_q < 1 || S == 0 || S == -1) return GQLA_ERR_SHAPE;  // S <= -2: balanced plan, -S slots
+    if (rows.block_table != nullptr && (rows.page_size < 1 || rows.max_pages < 1)) return GQLA_ERR_SHAPE;
     if (B == 0) return GQLA_OK;
-    if (seq_start == nullptr || seqlens == nullptr || o_part == nullptr || lse_part == nullptr) return GQLA_ERR_NULL;
+    if ((rows.seq_start == nullptr && rows.block_table == nullptr) || seqlens == nullptr || o_part == nullptr ||
+        lse_part == nullptr)
+        return GQLA_ERR_NULL;
     if (!aligned16(o_part)) return GQLA_ERR_ALIGN;
     return GQLA_OK;
 }
 
-gqla_status gqla_decode_absorb(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
-                               int32_t num_splits, const void* q_hat, const void* cache, int64_t cache_row_stride,
-                               int64_t cache_rows, const int64_t* seq_start, const int32_t* seqlens, float* o_part,
-                               float* lse_part, int32_t* status_word, void* stream) {
-    gqla_status s = check_decode_common(d, dtype, B, s_q, num_splits, seq_start, seqlens, o_part, lse_part);
+static RowMap packed_rows(const int64_t* seq_start) { return RowMap{seq_start, nullptr, 0, 0}; }
+static RowMap paged_rows(const int32_t* block_table, int32_t max_pages, int32_t page_size) {
+    return RowMap{nullptr, block_table, max_pages, page_size};
+}
+
+static gqla_status decode_absorb_any(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                                     int32_t num_splits, const void* q_hat, const void* cache, int64_t cache_row_stride,
+                                     int64_t cache_rows, const RowMap& rows, const int32_t* seqlens, float* o_part,
+                                     float* lse_part, int32_t* status_word, void* stream) {
+    gqla_status s = check_decode_common(d, dtype, B, s_q, num_splits, rows, seqlens, o_part, lse_part);
     if (s != GQLA_OK) return s;
     if (B == 0) return GQLA_OK;
     if (q_hat == nullptr || cache == nullptr) return GQLA_ERR_NULL;
@@ -311,7 +319,7 @@ gqla_status gqla_decode_absorb(const gqla_dims* d, gqla_dtype dtype, int32_t B, 
     if (cache_row_stride < d->r_kv + d->d_r || cache_rows < 0) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, 0)) {
-        s = tc_decode_absorb(*d, B, s_q, scale, num_splits, q_hat, cache, cache_row_stride, cache_rows, seq_start, seqlens,
+        s = tc_decode_absorb(*d, B, s_q, scale, num_splits, q_hat, cache, cache_row_stride, cache_rows, rows, seqlens,
                              o_part, lse_part, status_word, st);
         if (s != GQLA_ERR_UNSUPPORTED) return s;
     }
@@ -320,7 +328,51 @@ gqla_status gqla_decode_absorb(const gqla_dims* d, gqla_dtype dtype, int32_t B, 
     a.kA = cache; a.kA_stride = cache_row_stride; a.kA_gstride = 0; a.dA = d->r_kv + d->d_r;
     a.kB = nullptr; a.kB_stride = 0; a.dB = 0;
     a.v = cache; a.v_stride = cache_row_stride; a.v_gstride = 0; a.dv = d->r_kv;
-    a.seq_start = seq_start; a.seqlens = seqlens;
+    a.rows = rows; a.seqlens = seqlens;
+    a.B = B; a.S = num_splits < 0 ? -num_splits : num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
+    a.scale = scale; a.o_part = o_part; a.lse_part = lse_part;
+    return launch_decode_generic(dtype, a, st);
+}
+
+gqla_status gqla_decode_absorb(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                               int32_t num_splits, const void* q_hat, const void* cache, int64_t cache_row_stride,
+                               int64_t cache_rows, const int64_t* seq_start, const int32_t* seqlens, float* o_part,
+                               float* lse_part, int32_t* status_word, void* stream) {
+    return decode_absorb_any(d, dtype, B, s_q, scale, num_splits, q_hat, cache, cache_row_stride, cache_rows,
+                             packed_rows(seq_start), seqlens, o_part, lse_part, status_word, stream);
+}
+
+gqla_status gqla_decode_absorb_paged(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                                     int32_t num_splits, const void* q_hat, const void* cache, int64_t cache_row_stride,
+                                     int64_t cache_rows, const int32_t* block_table, int32_t max_pages,
+                                     int32_t page_size, const int32_t* seqlens, float* o_part, float* lse_part,
+                                     int32_t* status_word, void* stream) {
+    return decode_absorb_any(d, dtype, B, s_q, scale, num_splits, q_hat, cache, cache_row_stride, cache_rows,
+                             paged_rows(block_table, max_pages, page_size), seqlens, o_part, lse_part, status_word, stream);
+}
+
+static gqla_status decode_gqa_any(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                                  int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
+                                  int64_t k_r_row_stride, int64_t n_rows, const RowMap& rows, const int32_t* seqlens,
+                                  float* o_part, float* lse_part, int32_t* status_word, void* stream) {
+    gqla_status s = check_decode_common(d, dtype, B, s_q, num_splits, rows, seqlens, o_part, lse_part);
+    if (s != GQLA_OK) return s;
+    if (B == 0) return GQLA_OK;
+    if (q == nullptr || k_c == nullptr || v == nullptr || (d->d_r > 0 && k_r == nullptr)) return GQLA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k_c) || !aligned16(v) || !aligned16(k_r)) return GQLA_ERR_ALIGN;
+    if ((d->d_r > 0 && k_r_row_stride < d->d_r) || n_rows < 0) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, 1)) {
+        s = tc_decode_gqa(*d, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, n_rows, rows, seqlens, o_part,
+                          lse_part, status_word, st);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
+    DecodeArgs a{};
+    a.q = q;
+    a.kA = k_c; a.kA_stride = (int64_t)d->g * d->d_h; a.kA_gstride = d->d_h; a.dA = d->d_h;
+    a.kB = k_r; a.kB_stride = k_r_row_stride; a.dB = d->d_r;
+    a.v = v; a.v_stride = (int64_t)d->g * d->d_h; a.v_gstride = d->d_h; a.dv = d->d_h;
+    a.rows = rows; a.seqlens = seqlens;
     a.B = B; a.S = num_splits < 0 ? -num_splits : num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
     a.scale = scale; a.o_part = o_part; a.lse_part = lse_part;
     return launch_decode_generic(dtype, a, st);
@@ -330,27 +382,17 @@ gqla_status gqla_decode_gqa(const gqla_dims* d, gqla_dtype dtype, int32_t B, int
                             int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
                             int64_t k_r_row_stride, int64_t n_rows, const int64_t* seq_start, const int32_t* seqlens,
                             float* o_part, float* lse_part, int32_t* status_word, void* stream) {
-    gqla_status s = check_decode_common(d, dtype, B, s_q, num_splits, seq_start, seqlens, o_part, lse_part);
-    if (s != GQLA_OK) return s;
-    if (B == 0) return GQLA_OK;
-    if (q == nullptr || k_c == nullptr || v == nullptr || (d->d_r > 0 && k_r == nullptr)) return GQLA_ERR_NULL;
-    if (!aligned16(q) || !aligned16(k_c) || !aligned16(v) || !aligned16(k_r)) return GQLA_ERR_ALIGN;
-    if ((d->d_r > 0 && k_r_row_stride < d->d_r) || n_rows < 0) return GQLA_ERR_SHAPE;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, 1)) {
-        s = tc_decode_gqa(*d, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, n_rows, seq_start, seqlens, o_part,
-                          lse_part, status_word, st);
-        if (s != GQLA_ERR_UNSUPPORTED) return s;
-    }
-    DecodeArgs a{};
-    a.q = q;
-    a.kA = k_c; a.kA_stride = (int64_t)d->g * d->d_h; a.kA_gstride = d->d_h; a.dA = d->d_h;
-    a.kB = k_r; a.kB_stride = k_r_row_stride; a.dB = d->d_r;
-    a.v = v; a.v_stride = (int64_t)d->g * d->d_h; a.v_gstride = d->d_h; a.dv = d->d_h;
-    a.seq_start = seq_start; a.seqlens = seqlens;
-    a.B = B; a.S = num_splits < 0 ? -num_splits : num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
-    a.scale = scale; a.o_part = o_part; a.lse_part = lse_part;
-    return launch_decode_generic(dtype, a, st);
+    return decode_gqa_any(d, dtype, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, n_rows,
+                          packed_rows(seq_start), seqlens, o_part, lse_part, status_word, stream);
+}
+
+gqla_status gqla_decode_gqa_paged(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                                  int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
+                                  int64_t k_r_row_stride, int64_t n_rows, const int32_t* block_table, int32_t max_pages,
+                                  int32_t page_size, const int32_t* seqlens, float* o_part, float* lse_part,
+                                  int32_t* status_word, void* stream) {
+    return decode_gqa_any(d, dtype, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, n_rows,
+                          paged_rows(block_table, max_pages, page_size), seqlens, o_part, lse_part, status_word, stream);
 }
 
 gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_splits, int32_t d_out,

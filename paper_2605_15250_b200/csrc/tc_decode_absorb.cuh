@@ -39,7 +39,7 @@ struct AbsorbParams {
     int32_t B, S, s_q, h_q, rows_total /* s_q*h_q */, row_blocks /* ceil(rows_total/128) */;
     int32_t balanced, W;  // balanced plan: W pairs per row block, grid = 2 * W * row_blocks
     float scale_log2;
-    const int64_t* seq_start;
+    RowMap rows;      // packed or paged (pages a multiple of 128 rows, pieces starting on tile boundaries)
     const int32_t* seqlens;
     float* o_part;    // [B, S, s_q*h_q, 512]
     float* lse_part;  // [B, S, s_q*h_q]
@@ -170,10 +170,13 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
                 if (cta == 0) mbar_expect_tx(q_full, 2 * L::kQBytes);
                 for (int kb = 0; kb < 9; ++kb)
                     tma_load_2d_pair(tiles + kb * L::kBox, &tmQ, kb * 64, pc.b * p.rows_total + rho0, q_full_l);
-                const int64_t row0 = p.seq_start[pc.b] + pc.tok_begin;
-                // K groups in the order (tile, column third)
+                // K groups in the order (tile, column third); a tile never straddles a page
+                int64_t tile_row = p.rows.row(pc.b, pc.tok_begin);
                 for (int kt = 0; kt < pc.n_tiles && ok; ++kt) {
-                    const int32_t row = (int32_t)(row0 + (int64_t)kt * 128 + cta * 64);
+                    const int32_t row = (int32_t)(tile_row + cta * 64);
+                    // the next tile's row is fetched while this tile's slots are waited for
+                    if (kt + 1 < pc.n_tiles)
+                        tile_row = p.rows.paged() ? p.rows.row(pc.b, pc.tok_begin + (kt + 1) * 128) : tile_row + 128;
 #pragma unroll 1
                     for (int kg = 0; kg < 3; ++kg) {
                         if (!(ok = mbar_wait(&kempty[ks], kph, ab, 1))) break;
@@ -202,13 +205,16 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
                 if (pc.n_tiles == 0) continue;
                 // the V ring doubles as the output staging of the previous piece
                 if (pi > 0 && !(ok = mbar_wait(epi_done, (pi - 1) & 1, ab, 16))) break;
-                const int64_t row0 = p.seq_start[pc.b] + pc.tok_begin;
+                int64_t tile_row = p.rows.row(pc.b, pc.tok_begin);
                 for (int vt = 0; vt < pc.n_tiles && ok; ++vt) {
+                    const int64_t row0 = tile_row;
+                    if (vt + 1 < pc.n_tiles)
+                        tile_row = p.rows.paged() ? p.rows.row(pc.b, pc.tok_begin + (vt + 1) * 128) : tile_row + 128;
 #pragma unroll 1
                     for (int vh = 0; vh < 2; ++vh) {
                         if (!(ok = mbar_wait(&vempty[vs], vph, ab, 2))) break;
                         if (cta == 0) mbar_expect_tx(&vfull[vs], 2 * L::kVGroup);
-                        const int32_t row = (int32_t)(row0 + (int64_t)vt * 128 + vh * 64);
+                        const int32_t row = (int32_t)(row0 + vh * 64);
                         const uint32_t bar = mapa(smem_u32(&vfull[vs]), 0);
                         uint8_t* dst = tiles + L::kOffV + vs * L::kVGroup;
                         // box (m, i): latent columns [256m + 128cta + 64i, +64) -- this CTA's half of MMA m's N

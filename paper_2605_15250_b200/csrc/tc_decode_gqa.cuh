@@ -30,7 +30,7 @@ struct GqaParams {
     int32_t B, S, s_q, h_q, g, hpg, hpg_box;
     int32_t balanced, W;  // balanced plan: W workers per group, grid = W * g
     float scale_log2;
-    const int64_t* seq_start;
+    RowMap rows;  // packed or paged (pages a multiple of 128 rows, pieces starting on tile boundaries)
     const int32_t* seqlens;
     float* o_part;    // [B, S, s_q, h_q, 128]
     float* lse_part;  // [B, S, s_q, h_q]
@@ -155,12 +155,15 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
                             "l"(reinterpret_cast<uint64_t>(&tmQ)), "r"(smem_u32(q_full)), "r"(kb * 64), "r"(0), "r"(j),
                             "r"(pc.b * p.s_q)
                             : "memory");
-                const int64_t row0 = p.seq_start[pc.b] + pc.tok_begin;
+                int64_t tile_row = p.rows.row(pc.b, pc.tok_begin);
                 for (int t = 0; t < pc.n_tiles; ++t, ++gt) {
                     const int s = gt & 1;
                     const uint32_t ph = (gt >> 1) & 1;
                     uint8_t* st = stage0 + s * L::kStageBytes;
-                    const int32_t row = (int32_t)(row0 + (int64_t)t * 128);
+                    const int32_t row = (int32_t)tile_row;
+                    // the next tile's row is fetched while this tile's slots are waited for; a tile never straddles a page
+                    if (t + 1 < pc.n_tiles)
+                        tile_row = p.rows.paged() ? p.rows.row(pc.b, pc.tok_begin + (t + 1) * 128) : tile_row + 128;
                     if (!(ok = mbar_wait(&kempty[s], ph ^ 1, ab, 1))) break;
                     mbar_expect_tx(&kfull[s], L::kKcBytes + L::kKrBytes);
                     tma_load_3d(st, &tmK, 0, j, row, &kfull[s]);

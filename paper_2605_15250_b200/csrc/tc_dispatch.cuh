@@ -280,17 +280,20 @@ inline gqla_status tc_combine_up_proj(const gqla_dims& d, gqla_dtype dtype, int3
 
 inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S,
                                     const void* q_hat, const void* cache, int64_t cache_row_stride,
-                                    int64_t cache_rows, const int64_t* seq_start, const int32_t* seqlens,
+                                    int64_t cache_rows, const RowMap& rows, const int32_t* seqlens,
                                     float* o_part, float* lse_part, int32_t* status, cudaStream_t st) {
     if (!tc_covers(d, GQLA_BF16, s_q, 0) || !stride_ok(cache_row_stride) || cache_rows > 0x7fffffffLL ||
         cache_rows < 1)
         return GQLA_ERR_UNSUPPORTED;
+    if (rows.paged() && rows.page_size % kTileRows != 0) return GQLA_ERR_UNSUPPORTED;  // a tile must not straddle pages
     const int rows_total = s_q * d.h_q;
     const int row_blocks = (rows_total + 127) / 128;
     // S < 0: balanced plan with -S slots per sequence, W persistent pairs per row block
     const int32_t workers = S < 0 ? tc_balanced_workers(d, s_q, 0) : 0;
     const bool balanced = S < 0 && workers > 0;
     if (S < 0) S = -S;
+    // paged: pieces must start on tile boundaries, which the fixed plan's 64-row granule does not give for S > 1
+    if (rows.paged() && !balanced && S != 1) return GQLA_ERR_UNSUPPORTED;
     const int64_t pairs = balanced ? (int64_t)workers * row_blocks : (int64_t)B * S * row_blocks;
     if (2 * pairs > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     CUtensorMap tmQ, tmC;
@@ -310,7 +313,7 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
     p.B = B; p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.rows_total = rows_total; p.row_blocks = row_blocks;
     p.balanced = balanced ? 1 : 0; p.W = workers;
     p.scale_log2 = scale * 1.4426950408889634f;
-    p.seq_start = seq_start; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
+    p.rows = rows; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
     auto kern = tc::decode_absorb_tc_kernel<0>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AbsorbSmem::kTotal) != cudaSuccess)
         return GQLA_ERR_CUDA;
@@ -364,14 +367,16 @@ inline cudaError_t gqa_launch(const tc::GqaParams& p, const CUtensorMap& q, cons
 
 inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S, const void* q,
                                  const void* k_c, const void* v, const void* k_r, int64_t k_r_row_stride,
-                                 int64_t n_rows, const int64_t* seq_start, const int32_t* seqlens, float* o_part,
+                                 int64_t n_rows, const RowMap& rows, const int32_t* seqlens, float* o_part,
                                  float* lse_part, int32_t* status, cudaStream_t st) {
     if (!tc_covers(d, GQLA_BF16, s_q, 1) || !stride_ok(k_r_row_stride) || n_rows > 0x7fffffffLL || n_rows < 1)
         return GQLA_ERR_UNSUPPORTED;
+    if (rows.paged() && rows.page_size % kTileRows != 0) return GQLA_ERR_UNSUPPORTED;  // a tile must not straddle pages
     // S < 0: balanced plan with -S slots per sequence, W persistent CTAs per group
     const int32_t workers = S < 0 ? tc_balanced_workers(d, s_q, 1) : 0;
     const bool balanced = S < 0 && workers > 0;
     if (S < 0) S = -S;
+    if (rows.paged() && !balanced && S != 1) return GQLA_ERR_UNSUPPORTED;  // see tc_decode_absorb
     const int64_t units = balanced ? (int64_t)workers * d.g : (int64_t)B * S * d.g;
     if (units > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     const int hpg = d.h_q / d.g;
@@ -402,7 +407,7 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
     p.B = B; p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpg_box = hpg_box;
     p.balanced = balanced ? 1 : 0; p.W = workers;
     p.scale_log2 = scale * 1.4426950408889634f;
-    p.seq_start = seq_start; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
+    p.rows = rows; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
     cudaError_t e;
     switch (R) {
         case 8: e = gqa_launch<8>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;

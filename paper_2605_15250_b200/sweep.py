@@ -40,6 +40,48 @@ def _pieces(seqlens, S: int, W: int, batch: int) -> float:
     return sum(1 for pl in plan for lo, hi in pl if hi > lo) / batch
 
 
+def time_paged(dec: GqlaDecoder, w: synth.Workload, x: dict, path: str, S: int, page_size: int, steps: int,
+               warmup: int) -> dict:
+    """The decode kernel alone over a pool of shuffled pages holding the same rows (kernel time only)."""
+    dev = dec.device
+    slots = abs(S)
+    total_tokens = int(x["seqlens"].sum())
+    cache_p, table = synth.to_paged(x["cache"], x["seq_start"], x["seqlens"].numpy(), page_size, seed=w.seed + 1)
+    cache_p, table = cache_p.to(dev), table.to(dev)
+    if path == "absorb":
+        q_hat = torch.randn((w.batch, w.s_q, w.h_q, w.d_abs), device=dev).to(torch.bfloat16)
+        o_part = torch.empty((w.batch, slots, w.s_q, w.h_q, w.r_kv), dtype=torch.float32, device=dev)
+        lse_part = torch.empty((w.batch, slots, w.s_q, w.h_q), dtype=torch.float32, device=dev)
+
+        def kernel():
+            B.gqla_decode_absorb_paged(dec.dims, q_hat, cache_p, table, page_size, dec.seqlens, dec.scale, S, o_part,
+                                       lse_part, dec.status)
+    else:
+        k_c = torch.empty((cache_p.shape[0], w.g, w.d_h), dtype=torch.bfloat16, device=dev)
+        v = torch.empty_like(k_c)
+        B.gqla_expand_cache(dec.dims, cache_p, dec.w_uk, dec.w_uv, k_c, v, None)
+        q = torch.randn((w.batch, w.s_q, w.h_q, w.d_gqa), device=dev).to(torch.bfloat16)
+        o_part = torch.empty((w.batch, slots, w.s_q, w.h_q, w.d_h), dtype=torch.float32, device=dev)
+        lse_part = torch.empty((w.batch, slots, w.s_q, w.h_q), dtype=torch.float32, device=dev)
+
+        def kernel():
+            B.gqla_decode_gqa_paged(dec.dims, q, k_c, v, cache_p[:, w.r_kv:], table, page_size, dec.seqlens, dec.scale, S,
+                                    o_part, lse_part, dec.status)
+    for _ in range(warmup):
+        kernel()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev:
+        a.record()
+        kernel()
+        b.record()
+    torch.cuda.synchronize()
+    dec.check_status()
+    k_us = statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
+    return {"workload": w.name, "path": path, "s_q": w.s_q, "batch": w.batch, "total_tokens": total_tokens,
+            "layout": f"paged, {page_size} rows per page, shuffled", "plan": "balanced" if S < 0 else "fixed",
+            "slots": slots, "kernel_us": round(k_us, 1)}
+
+
 def time_case(dec: GqlaDecoder, w: synth.Workload, x: dict, path: str, S: int, steps: int, warmup: int) -> dict:
     dev = dec.device
     total_tokens = int(x["seqlens"].sum())
@@ -139,6 +181,10 @@ def run(names, steps: int, warmup: int):
                 res = time_case(dec, w, x, path, S, steps, warmup)
                 if res:
                     print(json.dumps(res), flush=True)
+            # the same kernel over a paged pool, on the two workloads the benchmark quotes
+            if (name, path) in (("C1", "absorb"), ("C2", "gqa")):
+                print(json.dumps(time_paged(dec, w, x, path, plans[0] if name == "C1" else plans[-1], 128, steps, warmup)),
+                      flush=True)
         del dec
         torch.cuda.empty_cache()
 

@@ -130,6 +130,30 @@ def make_inputs(w: Workload, seqlens: np.ndarray | None = None, q_gain: float = 
     }
 
 
+def to_paged(t: torch.Tensor, seq_start, seqlens, page_size: int, seed: int, fill: float = 3.0, spare_pages: int = 3):
+    """Scatters packed rows [N, ...] into a paged layout: the pages of every sequence are placed at seeded
+    random positions of a pool with a few spare pages; rows no sequence owns hold `fill` (finite, so a
+    tile that reads past a sequence's end sees harmless values).  Returns (paged [n_pages * page_size, ...],
+    block_table int32 [B, max_pages]); unused table entries are -1 ... never read."""
+    seqlens = np.asarray(seqlens)
+    pages_of = [(int(T) + page_size - 1) // page_size for T in seqlens]
+    max_pages = max(1, max(pages_of) if len(pages_of) else 1)
+    n_pages = sum(pages_of) + spare_pages
+    order = _rng(seed, 99).permutation(n_pages)
+    paged = torch.full((n_pages * page_size, *t.shape[1:]), fill, dtype=t.dtype)
+    table = np.full((len(seqlens), max_pages), -1, dtype=np.int32)
+    nxt = 0
+    for b, T in enumerate(seqlens):
+        for k in range(pages_of[b]):
+            page = int(order[nxt]); nxt += 1
+            table[b, k] = page
+            lo = k * page_size
+            n = min(page_size, int(T) - lo)
+            src = int(seq_start[b]) + lo
+            paged[page * page_size:page * page_size + n] = t[src:src + n]
+    return paged, torch.from_numpy(table)
+
+
 def to_f64(t: torch.Tensor) -> np.ndarray:
     """Exact widening of a stored tensor to float64 (for the CPU checker)."""
     return t.detach().cpu().to(torch.float64).numpy()

@@ -121,6 +121,13 @@ def test_argument_errors_return_before_launch():
     assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, p, p, 576, 10, None, p, p, p, None, None) == 1
     assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, p, p, 100, 10, p, p, p, p, None, None) == 2
     assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, odd, p, 576, 10, p, p, p, p, None, None) == 3
+    assert L.gqla_decode_absorb_paged(r(d), 0, 1, 1, 0.1, 1, p, p, 576, 10, None, 4, 128, p, p, p, None, None) == 1
+    assert L.gqla_decode_absorb_paged(r(d), 0, 1, 1, 0.1, 1, p, p, 576, 10, p, 4, 0, p, p, p, None, None) == 2  # page size
+    assert L.gqla_decode_absorb_paged(r(d), 0, 1, 1, 0.1, 1, p, p, 576, 10, p, 0, 128, p, p, p, None, None) == 2
+    assert L.gqla_decode_gqa_paged(r(d), 0, 1, 1, 0.1, 1, p, p, p, p, 64, 10, None, 4, 128, p, p, p, None, None) == 1
+    assert L.gqla_decode_gqa_paged(r(d), 0, 1, 1, 0.1, -1, p, p, p, p, 64, 10, p, 4, 128, p, p, p, None, None) == 2
+    assert L.gqla_decode_gqa_paged(r(d), 0, 0, 1, 0.1, 1, None, None, None, None, 64, 0, None, 4, 128, None, None, None,
+                                   None, None) == 0
     assert L.gqla_decode_gqa(r(d), 0, 1, 1, 0.1, 1, p, p, p, p, 32, 10, p, p, p, p, None, None) == 2  # k_r stride < d_r
     assert L.gqla_decode_gqa(r(d), 0, 1, 1, 0.1, 1, p, None, p, p, 64, 10, p, p, p, p, None, None) == 1
     assert L.gqla_combine_splits(1, 128, 0, 512, 0, p, p, p, None, None) == 2

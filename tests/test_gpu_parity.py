@@ -214,6 +214,82 @@ def test_shape_variants_of_the_paper(h_q, g, s_q):
     end_to_end(w, seqlens, -3, q_gain=4.0)
 
 
+@pytest.mark.parametrize("dims", [CANON, LLAMA])
+@pytest.mark.parametrize("s_q", [1, 2])
+@pytest.mark.parametrize("page_size,S", [(128, 1), (128, -3), (256, -3), (128, 3), (16, 2), (48, -3)])
+def test_paged_cache_gives_what_the_packed_cache_gives(dims, s_q, page_size, S):
+    """Paging is storage only (the paper's model leaves it out, Sec. 5.1): both decode calls over a pool of
+    shuffled pages must return what they return over the packed cache that holds the same rows -- bit for
+    bit where both runs use the same kernel and the same pieces (tensor-core kernels: pages of a multiple
+    of 128 rows with one split or the balanced plan; generic kernels: any page size) -- and match the oracle
+    fed with the rows gathered back."""
+    from tests.parity_util import assert_close, dims_of, round_to
+    from oracle import gqla_oracle as O
+    w = _wl("paged", 5, s_q, 160, **dims)
+    seqlens = np.array([700, 0, 129, 2050, 1], dtype=np.int32)
+    x = synth.make_inputs(w, seqlens=seqlens, q_gain=4.0)
+    od, bd = dims_of(w)
+    slots = abs(S)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sl = x["seqlens"].cuda()
+    cache_p, table = synth.to_paged(x["cache"], x["seq_start"], seqlens, page_size, seed=161)
+    table_d = table.cuda()
+    f = {k: synth.to_f64(x[k]) for k in ("q_c", "q_r", "cache", "w_uk", "w_uv")}
+    # the oracle reads the pool through its own gather
+    rows, ss = O.unpage(synth.to_f64(cache_p), table.numpy(), page_size, seqlens)
+    assert np.array_equal(rows, f["cache"])
+
+    # ---- absorb path
+    qh_in = round_to(w, O.absorb_q(od, f["q_c"], f["q_r"], f["w_uk"])).cuda()
+
+    def parts(D):
+        return (torch.full((w.batch, slots, s_q, w.h_q, D), float("nan"), dtype=torch.float32, device="cuda"),
+                torch.full((w.batch, slots, s_q, w.h_q), float("nan"), dtype=torch.float32, device="cuda"))
+
+    o_a, l_a = parts(w.r_kv)
+    B.gqla_decode_absorb(bd, qh_in, x["cache"].cuda(), x["seq_start"].cuda(), sl, w.scale, S, o_a, l_a, status)
+    o_b, l_b = parts(w.r_kv)
+    B.gqla_decode_absorb_paged(bd, qh_in, cache_p.cuda(), table_d, page_size, sl, w.scale, S, o_b, l_b, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    same_kernel = page_size % 128 == 0 and (S == 1 or S < 0)  # else the paged call runs on the generic kernel
+    live = ~torch.isneginf(l_a)  # partial outputs of empty slots are not written under the balanced plan
+    if same_kernel:  # same pieces too; otherwise only the merged result is comparable (below)
+        assert torch.equal(l_a, l_b) and torch.equal(o_a[live], o_b[live])
+    oh = torch.empty((w.batch, s_q, w.h_q, w.r_kv), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((w.batch, s_q, w.h_q), dtype=torch.float32, device="cuda")
+    B.gqla_combine_splits(o_b, l_b, oh, lse)
+    oh_ref, lse_ref = O.decode_absorb(od, synth.to_f64(qh_in), rows, ss, seqlens, s_q, w.scale)
+    assert_close(oh.float().cpu().numpy(), oh_ref, "paged absorb o_hat")
+    assert_close(lse.cpu().numpy(), lse_ref, "paged absorb lse")
+
+    # ---- GQA path: the expansion is per row, so the pool is expanded as it is
+    N_p = cache_p.shape[0]
+    kc_p = torch.empty((N_p, w.g, w.d_h), dtype=torch.bfloat16, device="cuda")
+    v_p = torch.empty_like(kc_p)
+    cache_pd = cache_p.cuda()
+    B.gqla_expand_cache(bd, cache_pd, x["w_uk"].cuda(), x["w_uv"].cuda(), kc_p, v_p, None)
+    N = x["cache"].shape[0]
+    kc = torch.empty((N, w.g, w.d_h), dtype=torch.bfloat16, device="cuda")
+    v = torch.empty_like(kc)
+    cache_d = x["cache"].cuda()
+    B.gqla_expand_cache(bd, cache_d, x["w_uk"].cuda(), x["w_uv"].cuda(), kc, v, None)
+    q = torch.cat([x["q_c"], x["q_r"]], -1).contiguous().cuda()
+    o_a, l_a = parts(w.d_h)
+    B.gqla_decode_gqa(bd, q, kc, v, cache_d[:, w.r_kv:], x["seq_start"].cuda(), sl, w.scale, S, o_a, l_a, status)
+    o_b, l_b = parts(w.d_h)
+    B.gqla_decode_gqa_paged(bd, q, kc_p, v_p, cache_pd[:, w.r_kv:], table_d, page_size, sl, w.scale, S, o_b, l_b, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    live = ~torch.isneginf(l_a)
+    if same_kernel:  # same pieces too; otherwise only the merged result is comparable (below)
+        assert torch.equal(l_a, l_b) and torch.equal(o_a[live], o_b[live])
+    o = torch.empty((w.batch, s_q, w.h_q, w.d_h), dtype=torch.bfloat16, device="cuda")
+    B.gqla_combine_splits(o_b, l_b, o, None)
+    o_ref = O.gqa_path(od, f["q_c"], f["q_r"], f["w_uk"], f["w_uv"], rows, ss, seqlens, s_q, w.scale)
+    assert_close(o.float().cpu().numpy(), o_ref, "paged gqa path")
+
+
 @pytest.mark.parametrize("hpg,g,s_q", [(1, 8, 1), (1, 4, 8), (3, 2, 1), (3, 4, 5), (5, 4, 3), (6, 2, 2), (7, 4, 4), (9, 1, 6),
                                        (12, 2, 7), (24, 4, 2), (32, 2, 3), (64, 1, 2), (128, 1, 1)])
 def test_heads_per_group_and_query_counts_off_the_powers_of_two(hpg, g, s_q):

@@ -400,3 +400,24 @@ def test_partials_with_an_explicit_plan_combine_to_the_same_output():
         fin = np.isfinite(ref_lse)
         assert np.array_equal(np.isneginf(lse), np.isneginf(ref_lse))
         np.testing.assert_allclose(lse[fin], ref_lse[fin], rtol=1e-12, atol=1e-12)
+
+
+def test_unpage_inverts_the_paged_layout():
+    """Paging is storage only.  The scatter that builds a paged pool (the input generator) and the oracle's
+    gather are written independently; composed, they must give back the packed rows, for page sizes that do
+    and do not divide the lengths, with empty sequences, and with the pages in a shuffled order."""
+    rng = np.random.default_rng(5)
+    seqlens = np.array([37, 0, 128, 1, 300], dtype=np.int32)
+    seq_start = np.concatenate([[0], np.cumsum(seqlens)[:-1]]).astype(np.int64)
+    packed = torch.from_numpy(rng.standard_normal((int(seqlens.sum()), 6)).astype(np.float32))
+    for page_size in (1, 16, 128, 256):
+        paged, table = synth.to_paged(packed, seq_start, seqlens, page_size, seed=11)
+        assert paged.shape[0] % page_size == 0
+        back, ss = O.unpage(paged.numpy(), table.numpy(), page_size, seqlens)
+        assert np.array_equal(ss, seq_start)
+        assert np.array_equal(back, packed.numpy())
+    # the identity table on an already paged-shaped array is a no-op
+    ident = np.arange(4, dtype=np.int32).reshape(1, 4)
+    x = rng.standard_normal((64, 3))
+    back, _ = O.unpage(x, ident, 16, np.array([64], dtype=np.int32))
+    assert np.array_equal(back, x)
