@@ -37,7 +37,7 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_absorb launch on C1 with the fixed plan S=1
 # (profiles/decode_absorb_tc_C1.md), valid for the kernel source with this digest only.
-NCU_TRAFFIC = {"bytes": 311.5e6 + 4.7e6, "kernel_sha256_16": "fc81fb26abc5cd4d", "num_splits": 1}
+NCU_TRAFFIC = {"bytes": 311.5e6 + 4.1e6, "kernel_sha256_16": "cedfc0569537fc07", "num_splits": 1}
 
 
 def load_peaks():

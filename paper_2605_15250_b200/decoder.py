@@ -15,8 +15,13 @@ class GqlaDecoder:
     """
 
     def __init__(self, h_q: int, g: int, d_h: int, r_kv: int, d_r: int, w_uk: torch.Tensor, w_uv: torch.Tensor,
-                 cache: torch.Tensor, seq_start: torch.Tensor, seqlens: torch.Tensor, scale: float):
+                 cache: torch.Tensor, seq_start: torch.Tensor | None, seqlens: torch.Tensor, scale: float,
+                 block_table: torch.Tensor | None = None, page_size: int = 0):
+        """Packed cache: `seq_start` [B] int64.  Paged cache: `block_table` [B, max_pages] int32 of page numbers
+        and `page_size` rows per page (`seq_start` is then ignored and may be None)."""
         assert cache.is_cuda and w_uk.is_cuda and w_uv.is_cuda
+        assert (block_table is None) == (page_size == 0) and (block_table is not None or seq_start is not None)
+        self.block_table, self.page_size = block_table, int(page_size)
         self.dims = B.make_dims(h_q, g, d_h, r_kv, d_r)
         self.h_q, self.g, self.d_h, self.r_kv, self.d_r = h_q, g, d_h, r_kv, d_r
         self.w_uk, self.w_uv, self.cache = w_uk, w_uv, cache
@@ -54,6 +59,8 @@ class GqlaDecoder:
     def append_expand(self, s_q: int) -> None:
         """After a step has written s_q new latent rows per sequence (and raised seqlens): expands just
         those rows into K_C, V (and k_R unless it aliases the latent cache)."""
+        if self.block_table is not None:
+            raise B.GqlaError("append_expand takes the packed layout; expand the touched pages with gqla_expand_cache")
         alias = self.k_r.data_ptr() == self.cache[:, self.r_kv:].data_ptr()
         B.gqla_append_expand(self.dims, s_q, self.cache, self.seq_start, self.seqlens, self.w_uk, self.w_uv, self.k_c,
                              self.v, None if alias else self.k_r)
@@ -71,8 +78,12 @@ class GqlaDecoder:
         lse = self._get("lse_a", (Bn, s_q, self.h_q), torch.float32) if want_lse else None
         o = self._get("o_a", (Bn, s_q, self.h_q, self.d_h), self.dtype)
         B.gqla_absorb_q(self.dims, q_c, q_r, self.w_uk, q_hat)
-        B.gqla_decode_absorb(self.dims, q_hat, self.cache, self.seq_start, self.seqlens, self.scale, num_splits,
-                             o_part, lse_part, self.status)
+        if self.block_table is None:
+            B.gqla_decode_absorb(self.dims, q_hat, self.cache, self.seq_start, self.seqlens, self.scale, num_splits,
+                                 o_part, lse_part, self.status)
+        else:
+            B.gqla_decode_absorb_paged(self.dims, q_hat, self.cache, self.block_table, self.page_size, self.seqlens,
+                                       self.scale, num_splits, o_part, lse_part, self.status)
         # with many slots per sequence the fused kernel (64 rows per CTA, one slot after the other) runs out of
         # parallelism; the separate merge streams the partials with every thread of the GPU
         if fused_tail and slots <= 4:
@@ -93,8 +104,12 @@ class GqlaDecoder:
         lse_part = self._get("lse_part_g", (Bn, slots, s_q, self.h_q), torch.float32)
         lse = self._get("lse_g", (Bn, s_q, self.h_q), torch.float32) if want_lse else None
         o = self._get("o_g", (Bn, s_q, self.h_q, self.d_h), self.dtype)
-        B.gqla_decode_gqa(self.dims, q, self.k_c, self.v, self.k_r, self.seq_start, self.seqlens, self.scale,
-                          num_splits, o_part, lse_part, self.status)
+        if self.block_table is None:
+            B.gqla_decode_gqa(self.dims, q, self.k_c, self.v, self.k_r, self.seq_start, self.seqlens, self.scale,
+                              num_splits, o_part, lse_part, self.status)
+        else:
+            B.gqla_decode_gqa_paged(self.dims, q, self.k_c, self.v, self.k_r, self.block_table, self.page_size,
+                                    self.seqlens, self.scale, num_splits, o_part, lse_part, self.status)
         B.gqla_combine_splits(o_part, lse_part, o, lse)
         return (o, lse) if want_lse else o
 

@@ -290,6 +290,36 @@ def test_paged_cache_gives_what_the_packed_cache_gives(dims, s_q, page_size, S):
     assert_close(o.float().cpu().numpy(), o_ref, "paged gqa path")
 
 
+def test_decoder_chains_over_a_paged_cache():
+    """GqlaDecoder with a block table: both chains (absorb with the fused tail, GQA after expanding the
+    whole pool) against the oracle on the rows gathered back."""
+    from tests.parity_util import assert_close, dims_of
+    from oracle import gqla_oracle as O
+    from paper_2605_15250_b200.decoder import GqlaDecoder
+    s_q, page_size = 2, 128
+    w = _wl("pagedec", 4, s_q, 170, **CANON)
+    seqlens = np.array([900, 3, 0, 260], dtype=np.int32)
+    x = synth.make_inputs(w, seqlens=seqlens, q_gain=4.0)
+    od, _ = dims_of(w)
+    cache_p, table = synth.to_paged(x["cache"], x["seq_start"], seqlens, page_size, seed=171)
+    dev = torch.device("cuda", 0)
+    dec = GqlaDecoder(w.h_q, w.g, w.d_h, w.r_kv, w.d_r, x["w_uk"].to(dev), x["w_uv"].to(dev), cache_p.to(dev), None,
+                      x["seqlens"].to(dev), w.scale, block_table=table.to(dev), page_size=page_size)
+    f = {k: synth.to_f64(x[k]) for k in ("q_c", "q_r", "w_uk", "w_uv")}
+    rows, ss = O.unpage(synth.to_f64(cache_p), table.numpy(), page_size, seqlens)
+    o = dec.absorb_step(x["q_c"].to(dev), x["q_r"].to(dev), -3)
+    assert_close(o.float().cpu().numpy(), O.absorb_path(od, f["q_c"], f["q_r"], f["w_uk"], f["w_uv"], rows, ss, seqlens, s_q,
+                                                        w.scale), "paged absorb chain")
+    dec.expand_cache()
+    q = torch.cat([x["q_c"], x["q_r"]], -1).contiguous().to(dev)
+    o = dec.gqa_step(q, -2)
+    dec.check_status()
+    assert_close(o.float().cpu().numpy(), O.gqa_path(od, f["q_c"], f["q_r"], f["w_uk"], f["w_uv"], rows, ss, seqlens, s_q,
+                                                     w.scale), "paged gqa chain")
+    with pytest.raises(B.GqlaError):
+        dec.append_expand(s_q)
+
+
 @pytest.mark.parametrize("hpg,g,s_q", [(1, 8, 1), (1, 4, 8), (3, 2, 1), (3, 4, 5), (5, 4, 3), (6, 2, 2), (7, 4, 4), (9, 1, 6),
                                        (12, 2, 7), (24, 4, 2), (32, 2, 3), (64, 1, 2), (128, 1, 1)])
 def test_heads_per_group_and_query_counts_off_the_powers_of_two(hpg, g, s_q):
