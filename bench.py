@@ -1,8 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the GQLA decode hot path on B200.
 
-A step = one pass of the absorb path (absorb_q -> decode_absorb -> combine_up_proj, the split merge
-fused with the up-projection)
+A step = one pass of the absorb path (absorb_q -> decode_absorb_final -> up_proj with one piece per
+sequence; absorb_q -> decode_absorb -> combine_up_proj, the split merge fused with the up-projection,
+when sequences are split)
 over the canonical workload (h_q=128, g=8, d_h=128, r_kv=512, d_r=64, B=64, T=4096, s_q=1,
 bf16 cache).  The GQA path (decode_gqa -> combine_splits on the expanded cache, s_q=2) is
 measured in the same run and reported under "paths".  One JSON line on stdout.
@@ -260,10 +261,16 @@ def run_ours(args):
         it["i"] += 1
         B.gqla_absorb_q(dec.dims, q_c, q_r, dec.w_uk, q_hat)
         a.record()
-        B.gqla_decode_absorb(dec.dims, q_hat, dec.cache, dec.seq_start, dec.seqlens, dec.scale, S_a, o_part, lse_part,
-                             dec.status)
-        b.record()
-        B.gqla_combine_up_proj(dec.dims, o_part, lse_part, dec.w_uv, o_out, None)
+        if S_a == 1:  # the chain GqlaDecoder.absorb_step runs with one piece per sequence
+            B.gqla_decode_absorb_final(dec.dims, q_hat, dec.cache, dec.seq_start, dec.seqlens, dec.scale, o_hat, None,
+                                       dec.status)
+            b.record()
+            B.gqla_up_proj(dec.dims, o_hat, dec.w_uv, o_out)
+        else:
+            B.gqla_decode_absorb(dec.dims, q_hat, dec.cache, dec.seq_start, dec.seqlens, dec.scale, S_a, o_part, lse_part,
+                                 dec.status)
+            b.record()
+            B.gqla_combine_up_proj(dec.dims, o_part, lse_part, dec.w_uv, o_out, None)
 
     # The step as a user serves it: the four launches captured once in a CUDA graph, one replay per step
     # (the eager chain costs more host time per step than the GPU needs to run it).
@@ -282,7 +289,8 @@ def run_ours(args):
     value = replicas.aggregate_tokens_per_s(world, w1.batch, w1.s_q, ms_per_step)
 
     kbytes = acct.decode_kernel_bytes("absorb", h_q=w1.h_q, g=w1.g, d_h=w1.d_h, r_kv=w1.r_kv, d_r=w1.d_r,
-                                      s_q=w1.s_q, batch=w1.batch, total_tokens=total_tokens, num_splits=pieces_a)
+                                      s_q=w1.s_q, batch=w1.batch, total_tokens=total_tokens, num_splits=pieces_a,
+                                      final=S_a == 1)
     kflops = acct.absorb_flops(w1.h_q, w1.r_kv, w1.d_r, w1.s_q, total_tokens)
     t_mem = kbytes / (peaks["hbm_gbs"] * 1e9)
     t_mma = kflops / (peaks["bf16_tflops"] * 1e12)
@@ -439,7 +447,7 @@ def run_ours(args):
             "config": {"workload": "C1 canonical absorb path: h_q=128 g=8 d_h=128 r_kv=512 d_r=64 B=64 T=4096 s_q=1 "
                                    "bf16 cache (576 elems/token)", "num_splits": S_a, "parallelism": "replicas only",
                        "l2": "inputs larger than L2 (302 MB cache vs 126 MB L2); no flush",
-                       "launch": "one CUDA-graph replay per step (3 kernels: absorb_q, decode_absorb, combine_up_proj); kernel time from an eager pass with events"},
+                       "launch": "one CUDA-graph replay per step (3 kernels: absorb_q, decode_absorb_final, up_proj with one piece per sequence; absorb_q, decode_absorb, combine_up_proj otherwise); kernel time from an eager pass with events"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * steps, "roofline": roof, "cpu_baseline": cpu,
             "paths": paths,
         }

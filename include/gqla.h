@@ -108,6 +108,16 @@ gqla_status gqla_decode_absorb(const gqla_dims* dims, gqla_dtype dtype, int32_t 
                                const int32_t* seqlens, float* o_part, float* lse_part, int32_t* status_word,
                                void* stream);
 
+/* Eq. (mqa), lines 3-5, for a whole sequence in one piece (no split-KV): the same attention as
+ * gqla_decode_absorb with num_splits = 1, but the normalised latent output is written once, in the
+ * storage dtype, instead of as an fp32 partial that a merge would only copy:
+ *   o_hat [B, s_q, h_q, r_kv] (out, same dtype as q_hat);  lse [B, s_q, h_q] fp32 (out) or NULL.
+ * It feeds gqla_up_proj directly.  Other arguments as for gqla_decode_absorb. */
+gqla_status gqla_decode_absorb_final(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                                     const void* q_hat, const void* cache, int64_t cache_row_stride,
+                                     int64_t cache_rows, const int64_t* seq_start, const int32_t* seqlens,
+                                     void* o_hat, float* lse, int32_t* status_word, void* stream);
+
 /* Sec. 3.1: k^C = W^UK c^KV, v^C = W^UV c^KV per group, k^R carried over -- the one-shot
  * cache expansion that switches from the absorb path to the GQA path.
  *   cache [N, r_kv+d_r] (row stride cache_row_stride);  w_uk, w_uv [g, r_kv, d_h]

@@ -27,14 +27,15 @@ def gqa_flops(h_q: int, d_h: int, d_r: int, s_q: int, total_tokens: int) -> int:
 
 
 def decode_kernel_bytes(path: str, *, h_q: int, g: int, d_h: int, r_kv: int, d_r: int, s_q: int, batch: int,
-                        total_tokens: int, num_splits: float, elem: int = 2) -> int:
+                        total_tokens: int, num_splits: float, elem: int = 2, final: bool = False) -> int:
     """Algorithmic bytes of ONE decode-kernel launch: cache once + queries + fp32 partials and LSE.
-    num_splits = partials written per sequence (under the balanced plan: live pieces / batch)."""
+    num_splits = partials written per sequence (under the balanced plan: live pieces / batch).
+    final: the whole-sequence absorb call, which writes the output once in the storage type and no LSE."""
     rows = batch * s_q * h_q
     if path == "absorb":
         cache = absorb_cache_bytes(r_kv, d_r, total_tokens, elem)
         q = elem * rows * (r_kv + d_r)
-        part = 4 * rows * num_splits * (r_kv + 1)
+        part = elem * rows * r_kv if final else 4 * rows * num_splits * (r_kv + 1)
     else:
         cache = gqa_cache_bytes(g, d_h, d_r, total_tokens, elem)
         q = elem * rows * (d_h + d_r)

@@ -37,6 +37,8 @@ _PROTOTYPES = {
     "gqla_absorb_q": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_decode_absorb": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
                                      c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_decode_absorb_final": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_int64,
+                                           c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_decode_absorb_paged": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
                                            c_int64, c_int64, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                            c_void_p, c_void_p]),
@@ -168,6 +170,20 @@ def gqla_expand_cache(dims: GqlaDims, cache: torch.Tensor, w_uk: torch.Tensor, w
     _check(lib().gqla_expand_cache(ctypes.byref(dims), _dtype_code(cache), cache.shape[0], _ptr(cache),
                                    cache.stride(0), _ptr(w_uk), _ptr(w_uv), _ptr(k_c), _ptr(v), _ptr(k_r),
                                    _stream()), "gqla_expand_cache")
+
+
+def gqla_decode_absorb_final(dims: GqlaDims, q_hat: torch.Tensor, cache: torch.Tensor, seq_start: torch.Tensor,
+                             seqlens: torch.Tensor, scale: float, o_hat: torch.Tensor, lse: torch.Tensor | None,
+                             status_word: torch.Tensor | None = None) -> None:
+    """Whole-sequence absorb-path attention (Eq. (mqa), lines 3-5): o_hat [B,s_q,h_q,r_kv] in the storage dtype."""
+    _contig(q_hat, seq_start, seqlens, o_hat, lse)
+    assert cache.dim() == 2 and cache.stride(1) == 1
+    assert seq_start.dtype == torch.int64 and seqlens.dtype == torch.int32 and o_hat.dtype == q_hat.dtype
+    assert lse is None or lse.dtype == torch.float32
+    B, s_q = q_hat.shape[0], q_hat.shape[1]
+    _check(lib().gqla_decode_absorb_final(ctypes.byref(dims), _dtype_code(q_hat), B, s_q, scale, _ptr(q_hat), _ptr(cache),
+                                          cache.stride(0), cache.shape[0], _ptr(seq_start), _ptr(seqlens), _ptr(o_hat),
+                                          _ptr(lse), _ptr(status_word), _stream()), "gqla_decode_absorb_final")
 
 
 def gqla_decode_absorb_paged(dims: GqlaDims, q_hat: torch.Tensor, cache: torch.Tensor, block_table: torch.Tensor,

@@ -20,6 +20,7 @@ struct DecodeArgs {
     float scale;
     float* o_part;    // [B, S, s_q, h_q, dv]
     float* lse_part;  // [B, S, s_q, h_q]
+    void* o_final;    // not null (S == 1 only): the output goes here in the storage type, o_part unused, lse_part may be null
 };
 
 constexpr int kGenericMaxV = 16;  // value columns per lane: dv <= 512
@@ -77,14 +78,18 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a) {
         m = m_new;
     }
 
-    float* o = a.o_part + row * a.dv;
     const float inv = l > 0.f ? 1.f / l : 0.f;
 #pragma unroll
     for (int c = 0; c < kGenericMaxV; ++c) {
         const int d = lane + 32 * c;
-        if (d < a.dv) o[d] = acc[c] * inv;
+        if (d < a.dv) {
+            if (a.o_final != nullptr)
+                stf((E*)a.o_final + row * a.dv + d, acc[c] * inv);
+            else
+                a.o_part[row * a.dv + d] = acc[c] * inv;
+        }
     }
-    if (lane == 0) a.lse_part[row] = l > 0.f ? m + logf(l) : -INFINITY;
+    if (lane == 0 && a.lse_part != nullptr) a.lse_part[row] = l > 0.f ? m + logf(l) : -INFINITY;
 }
 
 // Log-sum-exp merge: one block per (b, row).  Weights staged in shared memory.

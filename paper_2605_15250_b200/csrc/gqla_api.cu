@@ -342,6 +342,37 @@ gqla_status gqla_decode_absorb(const gqla_dims* d, gqla_dtype dtype, int32_t B, 
                              packed_rows(seq_start), seqlens, o_part, lse_part, status_word, stream);
 }
 
+gqla_status gqla_decode_absorb_final(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                                     const void* q_hat, const void* cache, int64_t cache_row_stride, int64_t cache_rows,
+                                     const int64_t* seq_start, const int32_t* seqlens, void* o_hat, float* lse,
+                                     int32_t* status_word, void* stream) {
+    gqla_status s;
+    if ((s = check_dims(d)) != GQLA_OK) return s;
+    if ((s = check_dtype(dtype)) != GQLA_OK) return s;
+    if (B < 0 || s_q < 1) return GQLA_ERR_SHAPE;
+    if (B == 0) return GQLA_OK;
+    if (q_hat == nullptr || cache == nullptr || seq_start == nullptr || seqlens == nullptr || o_hat == nullptr)
+        return GQLA_ERR_NULL;
+    if (!aligned16(q_hat) || !aligned16(cache) || !aligned16(o_hat)) return GQLA_ERR_ALIGN;
+    if (cache_row_stride < d->r_kv + d->d_r || cache_rows < 0) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const RowMap rows = packed_rows(seq_start);
+    if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, 0)) {
+        s = tc_decode_absorb(*d, B, s_q, scale, 1, q_hat, cache, cache_row_stride, cache_rows, rows, seqlens, nullptr, lse,
+                             status_word, st, o_hat);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
+    DecodeArgs a{};
+    a.q = q_hat;
+    a.kA = cache; a.kA_stride = cache_row_stride; a.kA_gstride = 0; a.dA = d->r_kv + d->d_r;
+    a.kB = nullptr; a.kB_stride = 0; a.dB = 0;
+    a.v = cache; a.v_stride = cache_row_stride; a.v_gstride = 0; a.dv = d->r_kv;
+    a.rows = rows; a.seqlens = seqlens;
+    a.B = B; a.S = 1; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
+    a.scale = scale; a.o_part = nullptr; a.lse_part = lse; a.o_final = o_hat;
+    return launch_decode_generic(dtype, a, st);
+}
+
 gqla_status gqla_decode_absorb_paged(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
                                      int32_t num_splits, const void* q_hat, const void* cache, int64_t cache_row_stride,
                                      int64_t cache_rows, const int32_t* block_table, int32_t max_pages,

@@ -43,6 +43,8 @@ struct AbsorbParams {
     const int32_t* seqlens;
     float* o_part;    // [B, S, s_q*h_q, 512]
     float* lse_part;  // [B, S, s_q*h_q]
+    __nv_bfloat16* o_final;  // not null: S = 1, fixed plan; the normalised output goes here as bf16 [B, s_q*h_q, 512]
+                             // (o_part unused, lse_part may be null)
     int32_t* status;
 };
 
@@ -328,7 +330,7 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
             const int32_t T = p.seqlens[pc.b];
             const int64_t slot0 = (int64_t)pc.b * p.S;
             // split slots this worker marks empty
-            if (part == 0 && row_valid)
+            if (part == 0 && row_valid && p.lse_part != nullptr)
                 for (int kk = pc.fill_begin; kk < pc.fill_end; ++kk) p.lse_part[(slot0 + kk) * p.rows_total + rho] = -INFINITY;
             if (pc.n_tiles == 0 && p.balanced) continue;  // an empty sequence: its slots were marked above
             int32_t lim = visible_limit(T, p.s_q, pq);
@@ -442,54 +444,90 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
             // P.V has completed) as 1 KB bulk stores, the 256 columns of MMA m = 0 first, then those of m = 1.
             // The padded pitch keeps the 16-byte stores of a quarter warp on distinct banks.
             uint8_t* stage = tiles + L::kOffP;
-            float* gbase = p.o_part + ((slot0 + pc.k) * p.rows_total + rho0) * 512;
+            if (p.o_final != nullptr) {
+                // whole-sequence call: the final bf16 rows (1 KB each) fit the staging at once -- one pass
+                uint4* dst = reinterpret_cast<uint4*>(stage + r * L::kOutPitch + (128 * hf + 64 * ch) * 2);
 #pragma unroll 1
-            for (int m = 0; m < 2; ++m) {
-                float4* dst = reinterpret_cast<float4*>(stage + r * L::kOutPitch + (128 * hf + 64 * ch) * 4);
-#pragma unroll 1
-                for (int c = 0; c < 64; c += 32) {
+                for (int mc = 0; mc < 4; ++mc) {  // (m, 32-column half) of this thread's 64 columns of each m
+                    const int m = mc >> 1, c = (mc & 1) * 32;
                     uint32_t o[32];
                     if (pc.n_tiles > 0 && ok) {  // warp-uniform
                         tmem_ld32(lane_base + kAColO + m * 128 + ch * 64 + c, o);
                         tmem_wait_ld();
                     }
+                    auto pk = [&](int e) -> uint32_t {  // columns e, e + 1 of this chunk, normalised (0 for a dead row)
+                        return live ? pack_bf16(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv) : 0u;
+                    };
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        dst[c / 4 + i] =
-                            live ? make_float4(__uint_as_float(o[4 * i]) * inv, __uint_as_float(o[4 * i + 1]) * inv,
-                                               __uint_as_float(o[4 * i + 2]) * inv, __uint_as_float(o[4 * i + 3]) * inv)
-                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int i = 0; i < 4; ++i)
+                        dst[(256 * m + c) * 2 / 16 + i] = make_uint4(pk(8 * i), pk(8 * i + 2), pk(8 * i + 4), pk(8 * i + 6));
                 }
-                fence_proxy_async_smem();  // staged rows -> visible to the bulk-copy engine
-                if (m == 1) {              // O has been read: the next piece's first P.V may overwrite it
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(o_free_l);
-                }
+                fence_proxy_async_smem();
+                tc_fence_before();
                 __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(o_free_l);
                 if (lane == 0) mbar_arrive(epi);
                 if (!__all_sync(0xffffffffu, mbar_wait(epi, ec & 1, ab, 12))) ok = false;
                 ++ec;
                 if (ok && lane < 8) {
-                    const int rr = (warp - 2) * 8 + lane;  // each softmax warp ships eight rows
+                    const int rr = (warp - 2) * 8 + lane;
                     if (rho0 + rr < p.rows_total) {
-                        bulk_store(gbase + (int64_t)rr * 512 + 256 * m, stage + rr * L::kOutPitch, 256 * 4);
+                        bulk_store(p.o_final + ((int64_t)pc.b * p.rows_total + rho0 + rr) * 512, stage + rr * L::kOutPitch,
+                                   512 * 2);
                         bulk_commit();
                         bulk_wait_read();
                     }
                 }
-                if (m == 0) {  // the staging is rewritten next: every warp's stores must have read it
+            } else {
+                float* gbase = p.o_part + ((slot0 + pc.k) * p.rows_total + rho0) * 512;
+#pragma unroll 1
+                for (int m = 0; m < 2; ++m) {
+                    float4* dst = reinterpret_cast<float4*>(stage + r * L::kOutPitch + (128 * hf + 64 * ch) * 4);
+#pragma unroll 1
+                    for (int c = 0; c < 64; c += 32) {
+                        uint32_t o[32];
+                        if (pc.n_tiles > 0 && ok) {  // warp-uniform
+                            tmem_ld32(lane_base + kAColO + m * 128 + ch * 64 + c, o);
+                            tmem_wait_ld();
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            dst[c / 4 + i] =
+                                live ? make_float4(__uint_as_float(o[4 * i]) * inv, __uint_as_float(o[4 * i + 1]) * inv,
+                                                   __uint_as_float(o[4 * i + 2]) * inv, __uint_as_float(o[4 * i + 3]) * inv)
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    fence_proxy_async_smem();  // staged rows -> visible to the bulk-copy engine
+                    if (m == 1) {              // O has been read: the next piece's first P.V may overwrite it
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(o_free_l);
+                    }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(epi);
                     if (!__all_sync(0xffffffffu, mbar_wait(epi, ec & 1, ab, 12))) ok = false;
                     ++ec;
+                    if (ok && lane < 8) {
+                        const int rr = (warp - 2) * 8 + lane;  // each softmax warp ships eight rows
+                        if (rho0 + rr < p.rows_total) {
+                            bulk_store(gbase + (int64_t)rr * 512 + 256 * m, stage + rr * L::kOutPitch, 256 * 4);
+                            bulk_commit();
+                            bulk_wait_read();
+                        }
+                    }
+                    if (m == 0) {  // the staging is rewritten next: every warp's stores must have read it
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(epi);
+                        if (!__all_sync(0xffffffffu, mbar_wait(epi, ec & 1, ab, 12))) ok = false;
+                        ++ec;
+                    }
                 }
             }
             // staging (and with it P and the V ring) is free again once every warp's stores have read it
             __syncwarp();
             if (lane == 0) mbar_arrive(epi_done);
             if (!__all_sync(0xffffffffu, mbar_wait(epi_done, pi & 1, ab, 12))) ok = false;
-            if (row_valid && part == 0)
+            if (row_valid && part == 0 && p.lse_part != nullptr)
                 p.lse_part[(slot0 + pc.k) * p.rows_total + rho] =
                     live ? (m_used + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
             gt += pc.n_tiles;

@@ -281,7 +281,8 @@ inline gqla_status tc_combine_up_proj(const gqla_dims& d, gqla_dtype dtype, int3
 inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S,
                                     const void* q_hat, const void* cache, int64_t cache_row_stride,
                                     int64_t cache_rows, const RowMap& rows, const int32_t* seqlens,
-                                    float* o_part, float* lse_part, int32_t* status, cudaStream_t st) {
+                                    float* o_part, float* lse_part, int32_t* status, cudaStream_t st,
+                                    void* o_final = nullptr) {
     if (!tc_covers(d, GQLA_BF16, s_q, 0) || !stride_ok(cache_row_stride) || cache_rows > 0x7fffffffLL ||
         cache_rows < 1)
         return GQLA_ERR_UNSUPPORTED;
@@ -314,6 +315,8 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
     p.balanced = balanced ? 1 : 0; p.W = workers;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.rows = rows; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
+    p.o_final = (__nv_bfloat16*)o_final;
+    if (o_final != nullptr && (balanced || S != 1)) return GQLA_ERR_UNSUPPORTED;
     auto kern = tc::decode_absorb_tc_kernel<0>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AbsorbSmem::kTotal) != cudaSuccess)
         return GQLA_ERR_CUDA;

@@ -68,7 +68,8 @@ class GqlaDecoder:
     # ---- absorb path ----
     def absorb_step(self, q_c: torch.Tensor, q_r: torch.Tensor, num_splits: int = 1, want_lse: bool = False,
                     fused_tail: bool = True):
-        """absorb_q -> decode_absorb -> combine_up_proj (or combine_splits -> up_proj when fused_tail is off)."""
+        """absorb_q -> decode_absorb -> combine_up_proj (or combine_splits -> up_proj when fused_tail is off);
+        with one split per sequence: absorb_q -> decode_absorb_final -> up_proj."""
         Bn, s_q = q_c.shape[0], q_c.shape[1]
         slots = abs(num_splits)  # num_splits < 0: balanced plan with that many slots per sequence
         q_hat = self._get("q_hat", (Bn, s_q, self.h_q, self.r_kv + self.d_r), self.dtype)
@@ -78,6 +79,12 @@ class GqlaDecoder:
         lse = self._get("lse_a", (Bn, s_q, self.h_q), torch.float32) if want_lse else None
         o = self._get("o_a", (Bn, s_q, self.h_q, self.d_h), self.dtype)
         B.gqla_absorb_q(self.dims, q_c, q_r, self.w_uk, q_hat)
+        if num_splits == 1 and self.block_table is None:
+            # one piece per sequence: no partials, the latent output goes straight to the up-projection
+            B.gqla_decode_absorb_final(self.dims, q_hat, self.cache, self.seq_start, self.seqlens, self.scale, o_hat, lse,
+                                       self.status)
+            B.gqla_up_proj(self.dims, o_hat, self.w_uv, o)
+            return (o, lse) if want_lse else o
         if self.block_table is None:
             B.gqla_decode_absorb(self.dims, q_hat, self.cache, self.seq_start, self.seqlens, self.scale, num_splits,
                                  o_part, lse_part, self.status)

@@ -94,9 +94,15 @@ def time_case(dec: GqlaDecoder, w: synth.Workload, x: dict, path: str, S: int, s
         o_part = dec._get("o_part_a", (w.batch, slots, w.s_q, w.h_q, w.r_kv), torch.float32)
         lse_part = dec._get("lse_part_a", (w.batch, slots, w.s_q, w.h_q), torch.float32)
 
+        o_hat = dec._get("o_hat", (w.batch, w.s_q, w.h_q, w.r_kv), torch.bfloat16)
+
         def kernel():
-            B.gqla_decode_absorb(dec.dims, q_hat, dec.cache, dec.seq_start, dec.seqlens, dec.scale, S, o_part, lse_part,
-                                 dec.status)
+            if S == 1:  # the call the chain uses with one piece per sequence
+                B.gqla_decode_absorb_final(dec.dims, q_hat, dec.cache, dec.seq_start, dec.seqlens, dec.scale, o_hat, None,
+                                           dec.status)
+            else:
+                B.gqla_decode_absorb(dec.dims, q_hat, dec.cache, dec.seq_start, dec.seqlens, dec.scale, S, o_part,
+                                     lse_part, dec.status)
 
         flops = acct.absorb_flops(w.h_q, w.r_kv, w.d_r, w.s_q, total_tokens)
     else:
@@ -116,7 +122,8 @@ def time_case(dec: GqlaDecoder, w: synth.Workload, x: dict, path: str, S: int, s
         return {}
     pieces = _pieces(x["seqlens"], S, W, w.batch)
     nbytes = acct.decode_kernel_bytes(path, h_q=w.h_q, g=w.g, d_h=w.d_h, r_kv=w.r_kv, d_r=w.d_r, s_q=w.s_q,
-                                      batch=w.batch, total_tokens=total_tokens, num_splits=pieces)
+                                      batch=w.batch, total_tokens=total_tokens, num_splits=pieces,
+                                      final=path == "absorb" and S == 1)
     replay, _ = dec.capture(step, *args)
     for _ in range(warmup):
         replay()

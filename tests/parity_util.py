@@ -73,6 +73,17 @@ def stagewise(w: synth.Workload, seqlens, num_splits: int, q_gain: float = 1.0, 
         errs["absorb_o_part"] = assert_close(o_part.cpu().numpy(), op_ref, "decode_absorb o_part")
         errs["absorb_lse_part"] = assert_close(lse_part.cpu().numpy(), lp_ref, "decode_absorb lse_part")
 
+    # the whole-sequence call: final latent output in the storage dtype, no partials
+    oh_w = torch.full((Bn, s_q, w.h_q, w.r_kv), float("nan"), dtype=dt, device="cuda")
+    lse_w = torch.full((Bn, s_q, w.h_q), float("nan"), dtype=torch.float32, device="cuda")
+    B.gqla_decode_absorb_final(bd, qh_in.cuda(), dev["cache"], dev["seq_start"], dev["seqlens"], w.scale, oh_w, lse_w, status)
+    ohw_ref, lw_ref = O.decode_absorb(od, synth.to_f64(qh_in), f["cache"], ss, sl, s_q, w.scale)
+    errs["absorb_final_o"] = assert_close(oh_w.float().cpu().numpy(), ohw_ref, "decode_absorb_final o_hat")
+    errs["absorb_final_lse"] = assert_close(lse_w.cpu().numpy(), lw_ref, "decode_absorb_final lse")
+    oh_n = torch.full_like(oh_w, float("nan"))
+    B.gqla_decode_absorb_final(bd, qh_in.cuda(), dev["cache"], dev["seq_start"], dev["seqlens"], w.scale, oh_n, None, status)
+    assert torch.equal(oh_n, oh_w), "decode_absorb_final without an lse output must give the same o_hat"
+
     # combine on the oracle's partials (fp32)
     op_in = torch.from_numpy(op_ref).float()
     lp_in = torch.from_numpy(lp_ref).float()

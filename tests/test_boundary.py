@@ -121,6 +121,11 @@ def test_argument_errors_return_before_launch():
     assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, p, p, 576, 10, None, p, p, p, None, None) == 1
     assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, p, p, 100, 10, p, p, p, p, None, None) == 2
     assert L.gqla_decode_absorb(r(d), 0, 1, 1, 0.1, 1, odd, p, 576, 10, p, p, p, p, None, None) == 3
+    assert L.gqla_decode_absorb_final(r(d), 0, 1, 0, 0.1, p, p, 576, 10, p, p, p, None, None, None) == 2  # s_q < 1
+    assert L.gqla_decode_absorb_final(r(d), 0, 1, 1, 0.1, p, p, 576, 10, p, p, None, None, None, None) == 1
+    assert L.gqla_decode_absorb_final(r(d), 0, 1, 1, 0.1, p, p, 576, 10, p, p, odd, None, None, None) == 3
+    assert L.gqla_decode_absorb_final(r(d), 0, 1, 1, 0.1, p, p, 100, 10, p, p, p, None, None, None) == 2
+    assert L.gqla_decode_absorb_final(r(d), 0, 0, 1, 0.1, None, None, 576, 0, None, None, None, None, None, None) == 0
     assert L.gqla_decode_absorb_paged(r(d), 0, 1, 1, 0.1, 1, p, p, 576, 10, None, 4, 128, p, p, p, None, None) == 1
     assert L.gqla_decode_absorb_paged(r(d), 0, 1, 1, 0.1, 1, p, p, 576, 10, p, 4, 0, p, p, p, None, None) == 2  # page size
     assert L.gqla_decode_absorb_paged(r(d), 0, 1, 1, 0.1, 1, p, p, 576, 10, p, 0, 128, p, p, p, None, None) == 2
