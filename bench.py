@@ -36,9 +36,9 @@ from paper_2605_15250_b200 import synth
 METRIC = "decode attn tokens/s (absorb path, canonical config, 1 B200)"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_absorb launch on C1 with the fixed plan S=1
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_absorb_final launch on C1 (one piece per sequence)
 # (profiles/decode_absorb_tc_C1.md), valid for the kernel source with this digest only.
-NCU_TRAFFIC = {"bytes": 311.5e6 + 4.1e6, "kernel_sha256_16": "cedfc0569537fc07", "num_splits": 1}
+NCU_TRAFFIC = {"bytes": 311.5e6 + 5.1e6, "kernel_sha256_16": "6bcbc12d46f63e73", "num_splits": 1}
 
 
 def load_peaks():
