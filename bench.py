@@ -32,6 +32,7 @@ import torch
 from paper_2605_15250_b200 import accounting as acct
 from paper_2605_15250_b200 import replicas
 from paper_2605_15250_b200 import synth
+from paper_2605_15250_b200.timing import kernel_ms_back_to_back
 
 METRIC = "decode attn tokens/s (absorb path, canonical config, 1 B200)"
 UNIT = "tokens/s"
@@ -188,31 +189,6 @@ def time_region(fn, steps: int, dist_on: bool):
     if dist_on:
         dist.barrier()
     return replicas.max_over_ranks(e0.elapsed_time(e1), "cuda")
-
-
-def kernel_ms_back_to_back(launch, launches: int) -> float:
-    """Mean device time of one launch when the kernel runs back to back: `launches` launches replayed from CUDA
-    graphs of ten (so the host's launch cost cannot stretch the figure), one event pair around all of them."""
-    per_graph = 10
-    launch()
-    g = torch.cuda.CUDAGraph()
-    side = torch.cuda.Stream()
-    side.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(side):
-        with torch.cuda.graph(g, stream=side):
-            for _ in range(per_graph):
-                launch()
-    torch.cuda.current_stream().wait_stream(side)
-    replays = max(1, launches // per_graph)
-    g.replay()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(replays):
-        g.replay()
-    e1.record()
-    torch.cuda.synchronize()
-    return e0.elapsed_time(e1) / (replays * per_graph)
 
 
 def run_ours(args):

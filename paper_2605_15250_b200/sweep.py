@@ -1,8 +1,8 @@
 """Timing sweep of both decode paths over the five workloads (python -m paper_2605_15250_b200.sweep).
 
-For every (workload, path, s_q, split plan) it times the decode kernel alone (CUDA events around each
-launch) and the whole path chain as one CUDA-graph replay per step, and prints one JSON line with
-tokens/s, algorithmic GB/s and TFLOP/s, and the fraction of the roofline time max(bytes/BW, FLOPs/peak)
+For every (workload, path, s_q, split plan) it times the decode kernel alone (running back to back, replayed
+from CUDA graphs of ten launches) and the whole path chain as one CUDA-graph replay per step, and prints one
+JSON line with tokens/s, algorithmic GB/s and TFLOP/s, and the fraction of the roofline time max(bytes/BW, FLOPs/peak)
 against the measured peaks (MEASURED_PEAKS.json beside bench.py, if present) and the nominal B200
 figures (8 TB/s, 2.25 PFLOP/s dense bf16).  Inputs are the seeded synthetic workloads of synth.py.
 """
@@ -11,7 +11,6 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import statistics
 
 import torch
 
@@ -20,6 +19,7 @@ from . import binding as B
 from . import build as gbuild
 from . import synth
 from .decoder import GqlaDecoder
+from .timing import kernel_ms_back_to_back
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
@@ -69,14 +69,8 @@ def time_paged(dec: GqlaDecoder, w: synth.Workload, x: dict, path: str, S: int, 
                                     o_part, lse_part, dec.status)
     for _ in range(warmup):
         kernel()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    for a, b in ev:
-        a.record()
-        kernel()
-        b.record()
-    torch.cuda.synchronize()
+    k_us = kernel_ms_back_to_back(kernel, steps) * 1e3
     dec.check_status()
-    k_us = statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
     return {"workload": w.name, "path": path, "s_q": w.s_q, "batch": w.batch, "total_tokens": total_tokens,
             "layout": f"paged, {page_size} rows per page, shuffled", "plan": "balanced" if S < 0 else "fixed",
             "slots": slots, "kernel_us": round(k_us, 1)}
@@ -136,14 +130,8 @@ def time_case(dec: GqlaDecoder, w: synth.Workload, x: dict, path: str, S: int, s
     e1.record()
     torch.cuda.synchronize()
     chain_us = e0.elapsed_time(e1) * 1e3 / steps
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    for a, b in ev:
-        a.record()
-        kernel()
-        b.record()
-    torch.cuda.synchronize()
+    k_us = kernel_ms_back_to_back(kernel, steps) * 1e3
     dec.check_status()
-    k_us = statistics.median(a.elapsed_time(b) for a, b in ev) * 1e3
     peaks, kind = _peaks()
     t = k_us * 1e-6
     out = {
