@@ -15,7 +15,6 @@ namespace {
 std::atomic<int> g_policy{GQLA_POLICY_AUTO};
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-inline size_t elem_size(gqla_dtype t) { return t == GQLA_BF16 ? 2 : 4; }
 
 gqla_status check_dims(const gqla_dims* d) {
     if (d == nullptr) return GQLA_ERR_NULL;
