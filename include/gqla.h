@@ -89,6 +89,16 @@ typedef enum { GQLA_POLICY_AUTO = 0, GQLA_POLICY_GENERIC = 1 } gqla_policy;
 void gqla_set_policy(gqla_policy p);
 int32_t gqla_get_policy(void);
 
+/* Status word of the calls that have no status_word argument (gqla_absorb_q, gqla_up_proj,
+ * gqla_expand_cache, gqla_append_expand, gqla_combine_up_proj; not in the paper: error reporting only).
+ * Their tensor-core kernels bound every device-side wait like the decode kernels do; with a word registered
+ * here (a device int32 the caller owns and has set to 0, process-wide, NULL = none, the default) an expired
+ * wait leaves GQLA_ERR_TIMEOUT | (place << 8) in it instead of going unnoticed.  The word must stay valid
+ * while any such call is in flight; it is read and written by kernels only, never by the host side of
+ * the library.  gqla_get_status_word returns what was registered. */
+void gqla_set_status_word(int32_t* device_word);
+int32_t* gqla_get_status_word(void);
+
 /* Eq. (mqa), line 2:  q_hat_i = [ (W^UK_{j(i)})^T q_i^C ; q_i^R ].
  *   q_c   [B, s_q, h_q, d_h]   q_r [B, s_q, h_q, d_r]   w_uk [g, r_kv, d_h]
  *   q_hat [B, s_q, h_q, r_kv + d_r]  (out, same dtype) */
@@ -154,14 +164,18 @@ gqla_status gqla_decode_gqa(const gqla_dims* dims, gqla_dtype dtype, int32_t B, 
  * manager claimed the whole GPU at start-up, a loop that cannot afford the device-wide synchronisation of
  * cudaMalloc/cudaFree, or a C caller with no allocator of its own.  The partials are kept in an array built
  * into the library's device image, so the call allocates and frees nothing.
- *   Inputs as for gqla_decode_gqa.  out [B, s_q, h_q, d_h] of `dtype` (device, 16-byte aligned),
- *   lse [B, s_q, h_q] fp32 (device) or NULL.
+ *   Inputs as for gqla_decode_gqa, except that num_splits must be >= 1 (the fixed split plan; the balanced
+ *   plan, num_splits <= -2, returns GQLA_ERR_SHAPE here).  out [B, s_q, h_q, d_h] of `dtype` (device,
+ *   16-byte aligned), lse [B, s_q, h_q] fp32 (device) or NULL.
  *   Limits: B*num_splits*s_q*h_q <= 65536 rows and rows*d_h <= 4194304 floats (16 MiB + 256 KiB in all);
  *   anything larger returns GQLA_ERR_CAPACITY before any launch -- use gqla_decode_gqa with your own
- *   buffers then.  Each GPU that runs the library's kernels holds the array until the process exits.
+ *   buffers then.  Each GPU that runs this entry point holds the array until the process exits.
  *   The first call on a device looks up the array's device address (one runtime query, remembered per
- *   device; the device must be current, as for every call).  Make that first call before starting any
- *   stream capture.
+ *   device; the device must be current, as for every call).  That query is also the moment the CUDA
+ *   runtime loads this part of the library onto the device and reserves the array there.  So make one
+ *   call per device at start-up -- B = 0 is enough: it performs the query and launches nothing -- before
+ *   any stream capture and, on a host whose memory manager takes the whole GPU, before it does so; if
+ *   the array cannot be placed any more the call returns GQLA_ERR_CUDA.
  *   All calls on one GPU share the array and it keeps the previous call's contents.  Nothing needs
  *   clearing (every partial is rewritten before it is read), but two calls that may run concurrently on
  *   the same GPU race on it: issue them on one stream or order them yourself. */

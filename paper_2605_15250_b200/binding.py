@@ -34,6 +34,8 @@ _lib = None
 _PROTOTYPES = {
     "gqla_set_policy": (None, [c_int32]),
     "gqla_get_policy": (c_int32, []),
+    "gqla_set_status_word": (None, [c_void_p]),
+    "gqla_get_status_word": (c_void_p, []),
     "gqla_absorb_q": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_decode_absorb": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
                                      c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -129,6 +131,19 @@ def set_policy(policy: int) -> None:
 
 def get_policy() -> int:
     return lib().gqla_get_policy()
+
+
+def set_status_word(word: torch.Tensor | None) -> None:
+    """Registers the device int32 that the projection calls (absorb_q, up_proj, expand_cache, append_expand,
+    combine_up_proj) report an expired device-side wait in; None unregisters.  Keep the tensor alive."""
+    if word is not None:
+        assert word.is_cuda and word.dtype == torch.int32 and word.numel() >= 1
+    lib().gqla_set_status_word(_ptr(word))
+
+
+def get_status_word() -> int:
+    """Address registered with set_status_word (0 = none)."""
+    return int(lib().gqla_get_status_word() or 0)
 
 
 def kernel_for(dims: GqlaDims, dtype: torch.dtype, s_q: int, path: str) -> str:
@@ -249,8 +264,10 @@ def gqla_decode_gqa_noalloc(dims: GqlaDims, q: torch.Tensor, k_c: torch.Tensor, 
                             status_word: torch.Tensor | None = None) -> None:
     """GQA-path step (attention + split merge) that keeps its split partials in the library's built-in
     device array instead of caller buffers, for hosts that must not allocate device memory while decoding.
-    out is [B, s_q, h_q, d_h]; raises (capacity) when B*num_splits*s_q*h_q > 65536 or that times d_h > 4 Mi.
-    Calls on one GPU share the array: keep them on one stream."""
+    out is [B, s_q, h_q, d_h]; num_splits >= 1 (fixed plan only); raises (capacity) when
+    B*num_splits*s_q*h_q > 65536 or that times d_h > 4 Mi.  Calls on one GPU share the array: keep them on
+    one stream.  Call it once per device at start-up (an empty batch will do) so that the array exists
+    before the host's memory manager claims the GPU."""
     _contig(q, k_c, v, seq_start, seqlens, out, lse)
     assert k_r.dim() == 2 and k_r.stride(1) == 1
     assert seq_start.dtype == torch.int64 and seqlens.dtype == torch.int32

@@ -47,6 +47,9 @@ extern "C" {
 void gqla_set_policy(gqla_policy p) { g_policy.store(p == GQLA_POLICY_GENERIC ? GQLA_POLICY_GENERIC : GQLA_POLICY_AUTO); }
 int32_t gqla_get_policy(void) { return g_policy.load(); }
 
+void gqla_set_status_word(int32_t* device_word) { projection_status_word() = device_word; }
+int32_t* gqla_get_status_word(void) { return projection_status_word(); }
+
 const char* gqla_status_str(gqla_status s) {
     switch (s) {
         case GQLA_OK: return "ok";

@@ -13,12 +13,18 @@
 // For them the partials live in a fixed array that is part of this library's device image.
 //
 // What that costs.  Every GPU on which the library's kernels get loaded carries the array
-// (kScratchBytes, a little over 16 MiB) until the process exits, used or not.  There is one array
+// (kScratchFloats floats, a little over 16 MiB) until the process exits, used or not.  There is one array
 // per GPU and every call on that GPU writes into it, so two calls whose kernels may overlap on the
 // device (different streams, no ordering between them) corrupt each other: keep such calls on one
 // stream or order them with events.  The array keeps whatever the previous call left there; this
 // is harmless because the attention kernel rewrites every partial of the current call, empty
 // splits included, before the merge reads it -- nothing in it has to start at zero.
+//
+// When the array comes into being.  The CUDA runtime loads a module lazily: the array is reserved on a
+// GPU when this file's device code is first needed there, which is the first call of the entry point on
+// that GPU (the address query below, also for a call with B = 0).  A host whose memory manager is going
+// to claim the whole GPU must therefore make one call per device -- B = 0 is enough, it launches nothing
+// -- at start-up, BEFORE it claims the memory; later calls allocate nothing.
 #include <cuda_runtime.h>
 #include <math.h>
 
@@ -32,8 +38,7 @@ namespace {
 // Capacity: partial outputs first, partial log-sum-exps behind them.
 constexpr int64_t kMaxPartialFloats = 4ll << 20;  // rows * d_h      <= 4 Mi floats (16 MiB)
 constexpr int64_t kMaxPartialRows = 64ll << 10;   // B*S*s_q*h_q     <= 64 Ki rows  (256 KiB)
-constexpr int64_t kScratchFloats = kMaxPartialFloats + kMaxPartialRows;
-constexpr int64_t kScratchBytes = kScratchFloats * (int64_t)sizeof(float);
+constexpr int64_t kScratchFloats = kMaxPartialFloats + kMaxPartialRows;  // 16 MiB + 256 KiB of floats
 
 // In host code this name is only a handle for the runtime's symbol table.  It is NOT a device
 // address: handing `g_split_scratch` itself to a kernel launch would give the kernel a host pointer.
@@ -102,12 +107,14 @@ extern "C" gqla_status gqla_decode_gqa_noalloc(const gqla_dims* dims, gqla_dtype
     if (dtype != GQLA_BF16 && dtype != GQLA_F32) return GQLA_ERR_DTYPE;
     if (dims->h_q <= 0 || dims->d_h <= 0 || B < 0 || s_q < 1 || num_splits < 1) return GQLA_ERR_SHAPE;
     if ((reinterpret_cast<uintptr_t>(out) & 15u) != 0) return GQLA_ERR_ALIGN;
-    if (B == 0) return GQLA_OK;
     // Capacity check before anything touches the device: the partials of this call must fit the array.
     const int64_t rows = (int64_t)B * num_splits * s_q * dims->h_q;
     if (rows > kMaxPartialRows || rows * dims->d_h > kMaxPartialFloats) return GQLA_ERR_CAPACITY;
+    // The address query comes before the B == 0 return on purpose: an empty call is the documented way to
+    // make the runtime load this module (and reserve the array) on the current device at start-up.
     float* scratch = scratch_for_current_device();
     if (scratch == nullptr) return GQLA_ERR_CUDA;
+    if (B == 0) return GQLA_OK;
     float* o_part = scratch;
     float* lse_part = scratch + kMaxPartialFloats;
     // The attention kernel is the library's ordinary one; it gets the translated device address.

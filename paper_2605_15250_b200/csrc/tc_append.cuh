@@ -33,6 +33,7 @@ struct AppendSmem {
     static constexpr int kNumBars = 3;  // a_ready b_full acc_full
     static constexpr int kThreads = 192;
     static constexpr int kTotal = 1024 + kTileBytes + kNumBars * 8 + 16 + kRows * 8;
+    static_assert(OneCtaPerSM<kTotal>::value, "");
 };
 
 __global__ void __launch_bounds__(AppendSmem::kThreads, 1)

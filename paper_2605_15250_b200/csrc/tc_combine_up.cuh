@@ -36,6 +36,7 @@ struct CombineUpSmem {
     static constexpr int kThreads = 192;
     static constexpr int kMaxS = 64;            // split slots the kernel takes (their lse is staged per row)
     static constexpr int kTotal = 1024 + kTileBytes + kNumBars * 8 + 16 + 2 * kRows * 4 + kRows * kMaxS * 4 + kRows * 8;
+    static_assert(OneCtaPerSM<kTotal>::value, "");
 };
 
 __global__ void __launch_bounds__(CombineUpSmem::kThreads, 1)

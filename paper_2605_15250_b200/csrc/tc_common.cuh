@@ -344,6 +344,19 @@ __device__ __forceinline__ void umma_commit2(uint64_t* bar, uint16_t mask) {
 // every CTA of that kernel has executed pdl_launch_dependents or exited.  It must call pdl_wait before it
 // touches global memory: the wait returns when the previous kernel has completed and its writes are
 // visible.  Both instructions do nothing in a kernel launched the ordinary way.
+//
+// Every tensor-core kernel here signals its dependents before (or while) it allocates tensor memory, and
+// tcgen05.alloc blocks until the columns are free.  That is only safe while two such CTAs can never share an
+// SM: otherwise a dependent CTA could take the SM's tensor memory first and then sit in pdl_wait for a
+// primary CTA that is blocked in its own allocation.  Shared memory rules it out -- each of these kernels
+// asks for more than half of an SM's shared memory -- and every kernel states that with this check.
+constexpr int kSmemPerSM = 233472;  // bytes of shared memory of one sm_100 SM
+template <int kDynamicSmemBytes>
+struct OneCtaPerSM {
+    static_assert(2 * kDynamicSmemBytes > kSmemPerSM,
+                  "two CTAs of a kernel that triggers its dependents before allocating tensor memory must not fit one SM");
+    static constexpr bool value = true;
+};
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 

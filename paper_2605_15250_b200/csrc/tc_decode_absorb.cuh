@@ -75,6 +75,7 @@ struct AbsorbSmem {
     static constexpr int kTotal = kTileBytes + kNumBars * 8 + 16 + 2 * 4 * 64 * 4;
     static_assert(2 * 4 * 64 >= kThreads + 4, "plan scratch must fit in sm_max");
     static_assert(kTotal <= 232448, "shared memory budget of one CTA");
+    static_assert(OneCtaPerSM<kTotal>::value, "");
 };
 
 constexpr uint32_t kAColO = 0;    // O: MMA m (latent columns [256m, 256m+256)) at TMEM columns [128m, 128m+128)

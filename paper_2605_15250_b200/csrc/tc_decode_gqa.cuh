@@ -57,6 +57,7 @@ struct GqaSmem {
     static constexpr int kTotal = kTileBytes + kNumBars * 8 + 16;
     static_assert(kMergeBytes >= (kThreads + 4) * 4, "plan scratch must fit in the merge buffer");
     static_assert(kTotal <= 232448, "shared memory budget of one CTA");
+    static_assert(OneCtaPerSM<kTotal>::value, "");
 };
 
 // TMEM columns (all 512 are used, so one CTA per SM)

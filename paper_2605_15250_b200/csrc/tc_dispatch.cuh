@@ -13,6 +13,13 @@
 
 namespace gqla {
 
+// Status word of the calls whose C signature has none (gqla_absorb_q, gqla_up_proj, gqla_expand_cache,
+// gqla_append_expand, gqla_combine_up_proj): registered once per process with gqla_set_status_word.
+inline int32_t*& projection_status_word() {
+    static int32_t* word = nullptr;
+    return word;
+}
+
 inline bool stride_ok(int64_t elems) { return (elems * 2) % 16 == 0; }
 inline int next_pow2(int x) {
     int p = 1;
@@ -102,7 +109,7 @@ inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t
     if (d.r_kv == 64 * tc::ExpandSmem::kKBlocks && d.g % 2 == 0 && (N + 255) / 256 * 2 <= 0x7fffffffLL) {
         tc::ExpandParams ep{};
         ep.n_rows = N; ep.g = d.g; ep.r_kv = d.r_kv; ep.d_r = d.d_r;
-        ep.k_c = k_c; ep.v = v; ep.cache = cache; ep.k_r = k_r; ep.cache_stride = cache_row_stride; ep.status = nullptr;
+        ep.k_c = k_c; ep.v = v; ep.cache = cache; ep.k_r = k_r; ep.cache_stride = cache_row_stride; ep.status = projection_status_word();
         auto kern = tc::expand_tc_kernel;
         static bool attr_set[64] = {};
         int dev = 0;
@@ -132,7 +139,7 @@ inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t
     p.m_total = N;
     p.h_q = d.h_q; p.g = d.g; p.hpg = d.h_q / d.g; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
     p.out0 = k_c; p.out1 = v; p.aux_in = cache; p.aux_out = k_r; p.aux_stride = cache_row_stride;
-    p.status = nullptr;
+    p.status = projection_status_word();
     // 128 x 256 output tiles (two adjacent groups) when g is even: the 128-row latent tile is then re-read
     // through L2 by g CTAs instead of 2g
     cudaError_t e = (d.g % 2 == 0)
@@ -171,7 +178,7 @@ inline gqla_status tc_absorb_q(const gqla_dims& d, gqla_dtype dtype, int32_t B, 
     p.k_blocks = d.d_h / 64;
     p.m_total = positions;
     p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpb = hpb; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
-    p.out0 = q_hat; p.aux_in = q_r;
+    p.out0 = q_hat; p.aux_in = q_r; p.status = projection_status_word();
     cudaError_t e = tc::gemm_launch<tc::kGemmAbsorbQ, 256, false>(
         p, tmA, tmB, tmB, dim3((unsigned)m_tiles, (unsigned)d.g, (unsigned)(d.r_kv / 256)), st);
     return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
@@ -197,7 +204,7 @@ inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, i
     p.k_blocks = d.r_kv / 64;
     p.m_total = positions;
     p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpb = hpb; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
-    p.out0 = o;
+    p.out0 = o; p.status = projection_status_word();
     cudaError_t e =
         tc::gemm_launch<tc::kGemmUpProj, 128, true>(p, tmA, tmB, tmB, dim3((unsigned)m_tiles, (unsigned)d.g, 1), st);
     return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
@@ -226,7 +233,7 @@ inline gqla_status tc_append_expand(const gqla_dims& d, gqla_dtype dtype, int32_
     p.B = B; p.s_q = s_q; p.g = d.g; p.r_kv = d.r_kv; p.d_r = d.d_r;
     p.cache = (const __nv_bfloat16*)cache; p.cache_stride = cache_row_stride;
     p.seq_start = seq_start; p.seqlens = seqlens;
-    p.k_c = (__nv_bfloat16*)k_c; p.v = (__nv_bfloat16*)v; p.k_r = (__nv_bfloat16*)k_r; p.status = nullptr;
+    p.k_c = (__nv_bfloat16*)k_c; p.v = (__nv_bfloat16*)v; p.k_r = (__nv_bfloat16*)k_r; p.status = projection_status_word();
     auto kern = tc::append_expand_tc_kernel;
     static bool attr_set[64] = {};
     int dev = 0;
@@ -262,7 +269,7 @@ inline gqla_status tc_combine_up_proj(const gqla_dims& d, gqla_dtype dtype, int3
     }
     tc::CombineUpParams p{};
     p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpb = hpb; p.r_kv = d.r_kv;
-    p.positions = positions; p.o_part = o_part; p.lse_part = lse_part; p.out = o; p.lse = lse; p.status = nullptr;
+    p.positions = positions; p.o_part = o_part; p.lse_part = lse_part; p.out = o; p.lse = lse; p.status = projection_status_word();
     auto kern = tc::combine_up_tc_kernel;
     static bool attr_set[64] = {};
     int dev = 0;

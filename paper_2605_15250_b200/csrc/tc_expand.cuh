@@ -40,6 +40,7 @@ struct ExpandSmem {
     static constexpr int kThreads = 192;
     static constexpr int kTotal = 1024 + kTileBytes + kNumBars * 8 + 16;
     static_assert(kTotal <= 232448, "shared memory budget of one CTA");
+    static_assert(OneCtaPerSM<kTotal>::value, "");
 };
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(ExpandSmem::kThreads, 1)

@@ -33,6 +33,7 @@ struct GemmSmem {
     static constexpr int kBBytes = BN * 128;   // K-major: BN rows x 64 k;  MN-major: (BN/64) boxes of 64 k-rows x 64 n
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kTotal = kStages * kStageBytes + 1024 /*align slack*/ + 256 /*barriers*/;
+    static_assert(OneCtaPerSM<kTotal>::value, "");
 };
 
 template <int MODE, int BN, bool B_MN>

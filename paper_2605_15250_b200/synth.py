@@ -100,8 +100,13 @@ def make_seqlens(w: Workload) -> np.ndarray:
     return np.full((w.batch,), w.seqlen, dtype=np.int32)
 
 
-def make_inputs(w: Workload, seqlens: np.ndarray | None = None, q_gain: float = 1.0) -> dict:
+def make_inputs(w: Workload, seqlens: np.ndarray | None = None, q_gain: float = 1.0,
+                cache_device: torch.device | str | None = None) -> dict:
     """CPU tensors of one decode step.
+
+    cache_device: draw the cache (by far the largest tensor) on that device with torch's seeded
+    generator instead of on the CPU -- same distribution, different bits; for timing runs of the
+    multi-gigabyte workloads, never for a comparison with the CPU checker.
 
     q_gain multiplies both query parts: 1.0 gives unit-variance scores (flat
     softmax, outputs ~1/sqrt(T)); 4.0 gives a peaked softmax whose outputs are
@@ -119,15 +124,33 @@ def make_inputs(w: Workload, seqlens: np.ndarray | None = None, q_gain: float = 
     seq_start[1:] = np.cumsum(seqlens.astype(np.int64))[:-1]
     n_rows = int(seqlens.astype(np.int64).sum())
     B, s, h = w.batch, w.s_q, w.h_q
+    if cache_device is not None:
+        gen = torch.Generator(device=cache_device)
+        gen.manual_seed(w.seed)
+        cache = torch.empty((max(n_rows, 1), w.d_abs), dtype=_torch_dtype(w.dtype), device=cache_device)
+        step = 1 << 18
+        for lo in range(0, cache.shape[0], step):
+            hi = min(lo + step, cache.shape[0])
+            cache[lo:hi] = torch.randn((hi - lo, w.d_abs), generator=gen, device=cache_device, dtype=torch.float32)
+        cache = cache[:n_rows]
+    else:
+        cache = _normal(w.seed, _T_CACHE, (max(n_rows, 1), w.d_abs), w.dtype)[:n_rows]
     return {
         "q_c": _normal(w.seed, _T_QC, (B, s, h, w.d_h), w.dtype, q_gain),
         "q_r": _normal(w.seed, _T_QR, (B, s, h, w.d_r), w.dtype, q_gain),
         "w_uk": _normal(w.seed, _T_WUK, (w.g, w.r_kv, w.d_h), w.dtype, 1.0 / float(np.sqrt(w.r_kv))),
         "w_uv": _normal(w.seed, _T_WUV, (w.g, w.r_kv, w.d_h), w.dtype, 1.0 / float(np.sqrt(w.r_kv))),
-        "cache": _normal(w.seed, _T_CACHE, (max(n_rows, 1), w.d_abs), w.dtype)[:n_rows],
+        "cache": cache,
         "seq_start": torch.from_numpy(seq_start),
         "seqlens": torch.from_numpy(seqlens.copy()),
     }
+
+
+def make_queries(w: Workload, q_gain: float = 1.0) -> dict:
+    """The two query tensors of make_inputs alone (same streams, same bits)."""
+    B, s, h = w.batch, w.s_q, w.h_q
+    return {"q_c": _normal(w.seed, _T_QC, (B, s, h, w.d_h), w.dtype, q_gain),
+            "q_r": _normal(w.seed, _T_QR, (B, s, h, w.d_r), w.dtype, q_gain)}
 
 
 def to_paged(t: torch.Tensor, seq_start, seqlens, page_size: int, seed: int, fill: float = 3.0, spare_pages: int = 3):

@@ -154,3 +154,16 @@ def test_policy_switch_and_kernel_names():
     assert B.get_policy() == B.POLICY_AUTO
     # fp32 storage is never on the tensor-core kernels
     assert B.kernel_for(d, torch.float32, 1, "gqa") == "generic"
+
+
+def test_status_word_registration_round_trips():
+    """The process-wide status word of the projection calls: what is registered is what the library
+    hands to its kernels, and NULL unregisters.  Nothing is launched and the address is never dereferenced."""
+    L = B.lib()
+    assert B.get_status_word() == 0
+    L.gqla_set_status_word(ctypes.c_void_p(0x7000))
+    try:
+        assert B.get_status_word() == 0x7000
+    finally:
+        L.gqla_set_status_word(None)
+    assert B.get_status_word() == 0

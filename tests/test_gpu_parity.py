@@ -491,6 +491,21 @@ def test_determinism_run_to_run():
     a1 = dec.absorb_step(qc, qr, 4).clone()
     a2 = dec.absorb_step(qc, qr, 4).clone()
     assert torch.equal(a1, a2)
+    # the GQA kernel, and both kernels under the balanced plan (no global counters: the cut points are a pure
+    # function of the lengths, so the reduction order is fixed there too)
+    dec.expand_cache()
+    q = torch.cat([x["q_c"], x["q_r"]], -1).contiguous().cuda()
+    for S in (4, 1, -3):
+        g1 = dec.gqa_step(q, S).clone()
+        g2 = dec.gqa_step(q, S).clone()
+        assert torch.equal(g1, g2), S
+    b1 = dec.absorb_step(qc, qr, -3).clone()
+    b2 = dec.absorb_step(qc, qr, -3).clone()
+    assert torch.equal(b1, b2)
+    f1 = dec.absorb_step(qc, qr, 1).clone()
+    f2 = dec.absorb_step(qc, qr, 1).clone()
+    assert torch.equal(f1, f2)
+    dec.check_status()
 
 
 # ------------------------------------------------------------------ workloads C1-C4 at full size
@@ -500,16 +515,18 @@ def test_c1_full_absorb():
     """Config 1: h_q=128, g=8, B=64, T=4096, s_q=1, absorb path (as the benchmark launches it)."""
     from tests.parity_util import end_to_end
     end_to_end(synth.WORKLOADS["C1"], None, 1, paths=("absorb",))
+    # the same launch on the peaked inputs (O(1) outputs: the relative term of the bound decides), every sequence
+    end_to_end(synth.WORKLOADS["C1"], None, 1, q_gain=4.0, paths=("absorb",))
 
 
 def test_c2_full_gqa_mtp():
-    """Config 2: same weights and latent, expanded cache, s_q=2 causal.  The oracle runs a sample
-    of sequences (all heads, both draft positions)."""
+    """Config 2: same weights and latent, expanded cache, s_q=2 causal."""
     from tests.parity_util import end_to_end
     end_to_end(synth.WORKLOADS["C2"], None, 1, sample_seqs=(0, 17, 63), paths=("gqa",))
     end_to_end(synth.WORKLOADS["C2"], None, 1, q_gain=4.0, sample_seqs=(5,), paths=("gqa", "absorb"))
-    # the launch configuration bench.py times: balanced plan, two slots per sequence
-    end_to_end(synth.WORKLOADS["C2"], None, -2, q_gain=4.0, sample_seqs=(3, 4, 60), paths=("gqa",))
+    # the launch configuration bench.py times (balanced plan, two slots per sequence), every sequence, all
+    # heads, both draft positions, on the peaked inputs
+    end_to_end(synth.WORKLOADS["C2"], None, -2, q_gain=4.0, paths=("gqa",))
 
 
 @pytest.mark.parametrize("s_q", [1, 2])

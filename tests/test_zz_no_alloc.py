@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import gqla_oracle as O
 from paper_2605_15250_b200 import binding as B
 from paper_2605_15250_b200 import build as gbuild
 from paper_2605_15250_b200 import synth
@@ -54,6 +55,8 @@ def test_noalloc_matches_caller_buffer_path_twice_in_a_row():
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     q_first = torch.cat([x["q_c"], x["q_r"]], -1).contiguous().cuda()
     q_second = (-0.5 * q_first.float()).flip(2).contiguous().to(torch.bfloat16)
+    od = O.Dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)
+    f_kc, f_v, f_kr = synth.to_f64(k_c), synth.to_f64(v), synth.to_f64(k_r)
 
     # second call: other queries and another split count, so stale partials of the first call would show
     for q, S in ((q_first, 3), (q_second, 2)):
@@ -78,3 +81,53 @@ def test_noalloc_matches_caller_buffer_path_twice_in_a_row():
         assert np.array_equal(np.isneginf(gl), np.isneginf(wl))
         fin = ~np.isneginf(wl)
         assert np.abs(gl[fin] - wl[fin]).max() <= REL * np.abs(wl[fin]).max() + ABS
+        # and against the CPU checker on the very planes the kernel read
+        o_ref, l_ref = O.decode_gqa(od, synth.to_f64(q), f_kc, f_v, f_kr, x["seq_start"].numpy(), x["seqlens"].numpy(),
+                                    w.s_q, w.scale)
+        assert np.abs(got - o_ref).max() <= REL * np.abs(o_ref).max() + ABS
+        assert np.array_equal(np.isneginf(gl), np.isneginf(l_ref))
+        assert np.abs(gl[fin] - l_ref[fin]).max() <= REL * np.abs(l_ref[fin]).max() + ABS
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype,policy", [("f32", "auto"), ("bf16", "generic")])
+def test_noalloc_other_kernels_and_types(dtype, policy):
+    """The fp32 storage type and the generic kernel policy go through the same built-in array; an empty
+    call first, as a host would make at start-up to have the array placed."""
+    gbuild.build()
+    assert torch.cuda.is_available()
+    B.lib()
+    B.set_policy(B.POLICY_GENERIC if policy == "generic" else B.POLICY_AUTO)
+    try:
+        w = synth.Workload("noalloc2", 8, 2, 16, 32, 8, batch=3, s_q=2, dtype=dtype, seed=0x2B)
+        seqlens = np.array([70, 0, 131], dtype=np.int32)
+        x = synth.make_inputs(w, seqlens=seqlens, q_gain=2.0)
+        dims = B.make_dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)
+        od = O.Dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)
+        f = {k: synth.to_f64(t) for k, t in x.items() if k not in ("seq_start", "seqlens")}
+        kc_ref, v_ref, kr_ref = O.expand_cache(od, f["cache"], f["w_uk"], f["w_uv"])
+        td = torch.bfloat16 if dtype == "bf16" else torch.float32
+        k_c, v, k_r = (torch.from_numpy(np.ascontiguousarray(a)).to(td).cuda() for a in (kc_ref, v_ref, kr_ref))
+        q = torch.cat([x["q_c"], x["q_r"]], -1).contiguous().cuda()
+        ss, sl = x["seq_start"].cuda(), x["seqlens"].cuda()
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out = torch.full((w.batch, w.s_q, w.h_q, w.d_h), float("nan"), dtype=td, device="cuda")
+        lse = torch.full((w.batch, w.s_q, w.h_q), float("nan"), dtype=torch.float32, device="cuda")
+        # warm-up: an empty batch (B = 0) performs the address query and launches nothing
+        B.gqla_decode_gqa_noalloc(dims, q[:0], k_c, v, k_r, ss[:0], sl[:0], w.scale, 1, out, None, status)
+        assert torch.isnan(out.float()).all()
+        o_ref, l_ref = O.decode_gqa(od, synth.to_f64(q), synth.to_f64(k_c), synth.to_f64(v), synth.to_f64(k_r),
+                                    x["seq_start"].numpy(), x["seqlens"].numpy(), w.s_q, w.scale)
+        for S in (2, 1):
+            out.fill_(float("nan")); lse.fill_(float("nan"))
+            B.gqla_decode_gqa_noalloc(dims, q, k_c, v, k_r, ss, sl, w.scale, S, out, lse, status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            got, gl = out.float().cpu().numpy(), lse.cpu().numpy()
+            assert not np.isnan(got).any()
+            assert np.abs(got - o_ref).max() <= REL * np.abs(o_ref).max() + ABS
+            assert np.array_equal(np.isneginf(gl), np.isneginf(l_ref))
+            fin = ~np.isneginf(l_ref)
+            assert np.abs(gl[fin] - l_ref[fin]).max() <= REL * np.abs(l_ref[fin]).max() + ABS
+    finally:
+        B.set_policy(B.POLICY_AUTO)
