@@ -16,6 +16,11 @@ Notation (paper Sec. 3.1 "Group-Query Latent Attention"):
     c     latent c^KV  [.., r_kv]    k_r   shared RoPE key k^R [.., d_r]
     W_UK, W_UV  stored as [g, r_kv, d_h]; W[j, r, d] is entry (d, r) of the
                 paper's group-j slice  W_j in R^{d_h x r_kv}.
+    d_v   value head dim d_h^V.  Sec. 3.1 gives W^UV the shape of W^UK (d_v = d_h); the
+          MLA -> GQLA factorisation of Sec. 3.2 carries a separate one
+          (W~^UKV in R^{g (d_h + d_h^V) x r_kv}).  It is read off the arrays: W_UV is
+          [g, r_kv, d_v], V is [N, g, d_v], outputs are d_v wide; Dims.d_v (0 = d_h)
+          only enters the cache-size accounting.
 
 Every function is pinned by tests/test_oracle_pins.py to something other than
 itself (brute force over python loops, closed forms, invariants, the two-path
@@ -45,6 +50,11 @@ class Dims:
     d_h: int
     r_kv: int
     d_r: int
+    d_v: int = 0  # value head dim d_h^V of Sec. 3.2; 0 means d_h (Sec. 3.1)
+
+    @property
+    def dv(self) -> int:
+        return self.d_v if self.d_v > 0 else self.d_h
 
     @property
     def hpg(self) -> int:
@@ -148,12 +158,12 @@ def absorb_q(dims: Dims, q_c: np.ndarray, q_r: np.ndarray, w_uk: np.ndarray) -> 
 def expand_cache(dims: Dims, cache: np.ndarray, w_uk: np.ndarray, w_uv: np.ndarray):
     """Sec. 3.1: k^C = W^UK c^KV, v^C = W^UV c^KV per group; k^R carried over.
 
-    cache [N, r_kv + d_r] -> K_C [N, g, d_h], V [N, g, d_h], k_R [N, d_r].
+    cache [N, r_kv + d_r] -> K_C [N, g, d_h], V [N, g, d_v], k_R [N, d_r]  (w_uv is [g, r_kv, d_v]).
     """
     c = cache[:, : dims.r_kv].astype(np.float64)
     N = c.shape[0]
     k_c = np.zeros((N, dims.g, dims.d_h), dtype=np.float64)
-    v = np.zeros((N, dims.g, dims.d_h), dtype=np.float64)
+    v = np.zeros((N, dims.g, w_uv.shape[2]), dtype=np.float64)
     for j in range(dims.g):
         k_c[:, j, :] = c @ w_uk[j].astype(np.float64)  # sum_r W[j,r,d] c[r]
         v[:, j, :] = c @ w_uv[j].astype(np.float64)
@@ -162,9 +172,9 @@ def expand_cache(dims: Dims, cache: np.ndarray, w_uk: np.ndarray, w_uv: np.ndarr
 
 
 def up_proj(dims: Dims, o_hat: np.ndarray, w_uv: np.ndarray) -> np.ndarray:
-    """Eq. (mqa): o_i = W^UV_{j(i)} o_hat_i.  o_hat [B, s_q, h_q, r_kv] -> [B, s_q, h_q, d_h]."""
+    """Eq. (mqa): o_i = W^UV_{j(i)} o_hat_i.  o_hat [B, s_q, h_q, r_kv] -> [B, s_q, h_q, d_v]."""
     B, s_q, h_q, _ = o_hat.shape
-    out = np.zeros((B, s_q, h_q, dims.d_h), dtype=np.float64)
+    out = np.zeros((B, s_q, h_q, w_uv.shape[2]), dtype=np.float64)
     for i in range(h_q):
         j = group_of_head(dims, i)
         out[:, :, i, :] = o_hat[:, :, i, :].astype(np.float64) @ w_uv[j].astype(np.float64)
@@ -253,7 +263,7 @@ def decode_absorb_partials(dims: Dims, q_hat, cache, seq_start, seqlens, s_q, sc
 def decode_gqa_partials(dims: Dims, q, k_c, v, k_r, seq_start, seqlens, s_q, scale, num_splits, plans=None):
     """Eq. (mha): head i attends k_{s,i} = [k^C_{s,j(i)} ; k^R_s] with values v^C_{s,j(i)}.
 
-    q [B, s_q, h_q, d_h+d_r]; k_c, v [N, g, d_h]; k_r [N, d_r]."""
+    q [B, s_q, h_q, d_h+d_r]; k_c [N, g, d_h]; v [N, g, d_v]; k_r [N, d_r]."""
     B = q.shape[0]
     q64 = q.astype(np.float64)
     hpg = dims.hpg
@@ -277,7 +287,7 @@ def decode_gqa_partials(dims: Dims, q, k_c, v, k_r, seq_start, seqlens, s_q, sca
     def q_rows_of(b, p):
         return [(slice(j * hpg, (j + 1) * hpg), q64[b, p, j * hpg:(j + 1) * hpg]) for j in range(dims.g)]
 
-    return _decode(dims, q_rows_of, K_of, V_of, dims.d_h, B, s_q, seq_start, seqlens, scale, num_splits, plans)
+    return _decode(dims, q_rows_of, K_of, V_of, v.shape[2], B, s_q, seq_start, seqlens, scale, num_splits, plans)
 
 
 def unpage(paged: np.ndarray, block_table: np.ndarray, page_size: int, seqlens: np.ndarray):
@@ -354,11 +364,12 @@ def brute_force_path(dims, q_c, q_r, w_uk, w_uv, cache, seq_start, seqlens, s_q,
     product at a time, and does a two-pass softmax with math.exp."""
     B = q_c.shape[0]
     h_q, g, d_h, r, d_r = dims.h_q, dims.g, dims.d_h, dims.r_kv, dims.d_r
+    d_v = w_uv.shape[2]
     reps = h_q // g
     # repeat(W, h_q/g): head i uses slice i of the group-wise replicated stack
     w_uk_hat = [w_uk[jj] for jj in range(g) for _ in range(reps)]
     w_uv_hat = [w_uv[jj] for jj in range(g) for _ in range(reps)]
-    out = np.zeros((B, s_q, h_q, d_h))
+    out = np.zeros((B, s_q, h_q, d_v))
     for b in range(B):
         T = int(seqlens[b])
         s0 = int(seq_start[b])
@@ -372,7 +383,7 @@ def brute_force_path(dims, q_c, q_r, w_uk, w_uv, cache, seq_start, seqlens, s_q,
                         continue
                     row = cache[s0 + s]
                     kc = [sum(float(Wk[rr, d]) * float(row[rr]) for rr in range(r)) for d in range(d_h)]
-                    vc = [sum(float(Wv[rr, d]) * float(row[rr]) for rr in range(r)) for d in range(d_h)]
+                    vc = [sum(float(Wv[rr, d]) * float(row[rr]) for rr in range(r)) for d in range(d_v)]
                     dot = sum(float(q_c[b, p, i, d]) * kc[d] for d in range(d_h))
                     dot += sum(float(q_r[b, p, i, d]) * float(row[r + d]) for d in range(d_r))
                     xs.append(scale * dot)
@@ -382,7 +393,7 @@ def brute_force_path(dims, q_c, q_r, w_uk, w_uv, cache, seq_start, seqlens, s_q,
                 m = max(xs)
                 es = [math.exp(x - m) for x in xs]
                 Z = sum(es)
-                for d in range(d_h):
+                for d in range(d_v):
                     out[b, p, i, d] = sum(es[n] * vs[n][d] for n in range(len(xs))) / Z
     return out
 
@@ -398,8 +409,8 @@ def mqa_cache_elems(dims: Dims) -> int:
 
 
 def gqa_cache_elems(dims: Dims) -> int:
-    """N^tok_GQA = 2 g d_h + d_h^R."""
-    return 2 * dims.g * dims.d_h + dims.d_r
+    """N^tok_GQA = 2 g d_h + d_h^R; with a separate value dim (Sec. 3.2) g (d_h + d_h^V) + d_h^R."""
+    return dims.g * (dims.d_h + dims.dv) + dims.d_r
 
 
 def mqa_bytes(dims: Dims, L: int, bytes_per_elem: int = 2) -> int:
@@ -418,8 +429,8 @@ def mqa_flops(dims: Dims, L: int, s_q: int) -> int:
 
 
 def gqa_flops(dims: Dims, L: int, s_q: int) -> int:
-    """F_GQA = 2 L h_q s_q (2 d_h + d_h^R)."""
-    return 2 * L * dims.h_q * s_q * (2 * dims.d_h + dims.d_r)
+    """F_GQA = 2 L h_q s_q (2 d_h + d_h^R); with a separate value dim d_h + d_h^V + d_h^R per (head, key)."""
+    return 2 * L * dims.h_q * s_q * (dims.d_h + dims.dv + dims.d_r)
 
 
 def roofline_step(flops: float, nbytes: float, peak_flops: float, bw: float):

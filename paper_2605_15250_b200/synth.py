@@ -33,6 +33,11 @@ class Workload:
     seed: int
     seqlen: int = 0  # fixed length, or
     seqlen_range: tuple[int, int] | None = None  # inclusive uniform range
+    d_v: int = 0  # value head dim d_h^V of the MLA -> GQLA factorisation (Sec. 3.2); 0 = d_h (Sec. 3.1)
+
+    @property
+    def dv(self) -> int:
+        return self.d_v if self.d_v > 0 else self.d_h
 
     @property
     def scale(self) -> float:
@@ -112,7 +117,7 @@ def make_inputs(w: Workload, seqlens: np.ndarray | None = None, q_gain: float = 
     softmax, outputs ~1/sqrt(T)); 4.0 gives a peaked softmax whose outputs are
     O(1), which is the more discriminating parity case.
 
-    Returns q_c [B,s_q,h_q,d_h], q_r [B,s_q,h_q,d_r], w_uk/w_uv [g,r_kv,d_h],
+    Returns q_c [B,s_q,h_q,d_h], q_r [B,s_q,h_q,d_r], w_uk [g,r_kv,d_h], w_uv [g,r_kv,d_v],
     cache [N, r_kv+d_r] (sequence b owns rows seq_start[b] .. +seqlens[b]),
     seq_start int64 [B], seqlens int32 [B].
     """
@@ -139,7 +144,7 @@ def make_inputs(w: Workload, seqlens: np.ndarray | None = None, q_gain: float = 
         "q_c": _normal(w.seed, _T_QC, (B, s, h, w.d_h), w.dtype, q_gain),
         "q_r": _normal(w.seed, _T_QR, (B, s, h, w.d_r), w.dtype, q_gain),
         "w_uk": _normal(w.seed, _T_WUK, (w.g, w.r_kv, w.d_h), w.dtype, 1.0 / float(np.sqrt(w.r_kv))),
-        "w_uv": _normal(w.seed, _T_WUV, (w.g, w.r_kv, w.d_h), w.dtype, 1.0 / float(np.sqrt(w.r_kv))),
+        "w_uv": _normal(w.seed, _T_WUV, (w.g, w.r_kv, w.dv), w.dtype, 1.0 / float(np.sqrt(w.r_kv))),
         "cache": cache,
         "seq_start": torch.from_numpy(seq_start),
         "seqlens": torch.from_numpy(seqlens.copy()),

@@ -15,10 +15,10 @@ from paper_2605_15250_b200 import synth
 CANON = O.Dims(128, 8, 128, 512, 64)
 
 
-def _tiny(h_q, g, d_h, r_kv, d_r, B, T, s_q, seed, dtype="f32", seqlens=None):
-    w = synth.Workload("t", h_q, g, d_h, r_kv, d_r, batch=B, s_q=s_q, dtype=dtype, seed=seed, seqlen=T)
+def _tiny(h_q, g, d_h, r_kv, d_r, B, T, s_q, seed, dtype="f32", seqlens=None, d_v=0):
+    w = synth.Workload("t", h_q, g, d_h, r_kv, d_r, batch=B, s_q=s_q, dtype=dtype, seed=seed, seqlen=T, d_v=d_v)
     x = synth.make_inputs(w, seqlens=seqlens)
-    d = O.Dims(h_q, g, d_h, r_kv, d_r)
+    d = O.Dims(h_q, g, d_h, r_kv, d_r, d_v)
     f = {k: synth.to_f64(v) for k, v in x.items() if k not in ("seq_start", "seqlens")}
     return w, d, f, x["seq_start"].numpy(), x["seqlens"].numpy()
 
@@ -200,6 +200,33 @@ def test_random_tiny_three_way_agreement(h_q, g, s_q):
     ref = max(np.abs(bf).max(), 1e-30)
     assert np.abs(a - bf).max() <= 1e-12 * ref
     assert np.abs(gq - bf).max() <= 1e-12 * ref
+
+
+@pytest.mark.parametrize("d_h,d_v", [(4, 6), (6, 4), (3, 8)])
+def test_separate_value_head_dim_three_way_agreement(d_h, d_v):
+    """Sec. 3.2 "From MLA to GQLA": W~^UKV in R^{g (d_h + d_h^V) x r_kv} carries a value head dim of its own.
+    Both paths against the python-loop brute force with d_v != d_h, plus the contractions against einsum."""
+    seqlens = np.array([9, 2, 1], dtype=np.int32)
+    w, d, f, ss, sl = _tiny(6, 2, d_h, 5, 2, B=3, T=0, s_q=2, seed=40 + d_h, seqlens=seqlens, d_v=d_v)
+    assert f["w_uv"].shape == (2, 5, d_v) and f["w_uk"].shape == (2, 5, d_h)
+    a, gq = _paths(d, f, ss, sl, 2, 0.37)
+    bf = O.brute_force_path(d, f["q_c"], f["q_r"], f["w_uk"], f["w_uv"], f["cache"], ss, sl, 2, 0.37)
+    assert a.shape == gq.shape == bf.shape == (3, 2, 6, d_v)
+    ref = np.abs(bf).max()
+    assert np.abs(a - bf).max() <= 1e-12 * ref and np.abs(gq - bf).max() <= 1e-12 * ref
+    kc, v, kr = O.expand_cache(d, f["cache"], f["w_uk"], f["w_uv"])
+    assert kc.shape[2] == d_h and v.shape[2] == d_v
+    c = torch.from_numpy(f["cache"])
+    np.testing.assert_allclose(v, torch.einsum("nr,grd->ngd", c[:, :5], torch.from_numpy(f["w_uv"])).numpy(),
+                               rtol=1e-13, atol=1e-13)
+    rep_v = torch.from_numpy(np.repeat(f["w_uv"], d.hpg, axis=0))
+    oh = np.random.default_rng(1).standard_normal((3, 2, 6, 5))
+    np.testing.assert_allclose(O.up_proj(d, oh, f["w_uv"]),
+                               torch.einsum("bphr,hrd->bphd", torch.from_numpy(oh), rep_v).numpy(), rtol=1e-13, atol=1e-13)
+    # cache elements per token: g (d_h + d_h^V) + d_h^R; equal value dim gives back 2 g d_h + d_h^R
+    assert O.gqa_cache_elems(d) == 2 * (d_h + d_v) + 2
+    assert O.gqa_cache_elems(O.Dims(128, 8, 128, 512, 64)) == 2112 == O.gqa_cache_elems(O.Dims(128, 8, 128, 512, 64, 128))
+    assert O.gqa_flops(O.Dims(128, 8, 128, 512, 64, 128), 8192, 2) == O.gqa_flops(CANON, 8192, 2)
 
 
 def test_two_paths_equal_at_larger_shapes():
