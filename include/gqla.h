@@ -220,6 +220,26 @@ gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_spl
 gqla_status gqla_up_proj(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int32_t s_q, const void* o_hat,
                          const void* w_uv, void* o, void* stream);
 
+/* The three calls a value head dimension of its own touches.  Sec. 3.1 gives W^UV the shape of W^UK, and
+ * gqla_dims says so (d_v == d_h); the MLA -> GQLA factorisation of Sec. 3.2 ("From MLA to GQLA") carries a
+ * separate d_h^V:  W~^UKV in R^{g (d_h + d_h^V) x r_kv}  (e.g. d_h = 192, d_h^V = 256).  These variants
+ * take it as `d_v` (>= 1); everything else is as for the call without the suffix:
+ *   gqla_expand_cache_dv   w_uv [g, r_kv, d_v]  ->  v [N, g, d_v]        (k_c stays [N, g, d_h])
+ *   gqla_decode_gqa_dv     v [N, g, d_v]        ->  o_part [B, S, s_q, h_q, d_v]
+ *   gqla_up_proj_dv        w_uv [g, r_kv, d_v]  ->  o [B, s_q, h_q, d_v]
+ * The absorb path needs nothing else (its attention runs in the latent space), and gqla_combine_splits
+ * takes the output width as d_out already.  With d_v == d_h they are the calls without the suffix; other
+ * values run on the generic kernels (d_v <= 512 for gqla_decode_gqa_dv). */
+gqla_status gqla_expand_cache_dv(const gqla_dims* dims, int32_t d_v, gqla_dtype dtype, int64_t N, const void* cache,
+                                 int64_t cache_row_stride, const void* w_uk, const void* w_uv, void* k_c, void* v,
+                                 void* k_r, void* stream);
+gqla_status gqla_decode_gqa_dv(const gqla_dims* dims, int32_t d_v, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                               int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
+                               int64_t k_r_row_stride, int64_t n_rows, const int64_t* seq_start, const int32_t* seqlens,
+                               float* o_part, float* lse_part, int32_t* status_word, void* stream);
+gqla_status gqla_up_proj_dv(const gqla_dims* dims, int32_t d_v, gqla_dtype dtype, int32_t B, int32_t s_q,
+                            const void* o_hat, const void* w_uv, void* o, void* stream);
+
 /* gqla_combine_splits followed by gqla_up_proj in one kernel (Eq. (mqa), line 6, applied to the merged
  * latent output): the merged o_hat never goes to memory.  Same arguments as the two calls:
  *   o_part [B, S, s_q, h_q, r_kv] fp32, lse_part [B, S, s_q, h_q] fp32, w_uv [g, r_kv, d_h]

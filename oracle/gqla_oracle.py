@@ -22,7 +22,7 @@ Notation (paper Sec. 3.1 "Group-Query Latent Attention"):
           [g, r_kv, d_v], V is [N, g, d_v], outputs are d_v wide; Dims.d_v (0 = d_h)
           only enters the cache-size accounting.
 
-Every function is pinned by tests/test_oracle_pins.py to something other than
+Every function is pinned by tests/test_oracle_pins.py (the FP8 ones by tests/test_oracle_fp8_pins.py) to something other than
 itself (brute force over python loops, closed forms, invariants, the two-path
 equivalence the paper states, the printed Roofline table).  Nothing here is
 "parity unpinned".
@@ -334,6 +334,90 @@ def decode_gqa(dims, q, k_c, v, k_r, seq_start, seqlens, s_q, scale):
     """Whole-sequence GQA-path attention: o [B, s_q, h_q, d_h], lse."""
     o, l = decode_gqa_partials(dims, q, k_c, v, k_r, seq_start, seqlens, s_q, scale, 1)
     return o[:, 0], l[:, 0]
+
+
+# --------------------------------------------------------------------------
+# FP8 (E4M3) cache: the paper leaves KV-cache quantisation out of its model (Limitations, item (i)); the
+# format, the scales and the rounding are this library's reading (element type: the 8-bit float with 4
+# exponent bits (bias 7), 3 mantissa bits, no infinities, largest finite value 448, NaN = S.1111.111).
+# --------------------------------------------------------------------------
+
+E4M3_MAX = 448.0
+
+
+def e4m3_decode(codes: np.ndarray) -> np.ndarray:
+    """Value of every 8-bit code, written out from the format's definition:
+    sign s, exponent field e (4 bits), mantissa field m (3 bits);
+    e = 0: (-1)^s 2^-6 (m/8)   (subnormal);   e > 0: (-1)^s 2^(e-7) (1 + m/8);   e = 15, m = 7: NaN."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    sign = np.where((c >> 7) & 1, -1.0, 1.0)
+    e = (c >> 3) & 15
+    m = c & 7
+    val = np.where(e == 0, 2.0 ** -6 * (m / 8.0), 2.0 ** (e - 7.0) * (1.0 + m / 8.0))
+    val = np.where((e == 15) & (m == 7), np.nan, val)
+    return sign * val
+
+
+def e4m3_encode(y: np.ndarray) -> np.ndarray:
+    """fp32 -> code: round to the nearest representable value, ties to the code with an even mantissa
+    field, magnitudes beyond 448 saturate to 448 (no infinity exists), NaN -> 0x7F.
+    Brute statement: among the 127 non-negative finite values pick the closest one to |y|."""
+    y = np.asarray(y, dtype=np.float32).astype(np.float64)  # fp32 values are exact in fp64
+    grid = e4m3_decode(np.arange(127, dtype=np.uint8))  # codes 0..126: 0 .. 448, increasing
+    a = np.minimum(np.abs(y), E4M3_MAX)
+    hi = np.clip(np.searchsorted(grid, a, side="left"), 0, 126)  # first grid value >= a
+    lo = np.maximum(hi - 1, 0)
+    d_lo, d_hi = a - grid[lo], grid[hi] - a
+    pick_lo = (d_lo < d_hi) | ((d_lo == d_hi) & (lo % 2 == 0))
+    code = np.where(pick_lo, lo, hi).astype(np.int64)
+    code = np.where(np.signbit(y), code | 0x80, code)
+    code = np.where(np.isnan(y), 0x7F, code)
+    return code.astype(np.uint8)
+
+
+def quantize_cols_e4m3(x: np.ndarray, split: int, scale_a: float, scale_b: float) -> np.ndarray:
+    """Per-tensor-plane quantisation of a stored tensor [..., width]: columns < split carry scale_a, the
+    others scale_b;  code = encode( fp32(x) * fp32(1 / scale) ), every step rounded to fp32 (the decision
+    that picks an integer code is taken in fp32 on both sides of a comparison)."""
+    x32 = np.asarray(x, dtype=np.float32)
+    inv = np.empty(x32.shape[-1], dtype=np.float32)
+    inv[:split] = np.float32(1.0) / np.float32(scale_a)
+    inv[split:] = np.float32(1.0) / np.float32(scale_b)
+    return e4m3_encode(x32 * inv)
+
+
+def quantize_rows_e4m3(x: np.ndarray, split: int, pre_a: float, pre_b: float):
+    """Per-row quantisation of query rows [..., width]: y = fp32(x) * pre (pre_a on columns < split, pre_b
+    on the others: the cache planes' scales, folded into the query so that scores need no per-column
+    factor), s = max|y| / 448 (1 for an all-zero row), code = encode(y * fp32(1 / s)).  Returns (codes,
+    s as fp32 [...]).  All arithmetic in fp32."""
+    x32 = np.asarray(x, dtype=np.float32)
+    pre = np.empty(x32.shape[-1], dtype=np.float32)
+    pre[:split] = np.float32(pre_a)
+    pre[split:] = np.float32(pre_b)
+    y = x32 * pre
+    amax = np.abs(y).max(axis=-1)
+    s = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    inv = (np.float32(1.0) / s).astype(np.float32)
+    return e4m3_encode(y * inv[..., None]), s
+
+
+def decode_absorb_fp8_partials(dims: Dims, q8, q_scale, cache8, v_scale, seq_start, seqlens, s_q, scale, num_splits,
+                               plans=None):
+    """Eq. (mqa), lines 3-5, on an E4M3 latent cache.  Scores  x_s = scale * q_scale[row] * sum_c dec(q8)[c] dec(k8_s)[c],
+    values  v_s = v_scale * dec(cache8_s)[: r_kv].  The plain definition on the decoded numbers (fp64)."""
+    q = e4m3_decode(q8) * np.asarray(q_scale, dtype=np.float64)[..., None]
+    o, l = decode_absorb_partials(dims, q, e4m3_decode(cache8), seq_start, seqlens, s_q, scale, num_splits, plans)
+    return o * float(v_scale), l
+
+
+def decode_gqa_fp8_partials(dims: Dims, q8, q_scale, k_c8, v8, k_r8, v_scale, seq_start, seqlens, s_q, scale,
+                            num_splits, plans=None):
+    """Eq. (mha) on E4M3 planes K_C, V, k_R; same conventions as decode_absorb_fp8_partials."""
+    q = e4m3_decode(q8) * np.asarray(q_scale, dtype=np.float64)[..., None]
+    o, l = decode_gqa_partials(dims, q, e4m3_decode(k_c8), e4m3_decode(v8), e4m3_decode(k_r8), seq_start, seqlens, s_q,
+                               scale, num_splits, plans)
+    return o * float(v_scale), l
 
 
 # --------------------------------------------------------------------------

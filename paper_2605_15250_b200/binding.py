@@ -62,6 +62,12 @@ _PROTOTYPES = {
     "gqla_combine_up_proj": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                        c_void_p, c_void_p, c_void_p]),
     "gqla_up_proj": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_up_proj_dv": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_expand_cache_dv": (c_int32, [c_void_p, c_int32, c_int32, c_int64, c_void_p, c_int64, c_void_p, c_void_p,
+                                       c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_decode_gqa_dv": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
+                                     c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
+                                     c_void_p, c_void_p]),
     "gqla_split_plan": (c_int32, [c_int32, c_int32, c_void_p, c_void_p]),
     "gqla_visible_limit": (c_int32, [c_int32, c_int32, c_int32]),
     "gqla_balanced_plan": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p]),
@@ -306,6 +312,43 @@ def gqla_combine_up_proj(dims: GqlaDims, o_part: torch.Tensor, lse_part: torch.T
     B, S, s_q = o_part.shape[0], o_part.shape[1], o_part.shape[2]
     _check(lib().gqla_combine_up_proj(ctypes.byref(dims), _dtype_code(o), B, s_q, S, _ptr(o_part), _ptr(lse_part),
                                       _ptr(w_uv), _ptr(o), _ptr(lse), _stream()), "gqla_combine_up_proj")
+
+
+# ------------------------------------------------------------------ a value head dimension of its own (Sec. 3.2)
+
+
+def gqla_expand_cache_dv(dims: GqlaDims, cache: torch.Tensor, w_uk: torch.Tensor, w_uv: torch.Tensor,
+                         k_c: torch.Tensor, v: torch.Tensor, k_r: torch.Tensor | None) -> None:
+    """gqla_expand_cache with w_uv [g, r_kv, d_v] and v [N, g, d_v]; d_v is read off w_uv."""
+    _contig(w_uk, w_uv, k_c, v, k_r)
+    assert cache.dim() == 2 and cache.stride(1) == 1 and v.shape[-1] == w_uv.shape[-1]
+    _check(lib().gqla_expand_cache_dv(ctypes.byref(dims), w_uv.shape[-1], _dtype_code(cache), cache.shape[0], _ptr(cache),
+                                      cache.stride(0), _ptr(w_uk), _ptr(w_uv), _ptr(k_c), _ptr(v), _ptr(k_r), _stream()),
+           "gqla_expand_cache_dv")
+
+
+def gqla_decode_gqa_dv(dims: GqlaDims, q: torch.Tensor, k_c: torch.Tensor, v: torch.Tensor, k_r: torch.Tensor,
+                       seq_start: torch.Tensor, seqlens: torch.Tensor, scale: float, num_splits: int,
+                       o_part: torch.Tensor, lse_part: torch.Tensor, status_word: torch.Tensor | None = None) -> None:
+    """gqla_decode_gqa with v [N, g, d_v] and o_part [B, S, s_q, h_q, d_v]; d_v is read off v."""
+    _contig(q, k_c, v, seq_start, seqlens, o_part, lse_part)
+    assert k_r.dim() == 2 and k_r.stride(1) == 1 and o_part.shape[-1] == v.shape[-1]
+    assert seq_start.dtype == torch.int64 and seqlens.dtype == torch.int32
+    assert o_part.dtype == torch.float32 and lse_part.dtype == torch.float32
+    B, s_q = q.shape[0], q.shape[1]
+    _check(lib().gqla_decode_gqa_dv(ctypes.byref(dims), v.shape[-1], _dtype_code(q), B, s_q, scale, num_splits, _ptr(q),
+                                    _ptr(k_c), _ptr(v), _ptr(k_r), k_r.stride(0), k_c.shape[0], _ptr(seq_start),
+                                    _ptr(seqlens), _ptr(o_part), _ptr(lse_part), _ptr(status_word), _stream()),
+           "gqla_decode_gqa_dv")
+
+
+def gqla_up_proj_dv(dims: GqlaDims, o_hat: torch.Tensor, w_uv: torch.Tensor, o: torch.Tensor) -> None:
+    """gqla_up_proj with w_uv [g, r_kv, d_v] and o [B, s_q, h_q, d_v]; d_v is read off w_uv."""
+    _contig(o_hat, w_uv, o)
+    assert o.shape[-1] == w_uv.shape[-1]
+    B, s_q = o_hat.shape[0], o_hat.shape[1]
+    _check(lib().gqla_up_proj_dv(ctypes.byref(dims), w_uv.shape[-1], _dtype_code(o_hat), B, s_q, _ptr(o_hat), _ptr(w_uv),
+                                 _ptr(o), _stream()), "gqla_up_proj_dv")
 
 
 # ------------------------------------------------------------------ integer helpers (host)

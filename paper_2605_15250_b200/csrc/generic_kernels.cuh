@@ -217,6 +217,7 @@ __global__ void __launch_bounds__(128) absorb_q_generic_kernel(int32_t h_q, int3
 }
 
 // o[row, d] = sum_r W_UV[j][r][d] * o_hat[row, r].  One block per row; o_hat row staged in smem.
+// d_h here is the width of W_UV's rows and of the output (the value head dim d_h^V when it differs from d_h).
 template <typename T>
 __global__ void __launch_bounds__(128) up_proj_generic_kernel(int32_t h_q, int32_t hpg, int32_t d_h, int32_t r_kv,
                                                               const T* __restrict__ o_hat, const T* __restrict__ w_uv,
@@ -281,8 +282,8 @@ __global__ void __launch_bounds__(128) combine_up_generic_kernel(int32_t h_q, in
 // owns one (j, d) output column of both planes for all staged rows.
 constexpr int kExpandRows = 8;
 template <typename T>
-__global__ void __launch_bounds__(256) expand_cache_generic_kernel(int64_t N, int32_t g, int32_t d_h, int32_t r_kv,
-                                                                   int32_t d_r, const T* __restrict__ cache,
+__global__ void __launch_bounds__(256) expand_cache_generic_kernel(int64_t N, int32_t g, int32_t d_h, int32_t d_v,
+                                                                   int32_t r_kv, int32_t d_r, const T* __restrict__ cache,
                                                                    int64_t cache_stride, const T* __restrict__ w_uk,
                                                                    const T* __restrict__ w_uv, T* __restrict__ k_c,
                                                                    T* __restrict__ v, T* __restrict__ k_r) {
@@ -294,29 +295,27 @@ __global__ void __launch_bounds__(256) expand_cache_generic_kernel(int64_t N, in
         cs[rr * r_kv + c] = ldf(cache + (n0 + rr) * cache_stride + c);
     }
     __syncthreads();
-    const int cols = g * d_h;
-    for (int col = threadIdx.x; col < cols; col += blockDim.x) {
-        const int j = col / d_h, d = col % d_h;
-        const T* wk = w_uk + (int64_t)j * r_kv * d_h + d;
-        const T* wv = w_uv + (int64_t)j * r_kv * d_h + d;
-        float ak[kExpandRows], av[kExpandRows];
+    // plane 0: K_C with W_UK [g, r_kv, d_h];  plane 1: V with W_UV [g, r_kv, d_v]
+    for (int plane = 0; plane < 2; ++plane) {
+        const int dd = plane == 0 ? d_h : d_v;
+        const T* wbase = plane == 0 ? w_uk : w_uv;
+        T* out = plane == 0 ? k_c : v;
+        const int cols = g * dd;
+        for (int col = threadIdx.x; col < cols; col += blockDim.x) {
+            const int j = col / dd, d = col % dd;
+            const T* w = wbase + (int64_t)j * r_kv * dd + d;
+            float acc[kExpandRows];
 #pragma unroll
-        for (int rr = 0; rr < kExpandRows; ++rr) ak[rr] = av[rr] = 0.f;
-        for (int r = 0; r < r_kv; ++r) {
-            const float a = ldf(wk + (int64_t)r * d_h), b = ldf(wv + (int64_t)r * d_h);
+            for (int rr = 0; rr < kExpandRows; ++rr) acc[rr] = 0.f;
+            for (int r = 0; r < r_kv; ++r) {
+                const float a = ldf(w + (int64_t)r * dd);
 #pragma unroll
-            for (int rr = 0; rr < kExpandRows; ++rr) {
-                const float c = cs[rr * r_kv + r];
-                ak[rr] = fmaf(a, c, ak[rr]);
-                av[rr] = fmaf(b, c, av[rr]);
+                for (int rr = 0; rr < kExpandRows; ++rr) acc[rr] = fmaf(a, cs[rr * r_kv + r], acc[rr]);
             }
+#pragma unroll
+            for (int rr = 0; rr < kExpandRows; ++rr)
+                if (rr < nr) stf(out + (n0 + rr) * cols + col, acc[rr]);
         }
-#pragma unroll
-        for (int rr = 0; rr < kExpandRows; ++rr)
-            if (rr < nr) {
-                stf(k_c + (n0 + rr) * cols + col, ak[rr]);
-                stf(v + (n0 + rr) * cols + col, av[rr]);
-            }
     }
     if (k_r != nullptr)
         for (int t = threadIdx.x; t < nr * d_r; t += blockDim.x) {

@@ -160,17 +160,22 @@ gqla_status gqla_absorb_q(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32
 
 gqla_status gqla_up_proj(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, const void* o_hat,
                          const void* w_uv, void* o, void* stream) {
+    return gqla_up_proj_dv(d, d == nullptr ? 0 : d->d_h, dtype, B, s_q, o_hat, w_uv, o, stream);
+}
+
+gqla_status gqla_up_proj_dv(const gqla_dims* d, int32_t d_v, gqla_dtype dtype, int32_t B, int32_t s_q,
+                            const void* o_hat, const void* w_uv, void* o, void* stream) {
     gqla_status s;
     if ((s = check_dims(d)) != GQLA_OK) return s;
     if ((s = check_dtype(dtype)) != GQLA_OK) return s;
-    if (B < 0 || s_q < 1) return GQLA_ERR_SHAPE;
+    if (B < 0 || s_q < 1 || d_v < 1) return GQLA_ERR_SHAPE;
     if (o_hat == nullptr || w_uv == nullptr || o == nullptr) return GQLA_ERR_NULL;
     if (!aligned16(o_hat) || !aligned16(w_uv) || !aligned16(o)) return GQLA_ERR_ALIGN;
     const int64_t rows = (int64_t)B * s_q * d->h_q;
     if (rows == 0) return GQLA_OK;
     if (rows > 0x7fffffffLL) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
-    if (g_policy.load() == GQLA_POLICY_AUTO) {
+    if (g_policy.load() == GQLA_POLICY_AUTO && d_v == d->d_h) {
         s = tc_up_proj(*d, dtype, B, s_q, o_hat, w_uv, o, st);
         if (s != GQLA_ERR_UNSUPPORTED) return s;
     }
@@ -179,9 +184,9 @@ gqla_status gqla_up_proj(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_
     if (smem > 48 * 1024) return GQLA_ERR_UNSUPPORTED;
     if (dtype == GQLA_BF16)
         up_proj_generic_kernel<__nv_bfloat16><<<(unsigned)rows, 128, smem, st>>>(
-            d->h_q, hpg, d->d_h, d->r_kv, (const __nv_bfloat16*)o_hat, (const __nv_bfloat16*)w_uv, (__nv_bfloat16*)o);
+            d->h_q, hpg, d_v, d->r_kv, (const __nv_bfloat16*)o_hat, (const __nv_bfloat16*)w_uv, (__nv_bfloat16*)o);
     else
-        up_proj_generic_kernel<float><<<(unsigned)rows, 128, smem, st>>>(d->h_q, hpg, d->d_h, d->r_kv,
+        up_proj_generic_kernel<float><<<(unsigned)rows, 128, smem, st>>>(d->h_q, hpg, d_v, d->r_kv,
                                                                         (const float*)o_hat, (const float*)w_uv,
                                                                         (float*)o);
     return launch_status();
@@ -221,17 +226,24 @@ gqla_status gqla_combine_up_proj(const gqla_dims* d, gqla_dtype dtype, int32_t B
 gqla_status gqla_expand_cache(const gqla_dims* d, gqla_dtype dtype, int64_t N, const void* cache,
                               int64_t cache_row_stride, const void* w_uk, const void* w_uv, void* k_c, void* v,
                               void* k_r, void* stream) {
+    return gqla_expand_cache_dv(d, d == nullptr ? 0 : d->d_h, dtype, N, cache, cache_row_stride, w_uk, w_uv, k_c, v, k_r,
+                                stream);
+}
+
+gqla_status gqla_expand_cache_dv(const gqla_dims* d, int32_t d_v, gqla_dtype dtype, int64_t N, const void* cache,
+                                 int64_t cache_row_stride, const void* w_uk, const void* w_uv, void* k_c, void* v,
+                                 void* k_r, void* stream) {
     gqla_status s;
     if ((s = check_dims(d)) != GQLA_OK) return s;
     if ((s = check_dtype(dtype)) != GQLA_OK) return s;
-    if (N < 0 || cache_row_stride < d->r_kv + d->d_r) return GQLA_ERR_SHAPE;
+    if (N < 0 || cache_row_stride < d->r_kv + d->d_r || d_v < 1) return GQLA_ERR_SHAPE;
     if (N == 0) return GQLA_OK;
     if (cache == nullptr || w_uk == nullptr || w_uv == nullptr || k_c == nullptr || v == nullptr) return GQLA_ERR_NULL;
     if (!aligned16(cache) || !aligned16(w_uk) || !aligned16(w_uv) || !aligned16(k_c) || !aligned16(v) ||
         !aligned16(k_r))
         return GQLA_ERR_ALIGN;
     cudaStream_t st = (cudaStream_t)stream;
-    if (g_policy.load() == GQLA_POLICY_AUTO) {
+    if (g_policy.load() == GQLA_POLICY_AUTO && d_v == d->d_h) {
         s = tc_expand_cache(*d, dtype, N, cache, cache_row_stride, w_uk, w_uv, k_c, v, k_r, st);
         if (s != GQLA_ERR_UNSUPPORTED) return s;
     }
@@ -241,12 +253,12 @@ gqla_status gqla_expand_cache(const gqla_dims* d, gqla_dtype dtype, int64_t N, c
     if (blocks > 0x7fffffffLL) return GQLA_ERR_SHAPE;
     if (dtype == GQLA_BF16)
         expand_cache_generic_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, smem, st>>>(
-            N, d->g, d->d_h, d->r_kv, d->d_r, (const __nv_bfloat16*)cache, cache_row_stride,
+            N, d->g, d->d_h, d_v, d->r_kv, d->d_r, (const __nv_bfloat16*)cache, cache_row_stride,
             (const __nv_bfloat16*)w_uk, (const __nv_bfloat16*)w_uv, (__nv_bfloat16*)k_c, (__nv_bfloat16*)v,
             (__nv_bfloat16*)k_r);
     else
         expand_cache_generic_kernel<float><<<(unsigned)blocks, 256, smem, st>>>(
-            N, d->g, d->d_h, d->r_kv, d->d_r, (const float*)cache, cache_row_stride, (const float*)w_uk,
+            N, d->g, d->d_h, d_v, d->r_kv, d->d_r, (const float*)cache, cache_row_stride, (const float*)w_uk,
             (const float*)w_uv, (float*)k_c, (float*)v, (float*)k_r);
     return launch_status();
 }
@@ -384,7 +396,7 @@ gqla_status gqla_decode_absorb_paged(const gqla_dims* d, gqla_dtype dtype, int32
                              paged_rows(block_table, max_pages, page_size), seqlens, o_part, lse_part, status_word, stream);
 }
 
-static gqla_status decode_gqa_any(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+static gqla_status decode_gqa_any(const gqla_dims* d, int32_t d_v, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
                                   int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
                                   int64_t k_r_row_stride, int64_t n_rows, const RowMap& rows, const int32_t* seqlens,
                                   float* o_part, float* lse_part, int32_t* status_word, void* stream) {
@@ -393,9 +405,9 @@ static gqla_status decode_gqa_any(const gqla_dims* d, gqla_dtype dtype, int32_t 
     if (B == 0) return GQLA_OK;
     if (q == nullptr || k_c == nullptr || v == nullptr || (d->d_r > 0 && k_r == nullptr)) return GQLA_ERR_NULL;
     if (!aligned16(q) || !aligned16(k_c) || !aligned16(v) || !aligned16(k_r)) return GQLA_ERR_ALIGN;
-    if ((d->d_r > 0 && k_r_row_stride < d->d_r) || n_rows < 0) return GQLA_ERR_SHAPE;
+    if ((d->d_r > 0 && k_r_row_stride < d->d_r) || n_rows < 0 || d_v < 1) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
-    if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, 1)) {
+    if (g_policy.load() == GQLA_POLICY_AUTO && d_v == d->d_h && tc_covers(*d, dtype, s_q, 1)) {
         s = tc_decode_gqa(*d, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, n_rows, rows, seqlens, o_part,
                           lse_part, status_word, st);
         if (s != GQLA_ERR_UNSUPPORTED) return s;
@@ -404,19 +416,27 @@ static gqla_status decode_gqa_any(const gqla_dims* d, gqla_dtype dtype, int32_t 
     a.q = q;
     a.kA = k_c; a.kA_stride = (int64_t)d->g * d->d_h; a.kA_gstride = d->d_h; a.dA = d->d_h;
     a.kB = k_r; a.kB_stride = k_r_row_stride; a.dB = d->d_r;
-    a.v = v; a.v_stride = (int64_t)d->g * d->d_h; a.v_gstride = d->d_h; a.dv = d->d_h;
+    a.v = v; a.v_stride = (int64_t)d->g * d_v; a.v_gstride = d_v; a.dv = d_v;
     a.rows = rows; a.seqlens = seqlens;
     a.B = B; a.S = num_splits < 0 ? -num_splits : num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
     a.scale = scale; a.o_part = o_part; a.lse_part = lse_part;
     return launch_decode_generic(dtype, a, st);
 }
 
+gqla_status gqla_decode_gqa_dv(const gqla_dims* d, int32_t d_v, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
+                               int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
+                               int64_t k_r_row_stride, int64_t n_rows, const int64_t* seq_start, const int32_t* seqlens,
+                               float* o_part, float* lse_part, int32_t* status_word, void* stream) {
+    return decode_gqa_any(d, d_v, dtype, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, n_rows,
+                          packed_rows(seq_start), seqlens, o_part, lse_part, status_word, stream);
+}
+
 gqla_status gqla_decode_gqa(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
                             int32_t num_splits, const void* q, const void* k_c, const void* v, const void* k_r,
                             int64_t k_r_row_stride, int64_t n_rows, const int64_t* seq_start, const int32_t* seqlens,
                             float* o_part, float* lse_part, int32_t* status_word, void* stream) {
-    return decode_gqa_any(d, dtype, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, n_rows,
-                          packed_rows(seq_start), seqlens, o_part, lse_part, status_word, stream);
+    return decode_gqa_any(d, d == nullptr ? 0 : d->d_h, dtype, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride,
+                          n_rows, packed_rows(seq_start), seqlens, o_part, lse_part, status_word, stream);
 }
 
 gqla_status gqla_decode_gqa_paged(const gqla_dims* d, gqla_dtype dtype, int32_t B, int32_t s_q, float scale,
@@ -424,8 +444,9 @@ gqla_status gqla_decode_gqa_paged(const gqla_dims* d, gqla_dtype dtype, int32_t 
                                   int64_t k_r_row_stride, int64_t n_rows, const int32_t* block_table, int32_t max_pages,
                                   int32_t page_size, const int32_t* seqlens, float* o_part, float* lse_part,
                                   int32_t* status_word, void* stream) {
-    return decode_gqa_any(d, dtype, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, n_rows,
-                          paged_rows(block_table, max_pages, page_size), seqlens, o_part, lse_part, status_word, stream);
+    return decode_gqa_any(d, d == nullptr ? 0 : d->d_h, dtype, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride,
+                          n_rows, paged_rows(block_table, max_pages, page_size), seqlens, o_part, lse_part, status_word,
+                          stream);
 }
 
 gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_splits, int32_t d_out,

@@ -508,6 +508,66 @@ def test_determinism_run_to_run():
     dec.check_status()
 
 
+# ------------------------------------------------------------------ a value head dimension of its own
+
+
+@pytest.mark.parametrize("dims,d_v,dtype", [(dict(h_q=20, g=4, d_h=192, r_kv=512, d_r=64), 256, "bf16"),   # GLM-like
+                                            (dict(h_q=32, g=8, d_h=128, r_kv=512, d_r=64), 256, "bf16"),
+                                            (dict(h_q=8, g=2, d_h=16, r_kv=32, d_r=8), 24, "f32")])
+def test_separate_value_head_dim(dims, d_v, dtype):
+    """Sec. 3.2 "From MLA to GQLA": d_h^V != d_h.  Both paths through the *_dv calls against the oracle, stage by
+    stage where d_v enters (expansion, GQA attention, up-projection) and end to end."""
+    from tests.parity_util import assert_close
+    from oracle import gqla_oracle as O
+    w = synth.Workload("dv", batch=3, s_q=2, dtype=dtype, seed=77, d_v=d_v, **dims)
+    seqlens = np.array([300, 1, 1029], dtype=np.int32)
+    x = synth.make_inputs(w, seqlens=seqlens, q_gain=3.0)
+    od = O.Dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r, d_v)
+    bd = B.make_dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    dev = {k: t.cuda() for k, t in x.items()}
+    f = {k: synth.to_f64(t) for k, t in x.items() if k not in ("seq_start", "seqlens")}
+    ss, sl = x["seq_start"].numpy(), x["seqlens"].numpy()
+    N, Bn, s_q, S = x["cache"].shape[0], w.batch, w.s_q, 3
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # expansion
+    k_c = torch.empty((N, w.g, w.d_h), dtype=td, device="cuda")
+    v = torch.empty((N, w.g, d_v), dtype=td, device="cuda")
+    k_r = torch.empty((N, w.d_r), dtype=td, device="cuda")
+    B.gqla_expand_cache_dv(bd, dev["cache"], dev["w_uk"], dev["w_uv"], k_c, v, k_r)
+    kc_ref, v_ref, kr_ref = O.expand_cache(od, f["cache"], f["w_uk"], f["w_uv"])
+    assert_close(k_c.float().cpu().numpy(), kc_ref, "expand_dv k_c")
+    assert_close(v.float().cpu().numpy(), v_ref, "expand_dv v")
+    assert np.array_equal(k_r.float().cpu().numpy(), kr_ref)
+    # GQA path on the library's own planes, against the oracle on those planes and on the unrounded chain
+    q = torch.cat([x["q_c"], x["q_r"]], -1).contiguous()
+    o_part = torch.full((Bn, S, s_q, w.h_q, d_v), float("nan"), dtype=torch.float32, device="cuda")
+    lse_part = torch.full((Bn, S, s_q, w.h_q), float("nan"), dtype=torch.float32, device="cuda")
+    B.gqla_decode_gqa_dv(bd, q.cuda(), k_c, v, k_r, dev["seq_start"], dev["seqlens"], w.scale, S, o_part, lse_part, status)
+    op_ref, lp_ref = O.decode_gqa_partials(od, synth.to_f64(q), synth.to_f64(k_c), synth.to_f64(v), synth.to_f64(k_r), ss, sl,
+                                           s_q, w.scale, S)
+    assert_close(o_part.cpu().numpy(), op_ref, "decode_gqa_dv o_part")
+    assert_close(lse_part.cpu().numpy(), lp_ref, "decode_gqa_dv lse_part")
+    o_g = torch.empty((Bn, s_q, w.h_q, d_v), dtype=td, device="cuda")
+    B.gqla_combine_splits(o_part, lse_part, o_g, None)
+    ref = O.gqa_path(od, f["q_c"], f["q_r"], f["w_uk"], f["w_uv"], f["cache"], ss, sl, s_q, w.scale)
+    assert ref.shape[-1] == d_v
+    assert_close(o_g.float().cpu().numpy(), ref, "gqa path with d_v")
+    # absorb path: the latent attention is unchanged, the up-projection is d_v wide
+    q_hat = torch.empty((Bn, s_q, w.h_q, w.d_abs), dtype=td, device="cuda")
+    B.gqla_absorb_q(bd, dev["q_c"], dev["q_r"], dev["w_uk"], q_hat)
+    oa_part = torch.empty((Bn, S, s_q, w.h_q, w.r_kv), dtype=torch.float32, device="cuda")
+    la_part = torch.empty((Bn, S, s_q, w.h_q), dtype=torch.float32, device="cuda")
+    B.gqla_decode_absorb(bd, q_hat, dev["cache"], dev["seq_start"], dev["seqlens"], w.scale, S, oa_part, la_part, status)
+    o_hat = torch.empty((Bn, s_q, w.h_q, w.r_kv), dtype=td, device="cuda")
+    B.gqla_combine_splits(oa_part, la_part, o_hat, None)
+    o_a = torch.empty((Bn, s_q, w.h_q, d_v), dtype=td, device="cuda")
+    B.gqla_up_proj_dv(bd, o_hat, dev["w_uv"], o_a)
+    assert_close(o_a.float().cpu().numpy(), O.up_proj(od, synth.to_f64(o_hat), f["w_uv"]), "up_proj_dv")
+    assert_close(o_a.float().cpu().numpy(), ref, "absorb path with d_v")
+    assert int(status.item()) == 0
+
+
 # ------------------------------------------------------------------ workloads C1-C4 at full size
 
 
