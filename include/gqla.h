@@ -206,6 +206,47 @@ gqla_status gqla_decode_gqa_paged(const gqla_dims* dims, gqla_dtype dtype, int32
                                   int32_t max_pages, int32_t page_size, const int32_t* seqlens, float* o_part,
                                   float* lse_part, int32_t* status_word, void* stream);
 
+/* FP8 (E4M3) KV cache.  The paper names KV-cache quantisation among the effects its model leaves out (Sec. 5.1
+ * "Limitations", item (i)); what follows is this library's reading.  Elements are E4M3 codes (8-bit float: 4
+ * exponent bits with bias 7, 3 mantissa bits, no infinities, largest finite value 448, NaN = S.1111.111), one
+ * byte each: 576 B per token on the absorb path, 2112 B on the GQA path.  Scales are fp32, one per tensor
+ * plane (latent part, RoPE part; K_C, V, k^R), chosen by the caller (e.g. max|x| / 448 from calibration):
+ * a stored value is  code * scale.  Queries are quantised per row, with the planes' scales folded in, so a
+ * score needs one factor per row and an output one factor per call:
+ *     x_s = scale * q_scale[row] * sum_c dec(q8[row, c]) dec(k8[s, c]),      o = v_scale * softmax(x) . dec(v8).
+ * The softmax probabilities are rounded to E4M3 before the P.V contraction on the tensor-core kernels (to fp32
+ * nothing on the generic ones), the counterpart of the bf16 rounding of the bf16 path.
+ *
+ * gqla_quantize_cols_e4m3: dst[r, c] = encode(float(src[r, c]) * (1 / scale)), scale = scale_a for columns
+ *   c < split and scale_b for the others (the latent cache: split = r_kv, scale_a = latent scale, scale_b = RoPE
+ *   scale; a single plane: split = width).  src [rows, width] of src_dtype with row stride src_row_stride
+ *   (elements); dst [rows, width] bytes, dense.  encode rounds to the nearest code, ties to the even mantissa,
+ *   saturating at +-448; the multiplication and the reciprocal are fp32 operations with IEEE rounding.
+ * gqla_quantize_rows_e4m3: per row  y = float(src) * pre  (pre_a for c < split, pre_b for the others: the
+ *   scales of the key planes the row will meet),  s = max|y| / 448  (1 for an all-zero row),
+ *   dst = encode(y * (1 / s)),  row_scale[row] = s.  src [rows, width] dense.  Use it on q_hat (absorb path:
+ *   split = r_kv) or on [q^C ; q^R] (GQA path: split = d_h). */
+gqla_status gqla_quantize_cols_e4m3(gqla_dtype src_dtype, int64_t rows, int32_t width, int32_t split, float scale_a,
+                                    float scale_b, const void* src, int64_t src_row_stride, uint8_t* dst, void* stream);
+gqla_status gqla_quantize_rows_e4m3(gqla_dtype src_dtype, int64_t rows, int32_t width, int32_t split, float pre_a,
+                                    float pre_b, const void* src, uint8_t* dst, float* row_scale, void* stream);
+/* Eq. (mqa), lines 3-5, over an E4M3 latent cache:  q8 [B, s_q, h_q, r_kv+d_r] codes, q_scale [B, s_q, h_q] fp32,
+ * cache8 [N, r_kv+d_r] codes with row stride cache_row_stride (bytes), v_scale = the latent plane's scale.
+ * Fixed split plan only (num_splits >= 1).  Outputs and the other arguments as for gqla_decode_absorb. */
+gqla_status gqla_decode_absorb_fp8(const gqla_dims* dims, int32_t B, int32_t s_q, float scale, int32_t num_splits,
+                                   const uint8_t* q8, const float* q_scale, const uint8_t* cache8,
+                                   int64_t cache_row_stride, int64_t cache_rows, float v_scale, const int64_t* seq_start,
+                                   const int32_t* seqlens, float* o_part, float* lse_part, int32_t* status_word,
+                                   void* stream);
+/* Eq. (mha) over E4M3 planes:  q8 [B, s_q, h_q, d_h+d_r], q_scale [B, s_q, h_q];  k_c8, v8 [N, g, d_h];
+ * k_r8 [N, .] with row stride k_r_row_stride (bytes);  v_scale = the V plane's scale.  Fixed split plan only.
+ * Outputs and the other arguments as for gqla_decode_gqa. */
+gqla_status gqla_decode_gqa_fp8(const gqla_dims* dims, int32_t B, int32_t s_q, float scale, int32_t num_splits,
+                                const uint8_t* q8, const float* q_scale, const uint8_t* k_c8, const uint8_t* v8,
+                                const uint8_t* k_r8, int64_t k_r_row_stride, int64_t n_rows, float v_scale,
+                                const int64_t* seq_start, const int32_t* seqlens, float* o_part, float* lse_part,
+                                int32_t* status_word, void* stream);
+
 /* Log-sum-exp merge of split partials (split-KV is not in the paper; it is the flash-decoding
  * reduction of the same softmax):  M = max_k lse_k, w_k = exp(lse_k - M),
  *   out = sum_k w_k o_k / sum_k w_k,   lse = M + ln sum_k w_k;  all splits empty -> out = 0, lse = -inf.

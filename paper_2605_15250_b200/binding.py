@@ -68,6 +68,15 @@ _PROTOTYPES = {
     "gqla_decode_gqa_dv": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p,
                                      c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p, c_void_p,
                                      c_void_p, c_void_p]),
+    "gqla_quantize_cols_e4m3": (c_int32, [c_int32, c_int64, c_int32, c_int32, c_float, c_float, c_void_p, c_int64, c_void_p,
+                                          c_void_p]),
+    "gqla_quantize_rows_e4m3": (c_int32, [c_int32, c_int64, c_int32, c_int32, c_float, c_float, c_void_p, c_void_p, c_void_p,
+                                          c_void_p]),
+    "gqla_decode_absorb_fp8": (c_int32, [c_void_p, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p, c_void_p, c_int64,
+                                         c_int64, c_float, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_decode_gqa_fp8": (c_int32, [c_void_p, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
+                                      c_void_p, c_int64, c_int64, c_float, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                      c_void_p]),
     "gqla_split_plan": (c_int32, [c_int32, c_int32, c_void_p, c_void_p]),
     "gqla_visible_limit": (c_int32, [c_int32, c_int32, c_int32]),
     "gqla_balanced_plan": (c_int32, [c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p]),
@@ -349,6 +358,59 @@ def gqla_up_proj_dv(dims: GqlaDims, o_hat: torch.Tensor, w_uv: torch.Tensor, o: 
     B, s_q = o_hat.shape[0], o_hat.shape[1]
     _check(lib().gqla_up_proj_dv(ctypes.byref(dims), w_uv.shape[-1], _dtype_code(o_hat), B, s_q, _ptr(o_hat), _ptr(w_uv),
                                  _ptr(o), _stream()), "gqla_up_proj_dv")
+
+
+# ------------------------------------------------------------------ FP8 (E4M3) cache
+
+
+def gqla_quantize_cols_e4m3(src: torch.Tensor, split: int, scale_a: float, scale_b: float, dst: torch.Tensor) -> None:
+    """dst (uint8 codes, dense [rows, width]) = encode(src / scale), scale_a for columns < split, scale_b beyond.
+    src is [rows, width] (rows may be strided) or any dense tensor whose last dimension is the width."""
+    if src.dim() != 2:
+        src = src.reshape(-1, src.shape[-1])
+    assert src.stride(1) == 1 and dst.dtype == torch.uint8 and dst.is_contiguous() and dst.numel() == src.numel()
+    _check(lib().gqla_quantize_cols_e4m3(_dtype_code(src), src.shape[0], src.shape[1], split, scale_a, scale_b, _ptr(src),
+                                         src.stride(0), _ptr(dst), _stream()), "gqla_quantize_cols_e4m3")
+
+
+def gqla_quantize_rows_e4m3(src: torch.Tensor, split: int, pre_a: float, pre_b: float, dst: torch.Tensor,
+                            row_scale: torch.Tensor) -> None:
+    """Per-row quantisation of query rows (last dimension = width): codes into dst (uint8, same shape), the row
+    scales into row_scale (fp32, shape without the last dimension)."""
+    _contig(src, dst, row_scale)
+    assert dst.dtype == torch.uint8 and row_scale.dtype == torch.float32
+    rows = src.numel() // src.shape[-1]
+    assert row_scale.numel() == rows and dst.numel() == src.numel()
+    _check(lib().gqla_quantize_rows_e4m3(_dtype_code(src), rows, src.shape[-1], split, pre_a, pre_b, _ptr(src), _ptr(dst),
+                                         _ptr(row_scale), _stream()), "gqla_quantize_rows_e4m3")
+
+
+def gqla_decode_absorb_fp8(dims: GqlaDims, q8: torch.Tensor, q_scale: torch.Tensor, cache8: torch.Tensor, v_scale: float,
+                           seq_start: torch.Tensor, seqlens: torch.Tensor, scale: float, num_splits: int,
+                           o_part: torch.Tensor, lse_part: torch.Tensor, status_word: torch.Tensor | None = None) -> None:
+    """Absorb-path attention over an E4M3 latent cache (codes [N, r_kv+d_r]); q8 / q_scale from gqla_quantize_rows_e4m3."""
+    _contig(q8, q_scale, seq_start, seqlens, o_part, lse_part)
+    assert q8.dtype == torch.uint8 and cache8.dtype == torch.uint8 and cache8.dim() == 2 and cache8.stride(1) == 1
+    assert q_scale.dtype == torch.float32 and o_part.dtype == torch.float32 and lse_part.dtype == torch.float32
+    B, s_q = q8.shape[0], q8.shape[1]
+    _check(lib().gqla_decode_absorb_fp8(ctypes.byref(dims), B, s_q, scale, num_splits, _ptr(q8), _ptr(q_scale), _ptr(cache8),
+                                        cache8.stride(0), cache8.shape[0], v_scale, _ptr(seq_start), _ptr(seqlens),
+                                        _ptr(o_part), _ptr(lse_part), _ptr(status_word), _stream()), "gqla_decode_absorb_fp8")
+
+
+def gqla_decode_gqa_fp8(dims: GqlaDims, q8: torch.Tensor, q_scale: torch.Tensor, k_c8: torch.Tensor, v8: torch.Tensor,
+                        k_r8: torch.Tensor, v_scale: float, seq_start: torch.Tensor, seqlens: torch.Tensor, scale: float,
+                        num_splits: int, o_part: torch.Tensor, lse_part: torch.Tensor,
+                        status_word: torch.Tensor | None = None) -> None:
+    """GQA-path attention over E4M3 planes K_C, V [N, g, d_h] and k_R [N, d_r] (k_R rows may be strided)."""
+    _contig(q8, q_scale, k_c8, v8, seq_start, seqlens, o_part, lse_part)
+    assert q8.dtype == k_c8.dtype == v8.dtype == k_r8.dtype == torch.uint8 and k_r8.dim() == 2 and k_r8.stride(1) == 1
+    assert q_scale.dtype == torch.float32 and o_part.dtype == torch.float32 and lse_part.dtype == torch.float32
+    B, s_q = q8.shape[0], q8.shape[1]
+    _check(lib().gqla_decode_gqa_fp8(ctypes.byref(dims), B, s_q, scale, num_splits, _ptr(q8), _ptr(q_scale), _ptr(k_c8),
+                                     _ptr(v8), _ptr(k_r8), k_r8.stride(0), k_c8.shape[0], v_scale, _ptr(seq_start),
+                                     _ptr(seqlens), _ptr(o_part), _ptr(lse_part), _ptr(status_word), _stream()),
+           "gqla_decode_gqa_fp8")
 
 
 # ------------------------------------------------------------------ integer helpers (host)

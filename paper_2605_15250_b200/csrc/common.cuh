@@ -1,6 +1,7 @@
 // Shared device/host helpers for the GQLA kernels (integer bookkeeping, type loads).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -37,6 +38,23 @@ struct RowMap {
     }
 };
 
+// FP8 E4M3 storage (4 exponent bits, bias 7; 3 mantissa bits; no infinity; largest finite value 448).
+struct e4m3 {
+    uint8_t code;
+};
+// One code -> fp32 (exact: every E4M3 value is an fp16 value).
+__device__ __forceinline__ float e4m3_to_float(uint8_t code) {
+    uint32_t h2;
+    asm("{\n\t.reg .b16 c;\n\tcvt.u16.u32 c, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, c;\n\t}" : "=r"(h2) : "r"((uint32_t)code));
+    return __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
+}
+// Two fp32 -> two codes (low byte = lo): round to nearest even, magnitudes beyond 448 saturate, NaN -> 0x7F.
+__device__ __forceinline__ uint16_t float2_to_e4m3x2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ float ldf(const e4m3* p) { return e4m3_to_float(p->code); }
 __device__ __forceinline__ float ldf(const float* p) { return *p; }
 __device__ __forceinline__ float ldf(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 __device__ __forceinline__ void stf(float* p, float v) { *p = v; }

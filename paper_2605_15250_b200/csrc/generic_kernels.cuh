@@ -2,6 +2,8 @@
 // They are the correctness floor for shapes the tensor-core kernels do not cover, and an
 // on-device cross-check for the ones they do.  fp32 arithmetic throughout.
 #pragma once
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace gqla {
@@ -21,6 +23,9 @@ struct DecodeArgs {
     float* o_part;    // [B, S, s_q, h_q, dv]
     float* lse_part;  // [B, S, s_q, h_q]
     void* o_final;    // not null (S == 1 only): the output goes here in the storage type, o_part unused, lse_part may be null
+    // FP8 cache: scores are multiplied by q_row_scale[(b, p, i)] (null = 1) and outputs by v_scale (0 = 1)
+    const float* q_row_scale;
+    float v_scale;
 };
 
 constexpr int kGenericMaxV = 16;  // value columns per lane: dv <= 512
@@ -54,6 +59,7 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a) {
 #pragma unroll
     for (int c = 0; c < kGenericMaxV; ++c) acc[c] = 0.f;
     float m = -INFINITY, l = 0.f;
+    const float x_scale = a.scale * (a.q_row_scale != nullptr ? a.q_row_scale[(int64_t)(b * a.s_q + p) * a.h_q + i] : 1.f);
 
     for (int32_t s = begin; s < end; ++s) {
         const int64_t n = a.rows.row(b, s);
@@ -64,7 +70,7 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a) {
             const E* kb = kB + n * a.kB_stride;
             for (int d = lane; d < a.dB; d += 32) dot = fmaf(ldf(q + a.dA + d), ldf(kb + d), dot);
         }
-        const float x = warp_sum(dot) * a.scale;
+        const float x = warp_sum(dot) * x_scale;
         const float m_new = fmaxf(m, x);
         const float corr = expf(m - m_new);  // exp(-inf) = 0 on the first row
         const float e = expf(x - m_new);
@@ -78,15 +84,20 @@ __global__ void __launch_bounds__(128) decode_generic_kernel(DecodeArgs a) {
         m = m_new;
     }
 
-    const float inv = l > 0.f ? 1.f / l : 0.f;
+    const float inv = (l > 0.f ? 1.f / l : 0.f) * (a.v_scale != 0.f ? a.v_scale : 1.f);
 #pragma unroll
     for (int c = 0; c < kGenericMaxV; ++c) {
         const int d = lane + 32 * c;
         if (d < a.dv) {
-            if (a.o_final != nullptr)
-                stf((E*)a.o_final + row * a.dv + d, acc[c] * inv);
-            else
+            if constexpr (!std::is_same<E, e4m3>::value) {
+                if (a.o_final != nullptr) {
+                    stf((E*)a.o_final + row * a.dv + d, acc[c] * inv);
+                    continue;
+                }
+            }
+            {
                 a.o_part[row * a.dv + d] = acc[c] * inv;
+            }
         }
     }
     if (lane == 0 && a.lse_part != nullptr) a.lse_part[row] = l > 0.f ? m + logf(l) : -INFINITY;
@@ -392,6 +403,55 @@ append_expand_kernel(int32_t B, int32_t s_q, int32_t g, int32_t d_h, int32_t r_k
             const int rr = t / d_r, c = t % d_r;
             if (rows[rr] >= 0) k_r[rows[rr] * d_r + c] = cache[rows[rr] * cache_stride + r_kv + c];
         }
+}
+
+
+// ------------------------------------------------------------------------------------------------ FP8 (E4M3)
+// Quantisers.  Every step is an fp32 operation with IEEE rounding (division included), so the code a value
+// gets is a pure function of its stored bits and the scales.
+
+// dst[r, c] = encode( float(src[r, c]) * (1 / scale) ),  scale = scale_a for c < split, scale_b otherwise.
+template <typename T>
+__global__ void __launch_bounds__(256) quantize_cols_kernel(int64_t rows, int32_t width, int32_t split, float scale_a,
+                                                            float scale_b, const T* __restrict__ src, int64_t src_stride,
+                                                            uint8_t* __restrict__ dst) {
+    const float inv_a = __fdiv_rn(1.f, scale_a), inv_b = __fdiv_rn(1.f, scale_b);
+    const int64_t pairs_per_row = (width + 1) / 2;
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * pairs_per_row) return;
+    const int64_t r = idx / pairs_per_row;
+    const int c = (int)(idx % pairs_per_row) * 2;
+    const float x0 = __fmul_rn(ldf(src + r * src_stride + c), c < split ? inv_a : inv_b);
+    if (c + 1 < width) {
+        const float x1 = __fmul_rn(ldf(src + r * src_stride + c + 1), c + 1 < split ? inv_a : inv_b);
+        const uint16_t pk = float2_to_e4m3x2(x0, x1);
+        dst[r * width + c] = (uint8_t)(pk & 0xff);
+        dst[r * width + c + 1] = (uint8_t)(pk >> 8);
+    } else {
+        dst[r * width + c] = (uint8_t)(float2_to_e4m3x2(x0, 0.f) & 0xff);
+    }
+}
+
+// Per row: y = float(src) * pre (pre_a for c < split, pre_b otherwise), s = max|y| / 448 (1 for a zero row),
+// dst = encode(y * (1 / s)), row_scale = s.  One warp per row.
+template <typename T>
+__global__ void __launch_bounds__(128) quantize_rows_kernel(int64_t rows, int32_t width, int32_t split, float pre_a,
+                                                            float pre_b, const T* __restrict__ src,
+                                                            uint8_t* __restrict__ dst, float* __restrict__ row_scale) {
+    const int lane = threadIdx.x & 31;
+    const int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (r >= rows) return;
+    const T* x = src + r * width;
+    float amax = 0.f;
+    for (int c = lane; c < width; c += 32) amax = fmaxf(amax, fabsf(__fmul_rn(ldf(x + c), c < split ? pre_a : pre_b)));
+    amax = warp_max(amax);
+    const float s = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+    const float inv = __fdiv_rn(1.f, s);
+    for (int c = lane; c < width; c += 32) {
+        const float y = __fmul_rn(__fmul_rn(ldf(x + c), c < split ? pre_a : pre_b), inv);
+        dst[r * width + c] = (uint8_t)(float2_to_e4m3x2(y, 0.f) & 0xff);
+    }
+    if (lane == 0) row_scale[r] = s;
 }
 
 }  // namespace gqla

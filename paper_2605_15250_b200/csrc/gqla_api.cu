@@ -40,6 +40,17 @@ gqla_status launch_decode_generic(gqla_dtype dtype, const DecodeArgs& a, cudaStr
     return launch_status();
 }
 
+gqla_status launch_decode_generic_fp8(const DecodeArgs& a, cudaStream_t st) {
+    if (a.dv > 32 * kGenericMaxV) return GQLA_ERR_UNSUPPORTED;
+    const int64_t nrows = (int64_t)a.B * a.S * a.s_q * a.h_q;
+    if (nrows == 0) return GQLA_OK;
+    const int warps = 4;
+    const int64_t blocks = (nrows + warps - 1) / warps;
+    if (blocks > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    decode_generic_kernel<e4m3><<<(unsigned)blocks, warps * 32, 0, st>>>(a);
+    return launch_status();
+}
+
 }  // namespace
 
 extern "C" {
@@ -485,6 +496,109 @@ gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_spl
         combine_generic_kernel<float><<<(unsigned)rows, 128, smem, st>>>(B, rows_per_seq, num_splits, d_out, o_part,
                                                                          lse_part, (float*)out, lse);
     return launch_status();
+}
+
+// ------------------------------------------------------------------------------------------------ FP8 (E4M3) cache
+
+gqla_status gqla_quantize_cols_e4m3(gqla_dtype src_dtype, int64_t rows, int32_t width, int32_t split, float scale_a,
+                                    float scale_b, const void* src, int64_t src_row_stride, uint8_t* dst, void* stream) {
+    gqla_status s;
+    if ((s = check_dtype(src_dtype)) != GQLA_OK) return s;
+    if (rows < 0 || width < 1 || split < 0 || split > width || src_row_stride < width) return GQLA_ERR_SHAPE;
+    if (!(scale_a > 0.f) || !(scale_b > 0.f)) return GQLA_ERR_SHAPE;
+    if (rows == 0) return GQLA_OK;
+    if (src == nullptr || dst == nullptr) return GQLA_ERR_NULL;
+    const int64_t items = rows * ((width + 1) / 2);
+    const int64_t blocks = (items + 255) / 256;
+    if (blocks > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (src_dtype == GQLA_BF16)
+        quantize_cols_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>(rows, width, split, scale_a, scale_b,
+                                                                              (const __nv_bfloat16*)src, src_row_stride, dst);
+    else
+        quantize_cols_kernel<float><<<(unsigned)blocks, 256, 0, st>>>(rows, width, split, scale_a, scale_b,
+                                                                      (const float*)src, src_row_stride, dst);
+    return launch_status();
+}
+
+gqla_status gqla_quantize_rows_e4m3(gqla_dtype src_dtype, int64_t rows, int32_t width, int32_t split, float pre_a,
+                                    float pre_b, const void* src, uint8_t* dst, float* row_scale, void* stream) {
+    gqla_status s;
+    if ((s = check_dtype(src_dtype)) != GQLA_OK) return s;
+    if (rows < 0 || width < 1 || split < 0 || split > width) return GQLA_ERR_SHAPE;
+    if (rows == 0) return GQLA_OK;
+    if (src == nullptr || dst == nullptr || row_scale == nullptr) return GQLA_ERR_NULL;
+    const int64_t blocks = (rows + 3) / 4;
+    if (blocks > 0x7fffffffLL) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (src_dtype == GQLA_BF16)
+        quantize_rows_kernel<__nv_bfloat16><<<(unsigned)blocks, 128, 0, st>>>(rows, width, split, pre_a, pre_b,
+                                                                              (const __nv_bfloat16*)src, dst, row_scale);
+    else
+        quantize_rows_kernel<float><<<(unsigned)blocks, 128, 0, st>>>(rows, width, split, pre_a, pre_b, (const float*)src,
+                                                                      dst, row_scale);
+    return launch_status();
+}
+
+static gqla_status check_fp8_common(const gqla_dims* d, int32_t B, int32_t s_q, int32_t S, const void* q8,
+                                    const float* q_scale, float v_scale, const int64_t* seq_start, const int32_t* seqlens,
+                                    const float* o_part, const float* lse_part) {
+    gqla_status s;
+    if ((s = check_dims(d)) != GQLA_OK) return s;
+    if (B < 0 || s_q < 1 || S < 1 || !(v_scale > 0.f)) return GQLA_ERR_SHAPE;
+    if (B == 0) return GQLA_OK;
+    if (q8 == nullptr || q_scale == nullptr || seq_start == nullptr || seqlens == nullptr || o_part == nullptr ||
+        lse_part == nullptr)
+        return GQLA_ERR_NULL;
+    if (!aligned16(q8) || !aligned16(o_part)) return GQLA_ERR_ALIGN;
+    return GQLA_OK;
+}
+
+gqla_status gqla_decode_absorb_fp8(const gqla_dims* d, int32_t B, int32_t s_q, float scale, int32_t num_splits,
+                                   const uint8_t* q8, const float* q_scale, const uint8_t* cache8, int64_t cache_row_stride,
+                                   int64_t cache_rows, float v_scale, const int64_t* seq_start, const int32_t* seqlens,
+                                   float* o_part, float* lse_part, int32_t* status_word, void* stream) {
+    gqla_status s = check_fp8_common(d, B, s_q, num_splits, q8, q_scale, v_scale, seq_start, seqlens, o_part, lse_part);
+    if (s != GQLA_OK) return s;
+    if (B == 0) return GQLA_OK;
+    if (cache8 == nullptr) return GQLA_ERR_NULL;
+    if (!aligned16(cache8)) return GQLA_ERR_ALIGN;
+    if (cache_row_stride < d->r_kv + d->d_r || cache_rows < 0) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    (void)status_word;
+    DecodeArgs a{};
+    a.q = q8;
+    a.kA = cache8; a.kA_stride = cache_row_stride; a.kA_gstride = 0; a.dA = d->r_kv + d->d_r;
+    a.kB = nullptr; a.kB_stride = 0; a.dB = 0;
+    a.v = cache8; a.v_stride = cache_row_stride; a.v_gstride = 0; a.dv = d->r_kv;
+    a.rows = packed_rows(seq_start); a.seqlens = seqlens;
+    a.B = B; a.S = num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
+    a.scale = scale; a.o_part = o_part; a.lse_part = lse_part; a.q_row_scale = q_scale; a.v_scale = v_scale;
+    return launch_decode_generic_fp8(a, st);
+}
+
+gqla_status gqla_decode_gqa_fp8(const gqla_dims* d, int32_t B, int32_t s_q, float scale, int32_t num_splits,
+                                const uint8_t* q8, const float* q_scale, const uint8_t* k_c8, const uint8_t* v8,
+                                const uint8_t* k_r8, int64_t k_r_row_stride, int64_t n_rows, float v_scale,
+                                const int64_t* seq_start, const int32_t* seqlens, float* o_part, float* lse_part,
+                                int32_t* status_word, void* stream) {
+    gqla_status s = check_fp8_common(d, B, s_q, num_splits, q8, q_scale, v_scale, seq_start, seqlens, o_part, lse_part);
+    if (s != GQLA_OK) return s;
+    if (B == 0) return GQLA_OK;
+    if (k_c8 == nullptr || v8 == nullptr || (d->d_r > 0 && k_r8 == nullptr)) return GQLA_ERR_NULL;
+    if (!aligned16(k_c8) || !aligned16(v8) || !aligned16(k_r8)) return GQLA_ERR_ALIGN;
+    if ((d->d_r > 0 && k_r_row_stride < d->d_r) || n_rows < 0) return GQLA_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    (void)status_word;
+    DecodeArgs a{};
+    a.q = q8;
+    a.kA = k_c8; a.kA_stride = (int64_t)d->g * d->d_h; a.kA_gstride = d->d_h; a.dA = d->d_h;
+    a.kB = k_r8; a.kB_stride = k_r_row_stride; a.dB = d->d_r;
+    a.v = v8; a.v_stride = (int64_t)d->g * d->d_h; a.v_gstride = d->d_h; a.dv = d->d_h;
+    a.rows = packed_rows(seq_start); a.seqlens = seqlens;
+    a.B = B; a.S = num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
+    a.scale = scale; a.o_part = o_part; a.lse_part = lse_part; a.q_row_scale = q_scale; a.v_scale = v_scale;
+    return launch_decode_generic_fp8(a, st);
 }
 
 }  // extern "C"
