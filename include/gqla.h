@@ -232,15 +232,16 @@ gqla_status gqla_quantize_rows_e4m3(gqla_dtype src_dtype, int64_t rows, int32_t 
                                     float pre_b, const void* src, uint8_t* dst, float* row_scale, void* stream);
 /* Eq. (mqa), lines 3-5, over an E4M3 latent cache:  q8 [B, s_q, h_q, r_kv+d_r] codes, q_scale [B, s_q, h_q] fp32,
  * cache8 [N, r_kv+d_r] codes with row stride cache_row_stride (bytes), v_scale = the latent plane's scale.
- * Fixed split plan only (num_splits >= 1).  Outputs and the other arguments as for gqla_decode_absorb. */
+ * num_splits as for gqla_decode_absorb (>= 1 fixed plan, <= -2 balanced).  Outputs and the other arguments as
+ * for gqla_decode_absorb. */
 gqla_status gqla_decode_absorb_fp8(const gqla_dims* dims, int32_t B, int32_t s_q, float scale, int32_t num_splits,
                                    const uint8_t* q8, const float* q_scale, const uint8_t* cache8,
                                    int64_t cache_row_stride, int64_t cache_rows, float v_scale, const int64_t* seq_start,
                                    const int32_t* seqlens, float* o_part, float* lse_part, int32_t* status_word,
                                    void* stream);
 /* Eq. (mha) over E4M3 planes:  q8 [B, s_q, h_q, d_h+d_r], q_scale [B, s_q, h_q];  k_c8, v8 [N, g, d_h];
- * k_r8 [N, .] with row stride k_r_row_stride (bytes);  v_scale = the V plane's scale.  Fixed split plan only.
- * Outputs and the other arguments as for gqla_decode_gqa. */
+ * k_r8 [N, .] with row stride k_r_row_stride (bytes);  v_scale = the V plane's scale.  num_splits as for
+ * gqla_decode_gqa.  Outputs and the other arguments as for gqla_decode_gqa. */
 gqla_status gqla_decode_gqa_fp8(const gqla_dims* dims, int32_t B, int32_t s_q, float scale, int32_t num_splits,
                                 const uint8_t* q8, const float* q_scale, const uint8_t* k_c8, const uint8_t* v8,
                                 const uint8_t* k_r8, int64_t k_r_row_stride, int64_t n_rows, float v_scale,

@@ -540,12 +540,14 @@ gqla_status gqla_quantize_rows_e4m3(gqla_dtype src_dtype, int64_t rows, int32_t 
     return launch_status();
 }
 
+// S >= 1: fixed split plan;  S <= -2: balanced plan with -S slots (tensor-core kernels; the generic ones run the
+// fixed plan with -S splits, also a valid set of partials)
 static gqla_status check_fp8_common(const gqla_dims* d, int32_t B, int32_t s_q, int32_t S, const void* q8,
                                     const float* q_scale, float v_scale, const int64_t* seq_start, const int32_t* seqlens,
                                     const float* o_part, const float* lse_part) {
     gqla_status s;
     if ((s = check_dims(d)) != GQLA_OK) return s;
-    if (B < 0 || s_q < 1 || S < 1 || !(v_scale > 0.f)) return GQLA_ERR_SHAPE;
+    if (B < 0 || s_q < 1 || S == 0 || S == -1 || !(v_scale > 0.f)) return GQLA_ERR_SHAPE;
     if (B == 0) return GQLA_OK;
     if (q8 == nullptr || q_scale == nullptr || seq_start == nullptr || seqlens == nullptr || o_part == nullptr ||
         lse_part == nullptr)
@@ -572,7 +574,7 @@ gqla_status gqla_decode_absorb_fp8(const gqla_dims* d, int32_t B, int32_t s_q, f
     a.kB = nullptr; a.kB_stride = 0; a.dB = 0;
     a.v = cache8; a.v_stride = cache_row_stride; a.v_gstride = 0; a.dv = d->r_kv;
     a.rows = packed_rows(seq_start); a.seqlens = seqlens;
-    a.B = B; a.S = num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
+    a.B = B; a.S = num_splits < 0 ? -num_splits : num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
     a.scale = scale; a.o_part = o_part; a.lse_part = lse_part; a.q_row_scale = q_scale; a.v_scale = v_scale;
     return launch_decode_generic_fp8(a, st);
 }
@@ -589,14 +591,18 @@ gqla_status gqla_decode_gqa_fp8(const gqla_dims* d, int32_t B, int32_t s_q, floa
     if (!aligned16(k_c8) || !aligned16(v8) || !aligned16(k_r8)) return GQLA_ERR_ALIGN;
     if ((d->d_r > 0 && k_r_row_stride < d->d_r) || n_rows < 0) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
-    (void)status_word;
+    if (g_policy.load() == GQLA_POLICY_AUTO) {
+        s = tc_decode_gqa_fp8(*d, B, s_q, scale, num_splits, q8, q_scale, k_c8, v8, k_r8, k_r_row_stride, n_rows, v_scale,
+                              packed_rows(seq_start), seqlens, o_part, lse_part, status_word, st);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
     DecodeArgs a{};
     a.q = q8;
     a.kA = k_c8; a.kA_stride = (int64_t)d->g * d->d_h; a.kA_gstride = d->d_h; a.dA = d->d_h;
     a.kB = k_r8; a.kB_stride = k_r_row_stride; a.dB = d->d_r;
     a.v = v8; a.v_stride = (int64_t)d->g * d->d_h; a.v_gstride = d->d_h; a.dv = d->d_h;
     a.rows = packed_rows(seq_start); a.seqlens = seqlens;
-    a.B = B; a.S = num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
+    a.B = B; a.S = num_splits < 0 ? -num_splits : num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
     a.scale = scale; a.o_part = o_part; a.lse_part = lse_part; a.q_row_scale = q_scale; a.v_scale = v_scale;
     return launch_decode_generic_fp8(a, st);
 }

@@ -6,6 +6,7 @@
 #include "common.cuh"
 #include "tc_decode_absorb.cuh"
 #include "tc_decode_gqa.cuh"
+#include "tc_decode_gqa_fp8.cuh"
 #include "tc_append.cuh"
 #include "tc_combine_up.cuh"
 #include "tc_expand.cuh"
@@ -425,6 +426,72 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
         case 32: e = gqa_launch<32>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
         case 64: e = gqa_launch<64>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
         case 128: e = gqa_launch<128>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
+        default: return GQLA_ERR_UNSUPPORTED;
+    }
+    return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
+}
+
+template <int R>
+inline cudaError_t gqa_fp8_launch(const tc::GqaFp8Params& p, const CUtensorMap& qc, const CUtensorMap& qr, const CUtensorMap& k,
+                                  const CUtensorMap& r, const CUtensorMap& v, unsigned grid, cudaStream_t st) {
+    auto kern = tc::decode_gqa_fp8_tc_kernel<R>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::GqaFp8Smem::kTotal);
+    if (e != cudaSuccess) return e;
+    return tc::launch_pdl(kern, dim3(grid), dim3(tc::GqaFp8Smem::kThreads), tc::GqaFp8Smem::kTotal, st, p, qc, qr, k, r, v);
+}
+
+// GQA path over E4M3 planes; covers what the bf16 tensor-core kernel covers (d_h = 128, d_r = 64, at most 128 rows
+// per group).  Strides are in bytes here (one byte per element) and must be multiples of 16.
+inline gqla_status tc_decode_gqa_fp8(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S, const uint8_t* q8,
+                                     const float* q_scale, const uint8_t* k_c8, const uint8_t* v8, const uint8_t* k_r8,
+                                     int64_t k_r_row_stride, int64_t n_rows, float v_scale, const RowMap& rows,
+                                     const int32_t* seqlens, float* o_part, float* lse_part, int32_t* status,
+                                     cudaStream_t st) {
+    if (!tc_covers(d, GQLA_BF16, s_q, 1) || k_r_row_stride % 16 != 0 || n_rows > 0x7fffffffLL || n_rows < 1)
+        return GQLA_ERR_UNSUPPORTED;
+    const int32_t workers = S < 0 ? tc_balanced_workers(d, s_q, 1) : 0;
+    const bool balanced = S < 0 && workers > 0;
+    if (S < 0) S = -S;
+    const int64_t units = balanced ? (int64_t)workers * d.g : (int64_t)B * S * d.g;
+    if (units > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
+    const int hpg = d.h_q / d.g;
+    int hpg_box = 0, sq_box = 0;
+    const int R = gqa_rows(d, s_q, &hpg_box, &sq_box);
+    CUtensorMap tmQc, tmQr, tmK, tmR, tmV;
+    {
+        const int feat = d.d_h + d.d_r;
+        const uint64_t dims[4] = {(uint64_t)feat, (uint64_t)hpg, (uint64_t)d.g, (uint64_t)B * s_q};
+        const uint64_t str[3] = {(uint64_t)feat, (uint64_t)hpg * feat, (uint64_t)d.h_q * feat};
+        const uint32_t box_c[4] = {128, (uint32_t)hpg_box, 1, (uint32_t)sq_box};
+        const uint32_t box_r[4] = {64, (uint32_t)hpg_box, 1, (uint32_t)sq_box};
+        if (!tc::make_tmap_u8(&tmQc, q8, 4, dims, str, box_c, CU_TENSOR_MAP_SWIZZLE_128B)) return GQLA_ERR_CUDA;
+        if (!tc::make_tmap_u8(&tmQr, q8, 4, dims, str, box_r, CU_TENSOR_MAP_SWIZZLE_64B)) return GQLA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[3] = {(uint64_t)d.d_h, (uint64_t)d.g, (uint64_t)n_rows};
+        const uint64_t str[2] = {(uint64_t)d.d_h, (uint64_t)d.g * d.d_h};
+        const uint32_t box[3] = {128, 1, 128};
+        if (!tc::make_tmap_u8(&tmK, k_c8, 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return GQLA_ERR_CUDA;
+        if (!tc::make_tmap_u8(&tmV, v8, 3, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return GQLA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)d.d_r, (uint64_t)n_rows};
+        const uint64_t str[1] = {(uint64_t)k_r_row_stride};
+        const uint32_t box[2] = {64, 128};
+        if (!tc::make_tmap_u8(&tmR, k_r8, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_64B)) return GQLA_ERR_CUDA;
+    }
+    tc::GqaFp8Params p{};
+    p.B = B; p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpg_box = hpg_box;
+    p.balanced = balanced ? 1 : 0; p.W = workers;
+    p.scale_log2 = scale * 1.4426950408889634f; p.v_scale = v_scale; p.q_scale = q_scale;
+    p.rows = rows; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
+    cudaError_t e;
+    switch (R) {
+        case 8: e = gqa_fp8_launch<8>(p, tmQc, tmQr, tmK, tmR, tmV, (unsigned)units, st); break;
+        case 16: e = gqa_fp8_launch<16>(p, tmQc, tmQr, tmK, tmR, tmV, (unsigned)units, st); break;
+        case 32: e = gqa_fp8_launch<32>(p, tmQc, tmQr, tmK, tmR, tmV, (unsigned)units, st); break;
+        case 64: e = gqa_fp8_launch<64>(p, tmQc, tmQr, tmK, tmR, tmV, (unsigned)units, st); break;
+        case 128: e = gqa_fp8_launch<128>(p, tmQc, tmQr, tmK, tmR, tmV, (unsigned)units, st); break;
         default: return GQLA_ERR_UNSUPPORTED;
     }
     return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
