@@ -567,7 +567,11 @@ gqla_status gqla_decode_absorb_fp8(const gqla_dims* d, int32_t B, int32_t s_q, f
     if (!aligned16(cache8)) return GQLA_ERR_ALIGN;
     if (cache_row_stride < d->r_kv + d->d_r || cache_rows < 0) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
-    (void)status_word;
+    if (g_policy.load() == GQLA_POLICY_AUTO) {
+        s = tc_decode_absorb_fp8(*d, B, s_q, scale, num_splits, q8, q_scale, cache8, cache_row_stride, cache_rows, v_scale,
+                                 packed_rows(seq_start), seqlens, o_part, lse_part, status_word, st);
+        if (s != GQLA_ERR_UNSUPPORTED) return s;
+    }
     DecodeArgs a{};
     a.q = q8;
     a.kA = cache8; a.kA_stride = cache_row_stride; a.kA_gstride = 0; a.dA = d->r_kv + d->d_r;

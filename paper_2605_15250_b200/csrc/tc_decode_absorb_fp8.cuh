@@ -1,0 +1,550 @@
+// Absorb-path split-KV flash decoding over an FP8 (E4M3) latent cache on tcgen05 (Eq. (mqa), lines 3-5; KV-cache
+// quantisation is among the effects the paper's model leaves out, Sec. 5.1 "Limitations").  The CTA-pair design
+// of tc_decode_absorb.cuh (2-CTA cluster, cta_group::2 MMAs of M = 128, each CTA holding 64 query rows, O in 256
+// TMEM columns, S in 64) with what one byte per element changes:
+//
+//   * MMAs are kind::f8f6f4 (E4M3 x E4M3 -> fp32), K = 32 per instruction: twice the contraction per instruction.
+//   * A [64 rows x 128 bytes] box now spans 128 latent columns.  Qh and this CTA's 64 cache rows of a tile are
+//     four such boxes plus one [64 x 64 bytes] RoPE box (64-byte swizzle); a V group (one token half of a tile,
+//     this CTA's 128 of every 256 latent columns) is two boxes.  A tile is 36 KB of K and 32 KB of V per CTA
+//     instead of 72 + 64, so both rings are two tiles deep in less shared memory than the bf16 kernel needs for one.
+//   * Scores are scaled per query row (q_scale, which folds the cache planes' scales in), outputs by v_scale.
+//   * P is rounded to E4M3; the softmax reference is held kAF8Bias binades below the running maximum and follows
+//     it as soon as it has grown by more than one binade, so that P <= 2^8 and terms down to 2^-16 of the largest
+//     one still count (the format's smallest positive value is 2^-9).
+#pragma once
+#include "common.cuh"
+#include "sched.cuh"
+#include "tc_common.cuh"
+#include "tc_decode_gqa_fp8.cuh"  // E4M3 descriptors, packing
+
+namespace gqla {
+namespace tc {
+
+struct AbsorbFp8Params {
+    int32_t B, S, s_q, h_q, rows_total /* s_q*h_q */, row_blocks /* ceil(rows_total/128) */;
+    int32_t balanced, W;  // balanced plan: W pairs per row block, grid = 2 * W * row_blocks
+    float scale_log2, v_scale;
+    const float* q_scale;  // [B, s_q * h_q]
+    RowMap rows;      // packed or paged (pages a multiple of 128 rows, pieces starting on tile boundaries)
+    const int32_t* seqlens;
+    float* o_part;    // [B, S, s_q*h_q, 512]
+    float* lse_part;  // [B, S, s_q*h_q]
+    __nv_bfloat16* o_final;  // not null: S = 1, fixed plan; the normalised output goes here as bf16 [B, s_q*h_q, 512]
+                             // (o_part unused, lse_part may be null)
+    int32_t* status;
+};
+
+struct AbsorbFp8Smem {
+    static constexpr int kBox = 8192;              // 64 rows x 128 E4M3, 128-byte swizzle
+    static constexpr int kRBox = 4096;             // 64 rows x 64 E4M3 (RoPE part), 64-byte swizzle
+    static constexpr int kQBytes = 4 * kBox + kRBox;  // 64 query rows x 576
+    static constexpr int kPBytes = kBox;           // 64 rows x 128 tokens
+    static constexpr int kKGroup = 2 * kBox + kRBox;  // group 0: latent boxes 0, 1;  group 1: boxes 2, 3 and the RoPE box
+    static constexpr int kVGroup = 2 * kBox;       // 64 tokens x this CTA's 2 x 128 latent columns
+    static constexpr int kKGroupsPerTile = 2;
+    static constexpr int kNK = 4;                  // ring of K groups: two tiles
+    static constexpr int kNV = 4;                  // ring of V groups: two tiles
+    static constexpr int kOffQ = 0;
+    static constexpr int kOffP = 37 * 1024;        // behind Qh (36 KB), 1 KB aligned
+    static constexpr int kOffV = kOffP + kPBytes;  // P and the V ring are contiguous: together the output staging
+    static constexpr int kOffK = kOffV + kNV * kVGroup;
+    static constexpr int kTileBytes = kOffK + kNK * kKGroup;
+    // kfull[kNK] kempty[kNK] vfull[kNV] vempty[kNV] q_full q_empty o_free epi_done s_full[2] p_ready[2]
+    // pv_done[2] xch[2] fin epi
+    static constexpr int kNumBars = 2 * kNK + 2 * kNV + 14;
+    static constexpr int kSoftmaxWarps = 8;
+    static constexpr int kVProducerWarp = 2 + kSoftmaxWarps;
+    static constexpr int kThreads = 96 + 32 * kSoftmaxWarps;
+    static constexpr int kOutPitch = 256 * 4 + 16;
+    static_assert(64 * kOutPitch <= kPBytes + kNV * kVGroup, "output staging must fit in P + V ring");
+    static_assert(kKGroup % 1024 == 0 && kOffP % 1024 == 0, "swizzled tiles need 1 KB alignment");
+    static constexpr int kTotal = kTileBytes + kNumBars * 8 + 16 + 2 * 4 * 64 * 4;
+    static_assert(2 * 4 * 64 >= kThreads + 4, "plan scratch must fit in sm_max");
+    static_assert(kTotal <= 232448, "shared memory budget of one CTA");
+    static_assert(OneCtaPerSM<kTotal>::value, "");
+};
+
+constexpr uint32_t kA8ColO = 0;    // O: MMA m (latent columns [256m, 256m+256)) at TMEM columns [128m, 128m+128)
+constexpr uint32_t kA8ColS = 256;  // two 64-column score buffers
+constexpr float kAF8Bias = 7.0f;     // log2 units the softmax reference sits below the running maximum
+constexpr float kAF8Refresh = 1.0f;  // the reference follows the maximum once it has grown by this much
+constexpr uint32_t kDescHiSw64 = (uint32_t)(((1ull << 46) | (4ull << 61) | ((uint64_t)(512 >> 4) << 32)) >> 32);
+// cta_group::2 MMA of kind::f8f6f4; descriptors as (low word, constant high word of their swizzle mode).
+template <bool ACCUMULATE>
+__device__ __forceinline__ void umma_f8_ss2_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t hi) {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
+        "mov.b64 da, {%1, %4};\n\tmov.b64 db, {%2, %4};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(hi), "n"(ACCUMULATE ? 1 : 0)
+        : "memory");
+}
+
+template <int DUMMY>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(AbsorbFp8Smem::kThreads, 1)
+decode_absorb_fp8_tc_kernel(const AbsorbFp8Params p, const __grid_constant__ CUtensorMap tmQ,
+                            const __grid_constant__ CUtensorMap tmQr, const __grid_constant__ CUtensorMap tmC,
+                            const __grid_constant__ CUtensorMap tmCr) {
+    using L = AbsorbFp8Smem;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* tiles = smem_raw;
+    if ((smem_u32(tiles) & 1023u) != 0) {  // swizzled tiles need 1 KB alignment; same answer in both CTAs
+        if (threadIdx.x == 0 && p.status != nullptr) atomicCAS(p.status, 0, kStatusTimeout | (15 << 8));
+        return;
+    }
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + L::kTileBytes);
+    uint64_t* kfull = bars;
+    uint64_t* kempty = kfull + L::kNK;
+    uint64_t* vfull = kempty + L::kNK;
+    uint64_t* vempty = vfull + L::kNV;
+    uint64_t* q_full = vempty + L::kNV;
+    uint64_t* q_empty = q_full + 1;    // every Qh Kh^T of a piece has completed: Q may be overwritten
+    uint64_t* o_free = q_empty + 1;    // leader only: both CTAs' softmax warps have read O of a piece
+    uint64_t* epi_done = o_free + 1;   // this CTA's output staging (P + V ring) is free again
+    uint64_t* s_full = epi_done + 1;   // [2]
+    uint64_t* p_ready = s_full + 2;    // [2] leader only: one arrival per softmax warp of the pair
+    uint64_t* pv_done = p_ready + 2;   // [2]
+    uint64_t* xch = pv_done + 2;       // [2] softmax warps of this CTA: per-tile max exchange
+    uint64_t* fin = xch + 2;           //     the final partial-sum exchange of a piece
+    uint64_t* epi = fin + 1;           //     and the steps of the output staging
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + L::kNumBars);
+    volatile int32_t* abort_flag = reinterpret_cast<volatile int32_t*>(tmem_slot + 1);
+    float* sm_max = reinterpret_cast<float*>(tmem_slot + 4);  // [2][4][64] per-tile partial maxima
+    // [4][64] final partial sums; written only after the last P.V of a piece, i.e. after every warp has
+    // arrived on p_ready of its last tile and hence finished reading sm_max
+    float* sm_l = sm_max;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta = cluster_ctarank();  // 0 = leader
+    const Abort ab{abort_flag, p.status};
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < L::kNumBars; ++i) {
+            uint64_t* bar = &bars[i];
+            const bool pair_wide = bar == &p_ready[0] || bar == &p_ready[1] || bar == o_free;
+            const bool cta_wide = bar == &xch[0] || bar == &xch[1] || bar == fin || bar == epi || bar == epi_done;
+            mbar_init(bar, pair_wide ? 2 * L::kSoftmaxWarps : (cta_wide ? L::kSoftmaxWarps : 1));
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc2(tmem_slot, 512);
+        tmem_relinquish2();
+    }
+
+    pdl_launch_dependents();
+    pdl_wait();  // barriers and TMEM are set up; everything below reads the caller's tensors
+    // the plan of this pair: row block rb, and either one (sequence, split) piece or worker w's share
+    const int pair = blockIdx.x >> 1;
+    const int rb = pair % p.row_blocks;
+    Walker walk;
+    if (p.balanced) {
+        const BalancedStart st = balanced_prepass(p.seqlens, p.B, p.S, pair / p.row_blocks, p.W,
+                                                  reinterpret_cast<int32_t*>(sm_max), L::kThreads);
+        walk.init_balanced(p.seqlens, p.B, p.S, pair / p.row_blocks, p.W, st);
+    } else {
+        const int unit = pair / p.row_blocks;
+        walk.init_fixed(p.seqlens, p.B, p.S, unit / p.S, unit % p.S);
+    }
+    const int rho0 = rb * 128 + (int)cta * 64;  // first (query, head) row of this CTA
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync();  // both CTAs' barriers exist before any remote arrival
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    Piece pc;
+    int pi = 0;  // non-empty pieces walked so far (phase of the per-piece barriers)
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer of Q and the K ring
+        // (both CTAs).  Every "full" barrier lives in the leader and counts the bytes of BOTH CTAs.
+        if (elect_one()) {
+            tma_prefetch_desc(&tmQ);
+            tma_prefetch_desc(&tmQr);
+            tma_prefetch_desc(&tmC);
+            tma_prefetch_desc(&tmCr);
+            const uint32_t q_full_l = mapa(smem_u32(q_full), 0);
+            int ks = 0;
+            uint32_t kph = 1;  // parity that means "slot is free"
+            bool ok = true;
+            while (ok && walk.next(pc)) {
+                if (pc.n_tiles == 0) continue;
+                // Q rows of this piece's sequence; the previous piece's Qh Kh^T must all have completed
+                if (pi > 0 && !(ok = mbar_wait(q_empty, (pi - 1) & 1, ab, 13))) break;
+                if (cta == 0) mbar_expect_tx(q_full, 2 * L::kQBytes);
+                for (int kb = 0; kb < 4; ++kb)
+                    tma_load_2d_pair(tiles + kb * L::kBox, &tmQ, kb * 128, pc.b * p.rows_total + rho0, q_full_l);
+                tma_load_2d_pair(tiles + 4 * L::kBox, &tmQr, 512, pc.b * p.rows_total + rho0, q_full_l);
+                // K groups in the order (tile, column half); a tile never straddles a page
+                int64_t tile_row = p.rows.row(pc.b, pc.tok_begin);
+                for (int kt = 0; kt < pc.n_tiles && ok; ++kt) {
+                    const int32_t row = (int32_t)(tile_row + cta * 64);
+                    // the next tile's row is fetched while this tile's slots are waited for
+                    if (kt + 1 < pc.n_tiles)
+                        tile_row = p.rows.paged() ? p.rows.row(pc.b, pc.tok_begin + (kt + 1) * 128) : tile_row + 128;
+#pragma unroll 1
+                    for (int kg = 0; kg < 2; ++kg) {
+                        if (!(ok = mbar_wait(&kempty[ks], kph, ab, 1))) break;
+                        // group 0: latent boxes 0, 1;  group 1: latent boxes 2, 3 and the RoPE box
+                        if (cta == 0) mbar_expect_tx(&kfull[ks], 2 * (2 * L::kBox + (kg == 1 ? L::kRBox : 0)));
+                        const uint32_t bar = mapa(smem_u32(&kfull[ks]), 0);
+                        uint8_t* dst = tiles + L::kOffK + ks * L::kKGroup;
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) tma_load_2d_pair(dst + i * L::kBox, &tmC, (2 * kg + i) * 128, row, bar);
+                        if (kg == 1) tma_load_2d_pair(dst + 2 * L::kBox, &tmCr, 512, row, bar);
+                        if (++ks == L::kNK) { ks = 0; kph ^= 1; }
+                    }
+                }
+                ++pi;
+            }
+        }
+    } else if (warp == L::kVProducerWarp) {
+        // ------------------------------------------------------------------ TMA producer of the V ring (both
+        // CTAs).  A thread issues a tensor load only every few hundred cycles, and a tile needs 17 of them:
+        // the two rings are fed by two threads.  V groups in the order (tile, token half); a V slot is free
+        // only after P.V of the previous tile, i.e. after Qh Kh^T of this tile has read the same cache rows
+        // as K boxes, so the V boxes come out of L2.
+        if (elect_one()) {
+            int vs = 0;
+            uint32_t vph = 1;
+            bool ok = true;
+            while (ok && walk.next(pc)) {
+                if (pc.n_tiles == 0) continue;
+                // the V ring doubles as the output staging of the previous piece
+                if (pi > 0 && !(ok = mbar_wait(epi_done, (pi - 1) & 1, ab, 16))) break;
+                int64_t tile_row = p.rows.row(pc.b, pc.tok_begin);
+                for (int vt = 0; vt < pc.n_tiles && ok; ++vt) {
+                    const int64_t row0 = tile_row;
+                    if (vt + 1 < pc.n_tiles)
+                        tile_row = p.rows.paged() ? p.rows.row(pc.b, pc.tok_begin + (vt + 1) * 128) : tile_row + 128;
+#pragma unroll 1
+                    for (int vh = 0; vh < 2; ++vh) {
+                        if (!(ok = mbar_wait(&vempty[vs], vph, ab, 2))) break;
+                        if (cta == 0) mbar_expect_tx(&vfull[vs], 2 * L::kVGroup);
+                        const int32_t row = (int32_t)(row0 + vh * 64);
+                        const uint32_t bar = mapa(smem_u32(&vfull[vs]), 0);
+                        uint8_t* dst = tiles + L::kOffV + vs * L::kVGroup;
+                        // box m: latent columns [256m + 128cta, +128) -- this CTA's half of MMA m's N
+#pragma unroll
+                        for (int m = 0; m < 2; ++m) tma_load_2d_pair(dst + m * L::kBox, &tmC, 256 * m + 128 * (int)cta, row, bar);
+                        if (++vs == L::kNV) { vs = 0; vph ^= 1; }
+                    }
+                }
+                ++pi;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (cta == 0 && elect_one()) {
+            constexpr uint32_t idesc_qk = idesc_e4m3(128, 128, 0, 0);
+            constexpr uint32_t idesc_pv = idesc_e4m3(128, 256, 0, 1);
+            const uint32_t q_lo = desc_lo(desc_kmajor_sw128(smem_u32(tiles)));
+            const uint32_t qr_lo = desc_lo(desc_kmajor_sw64(smem_u32(tiles + 4 * L::kBox)));
+            const uint32_t p_lo = desc_lo(desc_kmajor_sw128(smem_u32(tiles + L::kOffP)));
+            int ks = 0, vs = 0;
+            uint32_t kph = 0, vph = 0;
+            int gt = 0;  // tiles issued so far: score buffer = gt & 1, phase = (gt >> 1) & 1
+            auto issue_qk = [&](int n) -> bool {
+                const uint32_t d = tmem_base + kA8ColS + (uint32_t)(n & 1) * 64;
+#pragma unroll 1
+                for (int g2 = 0; g2 < 2; ++g2) {
+                    if (!mbar_wait(&kfull[ks], kph, ab, 3)) return false;
+                    tc_fence_after();
+                    const uint32_t kd = desc_lo(desc_kmajor_sw128(smem_u32(tiles + L::kOffK + ks * L::kKGroup)));
+                    const uint32_t qd = q_lo + ((g2 * 2 * L::kBox) >> 4);
+                    if (g2 == 0)
+                        umma_f8_ss2_lo<false>(d, qd, kd, idesc_qk, kDescHiSw128);  // the tile's first MMA overwrites S
+                    else
+                        umma_f8_ss2_lo<true>(d, qd, kd, idesc_qk, kDescHiSw128);
+#pragma unroll
+                    for (int i = 0; i < 2; ++i)
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            if ((i | kk) != 0)
+                                umma_f8_ss2_lo<true>(d, qd + ((i * L::kBox + kk * 32) >> 4), kd + ((i * L::kBox + kk * 32) >> 4),
+                                                     idesc_qk, kDescHiSw128);
+                    if (g2 == 1) {  // the RoPE part: 64 elements = 2 x 32, 64-byte swizzle
+                        const uint32_t krd = desc_lo(desc_kmajor_sw64(smem_u32(tiles + L::kOffK + ks * L::kKGroup + 2 * L::kBox)));
+#pragma unroll
+                        for (int kk = 0; kk < 2; ++kk)
+                            umma_f8_ss2_lo<true>(d, qr_lo + ((kk * 32) >> 4), krd + ((kk * 32) >> 4), idesc_qk, kDescHiSw64);
+                    }
+                    umma_commit2(&kempty[ks], 3);
+                    if (++ks == L::kNK) { ks = 0; kph ^= 1; }
+                }
+                umma_commit2(&s_full[n & 1], 3);
+                return true;
+            };
+            bool ok = true;
+            while (ok && walk.next(pc)) {
+                if (pc.n_tiles == 0) continue;
+                if (!(ok = mbar_wait(q_full, pi & 1, ab, 4))) break;
+                tc_fence_after();
+                if (!(ok = issue_qk(gt))) break;
+                for (int t = 0; t < pc.n_tiles && ok; ++t) {
+                    const int n = gt + t;
+                    if (t + 1 < pc.n_tiles) {
+                        if (!(ok = issue_qk(n + 1))) break;
+                    } else {
+                        umma_commit2(q_empty, 3);  // every Qh Kh^T of this piece has been issued
+                    }
+                    if (!(ok = mbar_wait(&p_ready[n & 1], (n >> 1) & 1, ab, 5))) break;
+                    // the first P.V of a piece overwrites O: the previous piece's O must have been read
+                    if (t == 0 && pi > 0 && !(ok = mbar_wait(o_free, (pi - 1) & 1, ab, 14))) break;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int h = 0; h < 2; ++h) {
+                        if (!(ok = mbar_wait(&vfull[vs], vph, ab, 6))) break;
+                        tc_fence_after();
+                        // V box m: [64 tokens x 128 latent columns], MN-major; a k-step is 32 token rows (4 KB)
+                        const uint32_t vd = desc_lo(desc_mnmajor_sw128(smem_u32(tiles + L::kOffV + vs * L::kVGroup), L::kBox));
+                        const uint32_t pd = p_lo + ((h * 64) >> 4);  // tokens [64h, 64h + 64) of the P rows
+#pragma unroll
+                        for (int m = 0; m < 2; ++m) {
+                            const uint32_t dm = tmem_base + kA8ColO + (uint32_t)m * 128;
+                            if ((t | h) == 0)
+                                umma_f8_ss2_lo<false>(dm, pd, vd + ((m * L::kBox) >> 4), idesc_pv, kDescHiSw128);  // first P.V of a piece
+                            else
+                                umma_f8_ss2_lo<true>(dm, pd, vd + ((m * L::kBox) >> 4), idesc_pv, kDescHiSw128);
+                            umma_f8_ss2_lo<true>(dm, pd + (32 >> 4), vd + ((m * L::kBox + 4096) >> 4), idesc_pv, kDescHiSw128);
+                        }
+                        umma_commit2(&vempty[vs], 3);
+                        if (++vs == L::kNV) { vs = 0; vph ^= 1; }
+                    }
+                    if (ok) umma_commit2(&pv_done[n & 1], 3);
+                }
+                gt += pc.n_tiles;
+                ++pi;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax
+        const int q = warp & 3;              // TMEM lane quadrant this warp may access
+        const int ch = (warp - 2) >> 2;      // which 32 of the lane's 64 score columns
+        const int Lr = q * 32 + lane;        // TMEM lane
+        const int r = Lr & 63;               // row within this CTA
+        const int hf = Lr >> 6;              // token half of each 128-token tile / column half of each O block
+        const int part = hf * 2 + ch;        // one of the four threads of row r
+        const int rho = rho0 + r;            // (query, head) row of the sequence
+        const bool row_valid = rho < p.rows_total;
+        const int pq = row_valid ? rho / p.h_q : 0;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t p_ready_l[2] = {mapa(smem_u32(&p_ready[0]), 0), mapa(smem_u32(&p_ready[1]), 0)};
+        const uint32_t o_free_l = mapa(smem_u32(o_free), 0);
+        int gt = 0;  // tiles walked so far
+        int ec = 0;  // completed phases of the `epi` barrier
+
+        while (walk.next(pc)) {
+            const int32_t T = p.seqlens[pc.b];
+            const int64_t slot0 = (int64_t)pc.b * p.S;
+            // split slots this worker marks empty
+            if (part == 0 && row_valid && p.lse_part != nullptr)
+                for (int kk = pc.fill_begin; kk < pc.fill_end; ++kk) p.lse_part[(slot0 + kk) * p.rows_total + rho] = -INFINITY;
+            if (pc.n_tiles == 0 && p.balanced) continue;  // an empty sequence: its slots were marked above
+            int32_t lim = visible_limit(T, p.s_q, pq);
+            if (lim > pc.tok_end) lim = pc.tok_end;
+            lim -= pc.tok_begin;
+            if (!row_valid) lim = 0;
+            // the row's score scale: softmax scale x log2(e) x the query row's quantisation scale
+            const float sl2 = p.scale_log2 * (row_valid ? p.q_scale[(int64_t)pc.b * p.rows_total + rho] : 1.f);
+            float m_used = -INFINITY, l = 0.f;
+            bool ok = true;
+
+            for (int t = 0; t < pc.n_tiles && ok; ++t) {
+                const int n = gt + t;
+                const int sb = n & 1;
+                const uint32_t nph = (n >> 1) & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(&s_full[sb], nph, ab, 7));
+                if (!ok) break;
+                tc_fence_after();
+                const int tok0 = t * 128 + hf * 64 + ch * 32;
+                uint32_t x[32];
+                tmem_ld32(lane_base + kA8ColS + (uint32_t)sb * 64 + ch * 32, x);
+                tmem_wait_ld();
+                const bool full = tok0 + 32 <= lim;  // every score of this thread is visible
+                float mx = -INFINITY;
+                if (full) {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(x[c]));
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (tok0 + c < lim) mx = fmaxf(mx, __uint_as_float(x[c]));
+                }
+                // the other three parts of this row live in other warps
+                float* mxs = sm_max + sb * 256;
+                mxs[part * 64 + r] = mx;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&xch[sb]);
+                ok = __all_sync(0xffffffffu, mbar_wait(&xch[sb], nph, ab, 10));
+                if (!ok) break;
+                mx = fmaxf(fmaxf(mxs[r], mxs[64 + r]), fmaxf(mxs[128 + r], mxs[192 + r]));
+                const float m_t = mx * sl2;
+                const bool need = m_t > m_used + kAF8Refresh;
+                const float factor = need ? ex2(m_used - m_t) : 1.f;
+                if (need) {
+                    l *= factor;
+                    m_used = m_t;
+                }
+                // exponent offset: the reference sits kAF8Bias binades below the (lazily tracked) maximum
+                const float m_sub = m_used == -INFINITY ? 0.f : m_used - kAF8Bias;
+                uint32_t pk[8];
+#pragma unroll
+                for (int c = 0; c < 32; c += 4) {
+                    float e[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        e[i] = (full || tok0 + c + i < lim) ? ex2(fmaf(__uint_as_float(x[c + i]), sl2, -m_sub)) : 0.f;
+                        l += e[i];
+                    }
+                    pk[c / 4] = pack_e4m3x4(e[0], e[1], e[2], e[3]);
+                }
+                // O may be rescaled, and the P buffer rewritten, only once P.V(n-1) has completed
+                if (t > 0) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, ab, 8));
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                if (__any_sync(0xffffffffu, need) && t > 0) {
+                    // this thread's share of the lane's O: columns [128m + 64ch, +64) for m = 0, 1
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t col = kA8ColO + (uint32_t)(c >> 1) * 128 + ch * 64 + (c & 1) * 32;
+                        uint32_t o[32];
+                        tmem_ld32(lane_base + col, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                        tmem_st32(lane_base + col, o);
+                    }
+                    tmem_wait_st();
+                }
+                // P row r: 128 bytes = 128 tokens = 8 chunks of 16 E4M3, chunk index XORed with (r & 7); this
+                // thread's 32 tokens are chunks 4 hf + 2 ch and the next one
+                uint8_t* prow = tiles + L::kOffP + r * 128;
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2)
+                    *reinterpret_cast<uint4*>(prow + (((hf * 4 + ch * 2 + c2) ^ (r & 7)) << 4)) =
+                        make_uint4(pk[4 * c2], pk[4 * c2 + 1], pk[4 * c2 + 2], pk[4 * c2 + 3]);
+                fence_proxy_async_smem();  // generic-proxy writes of P -> visible to the tensor core
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(p_ready_l[sb]);
+            }
+
+            // -------------------------------------------------------------- epilogue: normalise and store
+            const int n_last = gt + pc.n_tiles - 1;
+            if (pc.n_tiles > 0 && ok)
+                ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[n_last & 1], (n_last >> 1) & 1, ab, 9));
+            tc_fence_after();
+            sm_l[part * 64 + r] = l;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(fin);
+            if (!__all_sync(0xffffffffu, mbar_wait(fin, pi & 1, ab, 11))) ok = false;
+            const float Lt = (sm_l[r] + sm_l[64 + r]) + (sm_l[128 + r] + sm_l[192 + r]);
+            const bool live = ok && pc.n_tiles > 0 && Lt > 0.f && m_used > -INFINITY;
+            const float inv = live ? p.v_scale / Lt : 0.f;
+            // The CTA's 64 output rows leave through shared memory (P and the V ring are idle now: the last
+            // P.V has completed) as 1 KB bulk stores, the 256 columns of MMA m = 0 first, then those of m = 1.
+            // The padded pitch keeps the 16-byte stores of a quarter warp on distinct banks.
+            uint8_t* stage = tiles + L::kOffP;
+            if (p.o_final != nullptr) {
+                // whole-sequence call: the final bf16 rows (1 KB each) fit the staging at once -- one pass
+                uint4* dst = reinterpret_cast<uint4*>(stage + r * L::kOutPitch + (128 * hf + 64 * ch) * 2);
+#pragma unroll 1
+                for (int mc = 0; mc < 4; ++mc) {  // (m, 32-column half) of this thread's 64 columns of each m
+                    const int m = mc >> 1, c = (mc & 1) * 32;
+                    uint32_t o[32];
+                    if (pc.n_tiles > 0 && ok) {  // warp-uniform
+                        tmem_ld32(lane_base + kA8ColO + m * 128 + ch * 64 + c, o);
+                        tmem_wait_ld();
+                    }
+                    auto pk = [&](int e) -> uint32_t {  // columns e, e + 1 of this chunk, normalised (0 for a dead row)
+                        return live ? pack_bf16(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv) : 0u;
+                    };
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        dst[(256 * m + c) * 2 / 16 + i] = make_uint4(pk(8 * i), pk(8 * i + 2), pk(8 * i + 4), pk(8 * i + 6));
+                }
+                fence_proxy_async_smem();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(o_free_l);
+                if (lane == 0) mbar_arrive(epi);
+                if (!__all_sync(0xffffffffu, mbar_wait(epi, ec & 1, ab, 12))) ok = false;
+                ++ec;
+                if (ok && lane < 8) {
+                    const int rr = (warp - 2) * 8 + lane;
+                    if (rho0 + rr < p.rows_total) {
+                        bulk_store(p.o_final + ((int64_t)pc.b * p.rows_total + rho0 + rr) * 512, stage + rr * L::kOutPitch,
+                                   512 * 2);
+                        bulk_commit();
+                        bulk_wait_read();
+                    }
+                }
+            } else {
+                float* gbase = p.o_part + ((slot0 + pc.k) * p.rows_total + rho0) * 512;
+#pragma unroll 1
+                for (int m = 0; m < 2; ++m) {
+                    float4* dst = reinterpret_cast<float4*>(stage + r * L::kOutPitch + (128 * hf + 64 * ch) * 4);
+#pragma unroll 1
+                    for (int c = 0; c < 64; c += 32) {
+                        uint32_t o[32];
+                        if (pc.n_tiles > 0 && ok) {  // warp-uniform
+                            tmem_ld32(lane_base + kA8ColO + m * 128 + ch * 64 + c, o);
+                            tmem_wait_ld();
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            dst[c / 4 + i] =
+                                live ? make_float4(__uint_as_float(o[4 * i]) * inv, __uint_as_float(o[4 * i + 1]) * inv,
+                                                   __uint_as_float(o[4 * i + 2]) * inv, __uint_as_float(o[4 * i + 3]) * inv)
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    fence_proxy_async_smem();  // staged rows -> visible to the bulk-copy engine
+                    if (m == 1) {              // O has been read: the next piece's first P.V may overwrite it
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(o_free_l);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(epi);
+                    if (!__all_sync(0xffffffffu, mbar_wait(epi, ec & 1, ab, 12))) ok = false;
+                    ++ec;
+                    if (ok && lane < 8) {
+                        const int rr = (warp - 2) * 8 + lane;  // each softmax warp ships eight rows
+                        if (rho0 + rr < p.rows_total) {
+                            bulk_store(gbase + (int64_t)rr * 512 + 256 * m, stage + rr * L::kOutPitch, 256 * 4);
+                            bulk_commit();
+                            bulk_wait_read();
+                        }
+                    }
+                    if (m == 0) {  // the staging is rewritten next: every warp's stores must have read it
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(epi);
+                        if (!__all_sync(0xffffffffu, mbar_wait(epi, ec & 1, ab, 12))) ok = false;
+                        ++ec;
+                    }
+                }
+            }
+            // staging (and with it P and the V ring) is free again once every warp's stores have read it
+            __syncwarp();
+            if (lane == 0) mbar_arrive(epi_done);
+            if (!__all_sync(0xffffffffu, mbar_wait(epi_done, pi & 1, ab, 12))) ok = false;
+            if (row_valid && part == 0 && p.lse_part != nullptr)
+                p.lse_part[(slot0 + pc.k) * p.rows_total + rho] =
+                    live ? (m_used - kAF8Bias + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
+            gt += pc.n_tiles;
+            ++pi;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync();  // neither CTA leaves while the other may still signal its barriers
+    if (warp == 1) tmem_dealloc2(tmem_base, 512);
+}
+
+}  // namespace tc
+}  // namespace gqla

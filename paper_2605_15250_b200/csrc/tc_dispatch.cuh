@@ -7,6 +7,7 @@
 #include "tc_decode_absorb.cuh"
 #include "tc_decode_gqa.cuh"
 #include "tc_decode_gqa_fp8.cuh"
+#include "tc_decode_absorb_fp8.cuh"
 #include "tc_append.cuh"
 #include "tc_combine_up.cuh"
 #include "tc_expand.cuh"
@@ -429,6 +430,50 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
         default: return GQLA_ERR_UNSUPPORTED;
     }
     return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
+}
+
+// Absorb path over an E4M3 latent cache; covers what the bf16 pair kernel covers (r_kv = 512, d_r = 64).
+inline gqla_status tc_decode_absorb_fp8(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S, const uint8_t* q8,
+                                        const float* q_scale, const uint8_t* cache8, int64_t cache_row_stride,
+                                        int64_t cache_rows, float v_scale, const RowMap& rows, const int32_t* seqlens,
+                                        float* o_part, float* lse_part, int32_t* status, cudaStream_t st) {
+    if (!tc_covers(d, GQLA_BF16, s_q, 0) || cache_row_stride % 16 != 0 || cache_rows > 0x7fffffffLL || cache_rows < 1)
+        return GQLA_ERR_UNSUPPORTED;
+    const int rows_total = s_q * d.h_q;
+    const int row_blocks = (rows_total + 127) / 128;
+    const int32_t workers = S < 0 ? tc_balanced_workers(d, s_q, 0) : 0;
+    const bool balanced = S < 0 && workers > 0;
+    if (S < 0) S = -S;
+    const int64_t pairs = balanced ? (int64_t)workers * row_blocks : (int64_t)B * S * row_blocks;
+    if (2 * pairs > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
+    CUtensorMap tmQ, tmQr, tmC, tmCr;
+    {
+        const uint64_t dims[2] = {(uint64_t)(d.r_kv + d.d_r), (uint64_t)B * rows_total};
+        const uint64_t str[1] = {(uint64_t)(d.r_kv + d.d_r)};
+        const uint32_t box[2] = {128, 64}, box_r[2] = {64, 64};
+        if (!tc::make_tmap_u8(&tmQ, q8, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return GQLA_ERR_CUDA;
+        if (!tc::make_tmap_u8(&tmQr, q8, 2, dims, str, box_r, CU_TENSOR_MAP_SWIZZLE_64B)) return GQLA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)(d.r_kv + d.d_r), (uint64_t)cache_rows};
+        const uint64_t str[1] = {(uint64_t)cache_row_stride};
+        const uint32_t box[2] = {128, 64}, box_r[2] = {64, 64};
+        if (!tc::make_tmap_u8(&tmC, cache8, 2, dims, str, box, CU_TENSOR_MAP_SWIZZLE_128B)) return GQLA_ERR_CUDA;
+        if (!tc::make_tmap_u8(&tmCr, cache8, 2, dims, str, box_r, CU_TENSOR_MAP_SWIZZLE_64B)) return GQLA_ERR_CUDA;
+    }
+    tc::AbsorbFp8Params p{};
+    p.B = B; p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.rows_total = rows_total; p.row_blocks = row_blocks;
+    p.balanced = balanced ? 1 : 0; p.W = workers;
+    p.scale_log2 = scale * 1.4426950408889634f; p.v_scale = v_scale; p.q_scale = q_scale;
+    p.rows = rows; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
+    p.o_final = nullptr;
+    auto kern = tc::decode_absorb_fp8_tc_kernel<0>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AbsorbFp8Smem::kTotal) != cudaSuccess)
+        return GQLA_ERR_CUDA;
+    return tc::launch_pdl(kern, dim3((unsigned)(2 * pairs)), dim3(tc::AbsorbFp8Smem::kThreads), tc::AbsorbFp8Smem::kTotal, st,
+                          p, tmQ, tmQr, tmC, tmCr) == cudaSuccess
+               ? GQLA_OK
+               : GQLA_ERR_CUDA;
 }
 
 template <int R>
