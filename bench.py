@@ -152,6 +152,8 @@ def extra_paths(dev, local_rank: int, steps: int, warmup: int, seconds: float) -
     from paper_2605_15250_b200 import sweep
     from paper_2605_15250_b200.decoder import GqlaDecoder
 
+    import time as _time
+
     out = {}
     cases = {"C3": [("absorb", 1, -3), ("absorb", 2, -3), ("gqa", 1, -2), ("gqa", 2, -2)],
              "C4": [("absorb", 1, -32), ("absorb", 2, -32), ("gqa", 1, -32), ("gqa", 2, -32)]}
@@ -164,11 +166,109 @@ def extra_paths(dev, local_rank: int, steps: int, warmup: int, seconds: float) -
         for path, s_q, S in lst:
             w = base.with_(s_q=s_q)
             xq = {**x, **synth.make_queries(w)}
+            _time.sleep(0.3)  # let the clocks recover from the previous case's load
             res = sweep.time_case(dec, w, xq, path, S, steps, warmup)
             if res:
                 out[f"{name}_{path}_sq{s_q}"] = res
         del dec, x
         torch.cuda.empty_cache()
+    return out
+
+
+def fp8_paths(dec, x, x2, q2, peaks, peak_kind: str, steps: int) -> dict:
+    """Both decode paths over an FP8 (E4M3) cache holding the same rows: C1 (absorb, s_q = 1) and C2 (GQA, s_q = 2).
+    Per-plane scales max|x| / 448; the queries are quantised per row inside the timed chain.  The tensor roof is
+    twice the measured bf16 matmul rate (no FP8 rate is measured on this machine; the nominal ratio is 2)."""
+    from paper_2605_15250_b200 import binding as B
+
+    w1, w2 = synth.WORKLOADS["C1"], synth.WORKLOADS["C2"]
+    dev = dec.device
+    N = dec.cache.shape[0]
+    total_tokens = int(x["seqlens"].sum())
+    amax = lambda t: max(float(t.float().abs().max()) / 448.0, 1e-8)
+    sc, sr = amax(dec.cache[:, :w1.r_kv]), amax(dec.cache[:, w1.r_kv:])
+    sk, sv = amax(dec.k_c), amax(dec.v)
+    u8 = lambda *shape: torch.empty(shape, dtype=torch.uint8, device=dev)
+    cache8, kc8, v8, kr8 = u8(N, w1.d_abs), u8(N, w1.g, w1.d_h), u8(N, w1.g, w1.d_h), u8(N, w1.d_r)
+    B.gqla_quantize_cols_e4m3(dec.cache, w1.r_kv, sc, sr, cache8)
+    B.gqla_quantize_cols_e4m3(dec.k_c, w1.d_h, sk, sk, kc8)
+    B.gqla_quantize_cols_e4m3(dec.v, w1.d_h, sv, sv, v8)
+    B.gqla_quantize_cols_e4m3(dec.cache[:, w1.r_kv:], w1.d_r, sr, sr, kr8)
+    out = {}
+    tf8 = 2.0 * peaks["bf16_tflops"]
+
+    def entry(name, w, chain, kernel, nbytes, flops, extra):
+        replay, _ = dec.capture(chain)
+        for _ in range(3):
+            replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            replay()
+        e1.record()
+        torch.cuda.synchronize()
+        chain_us = e0.elapsed_time(e1) * 1e3 / steps
+        k_us = kernel_ms_back_to_back(kernel, steps) * 1e3
+        t = k_us * 1e-6
+        t_mem, t_mma = nbytes / (peaks["hbm_gbs"] * 1e9), flops / (tf8 * 1e12)
+        out[name] = {"workload": w.name, "s_q": w.s_q, "cache": "E4M3, one byte per element", "kernel_us": k_us,
+                     "path_us": chain_us, "tokens_per_s": w.batch * w.s_q / (chain_us * 1e-6), "gbs": nbytes / t / 1e9,
+                     "tflops": flops / t / 1e12, "algorithmic_bytes": nbytes, "flops": flops,
+                     "roofline": {"bound": "hbm" if t_mem >= t_mma else "tensor", "frac": max(t_mem, t_mma) / t,
+                                  "peak_hbm_gbs": peaks["hbm_gbs"], "peak_fp8_tflops": tf8,
+                                  "peak_source": f"hbm of {peak_kind}; fp8 tensor = 2 x bf16 of {peak_kind} (nominal ratio)",
+                                  "frac_of_nominal_roofline": acct.roofline_time(flops, nbytes, 4.5e15, 8e12) / t}, **extra}
+
+    # absorb path: absorb_q (bf16) -> per-row quantisation -> FP8 attention (one piece per sequence) -> merge + up-projection
+    q_c, q_r = x["q_c"].to(dev), x["q_r"].to(dev)
+    q_hat = dec._get("q_hat", (w1.batch, w1.s_q, w1.h_q, w1.d_abs), torch.bfloat16)
+    qh8, qhs = u8(*q_hat.shape), torch.empty(q_hat.shape[:-1], dtype=torch.float32, device=dev)
+    o_part = dec._get("o_part_a8", (w1.batch, 1, w1.s_q, w1.h_q, w1.r_kv), torch.float32)
+    lse_part = dec._get("lse_part_a8", (w1.batch, 1, w1.s_q, w1.h_q), torch.float32)
+    o_out = dec._get("o_a", (w1.batch, w1.s_q, w1.h_q, w1.d_h), torch.bfloat16)
+
+    o_hat = dec._get("o_hat", (w1.batch, w1.s_q, w1.h_q, w1.r_kv), torch.bfloat16)
+
+    def absorb_kernel():
+        B.gqla_decode_absorb_fp8_final(dec.dims, qh8, qhs, cache8, sc, dec.seq_start, dec.seqlens, dec.scale, o_hat, None,
+                                       dec.status)
+
+    def absorb_chain():
+        B.gqla_absorb_q(dec.dims, q_c, q_r, dec.w_uk, q_hat)
+        B.gqla_quantize_rows_e4m3(q_hat, w1.r_kv, sc, sr, qh8, qhs)
+        absorb_kernel()
+        B.gqla_up_proj(dec.dims, o_hat, dec.w_uv, o_out)
+        return o_out
+
+    rows1 = w1.batch * w1.s_q * w1.h_q
+    nb = w1.d_abs * total_tokens + rows1 * (w1.d_abs + 4) + 2 * rows1 * w1.r_kv
+    entry("absorb_fp8", w1, absorb_chain, absorb_kernel, nb, acct.absorb_flops(w1.h_q, w1.r_kv, w1.d_r, w1.s_q, total_tokens),
+          {"chain": "absorb_q, quantize_rows_e4m3, decode_absorb_fp8_final, up_proj"})
+
+    # GQA path: per-row quantisation of [q^C ; q^R] -> FP8 attention (balanced plan) -> merge
+    q8, qs = u8(*q2.shape), torch.empty(q2.shape[:-1], dtype=torch.float32, device=dev)
+    S_g = -2 if B.gqla_balanced_workers(dec.dims, torch.bfloat16, w2.s_q, "gqa") > 0 else 1
+    og_part = dec._get("o_part_g8", (w2.batch, abs(S_g), w2.s_q, w2.h_q, w2.d_h), torch.float32)
+    lg_part = dec._get("lse_part_g8", (w2.batch, abs(S_g), w2.s_q, w2.h_q), torch.float32)
+    og = dec._get("o_g", (w2.batch, w2.s_q, w2.h_q, w2.d_h), torch.bfloat16)
+
+    def gqa_kernel():
+        B.gqla_decode_gqa_fp8(dec.dims, q8, qs, kc8, v8, kr8, sv, dec.seq_start, dec.seqlens, dec.scale, S_g, og_part, lg_part,
+                              dec.status)
+
+    def gqa_chain():
+        B.gqla_quantize_rows_e4m3(q2, w2.d_h, sk, sr, q8, qs)
+        gqa_kernel()
+        B.gqla_combine_splits(og_part, lg_part, og, None)
+        return og
+
+    rows2 = w2.batch * w2.s_q * w2.h_q
+    pieces = 1.25 if S_g < 0 else 1.0
+    nb2 = (2 * w2.g * w2.d_h + w2.d_r) * total_tokens + rows2 * (w2.d_gqa + 4) + int(4 * rows2 * pieces * (w2.d_h + 1))
+    entry("gqa_fp8", w2, gqa_chain, gqa_kernel, nb2, acct.gqa_flops(w2.h_q, w2.d_h, w2.d_r, w2.s_q, total_tokens),
+          {"chain": "quantize_rows_e4m3, decode_gqa_fp8, combine_splits", "num_splits": S_g})
+    dec.check_status()
     return out
 
 
@@ -445,7 +545,10 @@ def run_ours(args):
                 "expand_cache_ms_one_shot": expand_ms},
     }
 
-    # ---- the other workloads of the metric, rank 0 at N=1 only (their caches take 2.5 + 9 GB)
+    # ---- the same two workloads over an FP8 cache, then the other workloads of the metric: rank 0 at N=1 only
+    # (the C3 caches take 2.5 + 9 GB)
+    if world == 1 and not args.no_fp8_paths:
+        paths.update(fp8_paths(dec, x, x2, q2, peaks, peak_kind, min(steps, 50)))
     if world == 1 and not args.no_extra_paths:
         del replay_e2e, replay_gqa, replay_absorb
         paths.update(extra_paths(dev, local_rank, min(steps, 30), 3, args.sustained_seconds))
@@ -494,6 +597,7 @@ def main():
     ap.add_argument("--no-sustained", action="store_true", help="skip the long back-to-back loops of the two decode kernels")
     ap.add_argument("--sustained-seconds", type=float, default=1.0)
     ap.add_argument("--no-extra-paths", action="store_true", help="skip the C3 / C4 entries of \"paths\"")
+    ap.add_argument("--no-fp8-paths", action="store_true", help="skip the FP8-cache entries of \"paths\"")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -44,6 +44,11 @@
  *     W depends on the GPU and the shape: gqla_balanced_workers reports it, gqla_balanced_plan lists
  *     the row ranges.  Where no kernel with this scheduler covers the call (gqla_balanced_workers
  *     returns 0) the fixed plan with S splits is used instead -- also a valid set of partials.
+ *   - Weights (w_uk, w_uv) are constants of a decode loop, and the projection kernels treat them so: their tiles
+ *     are requested before the kernel waits for the preceding work of the stream.  Write or update weights, then
+ *     synchronise the stream once, before the first call that reads them; never produce a weight tensor with a
+ *     kernel that may still be running when a call of this library is enqueued behind it.  Every other input
+ *     (queries, caches, lengths, partials) is read only after the preceding work of the stream has completed.
  *   - Errors: argument violations return a code before anything is launched.
  *     A launch failure returns GQLA_ERR_CUDA.  Device-side waits are bounded;
  *     if one expires the kernel writes a non-zero code to *status_word (device
@@ -239,6 +244,15 @@ gqla_status gqla_decode_absorb_fp8(const gqla_dims* dims, int32_t B, int32_t s_q
                                    int64_t cache_row_stride, int64_t cache_rows, float v_scale, const int64_t* seq_start,
                                    const int32_t* seqlens, float* o_part, float* lse_part, int32_t* status_word,
                                    void* stream);
+/* The whole-sequence form (no split-KV), the FP8 counterpart of gqla_decode_absorb_final: the normalised latent
+ * output goes out once, as bf16 o_hat [B, s_q, h_q, r_kv] (lse [B, s_q, h_q] fp32 or NULL), ready for gqla_up_proj.
+ * Tensor-core shapes only (r_kv = 512, d_r = 64, AUTO policy): GQLA_ERR_UNSUPPORTED otherwise -- use
+ * gqla_decode_absorb_fp8 with one split and gqla_combine_splits there. */
+gqla_status gqla_decode_absorb_fp8_final(const gqla_dims* dims, int32_t B, int32_t s_q, float scale, const uint8_t* q8,
+                                         const float* q_scale, const uint8_t* cache8, int64_t cache_row_stride,
+                                         int64_t cache_rows, float v_scale, const int64_t* seq_start,
+                                         const int32_t* seqlens, void* o_hat, float* lse, int32_t* status_word,
+                                         void* stream);
 /* Eq. (mha) over E4M3 planes:  q8 [B, s_q, h_q, d_h+d_r], q_scale [B, s_q, h_q];  k_c8, v8 [N, g, d_h];
  * k_r8 [N, .] with row stride k_r_row_stride (bytes);  v_scale = the V plane's scale.  num_splits as for
  * gqla_decode_gqa.  Outputs and the other arguments as for gqla_decode_gqa. */

@@ -74,6 +74,8 @@ _PROTOTYPES = {
                                           c_void_p]),
     "gqla_decode_absorb_fp8": (c_int32, [c_void_p, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p, c_void_p, c_int64,
                                          c_int64, c_float, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "gqla_decode_absorb_fp8_final": (c_int32, [c_void_p, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p, c_int64,
+                                               c_int64, c_float, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "gqla_decode_gqa_fp8": (c_int32, [c_void_p, c_int32, c_int32, c_float, c_int32, c_void_p, c_void_p, c_void_p, c_void_p,
                                       c_void_p, c_int64, c_int64, c_float, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                       c_void_p]),
@@ -396,6 +398,20 @@ def gqla_decode_absorb_fp8(dims: GqlaDims, q8: torch.Tensor, q_scale: torch.Tens
     _check(lib().gqla_decode_absorb_fp8(ctypes.byref(dims), B, s_q, scale, num_splits, _ptr(q8), _ptr(q_scale), _ptr(cache8),
                                         cache8.stride(0), cache8.shape[0], v_scale, _ptr(seq_start), _ptr(seqlens),
                                         _ptr(o_part), _ptr(lse_part), _ptr(status_word), _stream()), "gqla_decode_absorb_fp8")
+
+
+def gqla_decode_absorb_fp8_final(dims: GqlaDims, q8: torch.Tensor, q_scale: torch.Tensor, cache8: torch.Tensor, v_scale: float,
+                                 seq_start: torch.Tensor, seqlens: torch.Tensor, scale: float, o_hat: torch.Tensor,
+                                 lse: torch.Tensor | None = None, status_word: torch.Tensor | None = None) -> None:
+    """Whole-sequence absorb-path attention over an E4M3 latent cache: bf16 o_hat [B, s_q, h_q, r_kv] for gqla_up_proj."""
+    _contig(q8, q_scale, seq_start, seqlens, o_hat, lse)
+    assert q8.dtype == torch.uint8 and cache8.dtype == torch.uint8 and cache8.dim() == 2 and cache8.stride(1) == 1
+    assert q_scale.dtype == torch.float32 and o_hat.dtype == torch.bfloat16
+    B, s_q = q8.shape[0], q8.shape[1]
+    _check(lib().gqla_decode_absorb_fp8_final(ctypes.byref(dims), B, s_q, scale, _ptr(q8), _ptr(q_scale), _ptr(cache8),
+                                              cache8.stride(0), cache8.shape[0], v_scale, _ptr(seq_start), _ptr(seqlens),
+                                              _ptr(o_hat), _ptr(lse), _ptr(status_word), _stream()),
+           "gqla_decode_absorb_fp8_final")
 
 
 def gqla_decode_gqa_fp8(dims: GqlaDims, q8: torch.Tensor, q_scale: torch.Tensor, k_c8: torch.Tensor, v8: torch.Tensor,

@@ -438,6 +438,9 @@ template <typename T>
 __global__ void __launch_bounds__(128) quantize_rows_kernel(int64_t rows, int32_t width, int32_t split, float pre_a,
                                                             float pre_b, const T* __restrict__ src,
                                                             uint8_t* __restrict__ dst, float* __restrict__ row_scale) {
+    // (dependent-launch instructions; no-ops when the kernel is launched the ordinary way)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int lane = threadIdx.x & 31;
     const int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (r >= rows) return;

@@ -531,13 +531,14 @@ gqla_status gqla_quantize_rows_e4m3(gqla_dtype src_dtype, int64_t rows, int32_t 
     const int64_t blocks = (rows + 3) / 4;
     if (blocks > 0x7fffffffLL) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e;
     if (src_dtype == GQLA_BF16)
-        quantize_rows_kernel<__nv_bfloat16><<<(unsigned)blocks, 128, 0, st>>>(rows, width, split, pre_a, pre_b,
-                                                                              (const __nv_bfloat16*)src, dst, row_scale);
+        e = tc::launch_pdl(quantize_rows_kernel<__nv_bfloat16>, dim3((unsigned)blocks), dim3(128), 0, st, rows, width, split,
+                           pre_a, pre_b, (const __nv_bfloat16*)src, dst, row_scale);
     else
-        quantize_rows_kernel<float><<<(unsigned)blocks, 128, 0, st>>>(rows, width, split, pre_a, pre_b, (const float*)src,
-                                                                      dst, row_scale);
-    return launch_status();
+        e = tc::launch_pdl(quantize_rows_kernel<float>, dim3((unsigned)blocks), dim3(128), 0, st, rows, width, split, pre_a,
+                           pre_b, (const float*)src, dst, row_scale);
+    return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
 }
 
 // S >= 1: fixed split plan;  S <= -2: balanced plan with -S slots (tensor-core kernels; the generic ones run the
@@ -581,6 +582,24 @@ gqla_status gqla_decode_absorb_fp8(const gqla_dims* d, int32_t B, int32_t s_q, f
     a.B = B; a.S = num_splits < 0 ? -num_splits : num_splits; a.s_q = s_q; a.h_q = d->h_q; a.hpg = d->h_q / d->g;
     a.scale = scale; a.o_part = o_part; a.lse_part = lse_part; a.q_row_scale = q_scale; a.v_scale = v_scale;
     return launch_decode_generic_fp8(a, st);
+}
+
+gqla_status gqla_decode_absorb_fp8_final(const gqla_dims* d, int32_t B, int32_t s_q, float scale, const uint8_t* q8,
+                                         const float* q_scale, const uint8_t* cache8, int64_t cache_row_stride,
+                                         int64_t cache_rows, float v_scale, const int64_t* seq_start, const int32_t* seqlens,
+                                         void* o_hat, float* lse, int32_t* status_word, void* stream) {
+    gqla_status s;
+    if ((s = check_dims(d)) != GQLA_OK) return s;
+    if (B < 0 || s_q < 1 || !(v_scale > 0.f)) return GQLA_ERR_SHAPE;
+    if (B == 0) return GQLA_OK;
+    if (q8 == nullptr || q_scale == nullptr || cache8 == nullptr || seq_start == nullptr || seqlens == nullptr ||
+        o_hat == nullptr)
+        return GQLA_ERR_NULL;
+    if (!aligned16(q8) || !aligned16(cache8) || !aligned16(o_hat)) return GQLA_ERR_ALIGN;
+    if (cache_row_stride < d->r_kv + d->d_r || cache_rows < 0) return GQLA_ERR_SHAPE;
+    if (g_policy.load() != GQLA_POLICY_AUTO) return GQLA_ERR_UNSUPPORTED;
+    return tc_decode_absorb_fp8(*d, B, s_q, scale, 1, q8, q_scale, cache8, cache_row_stride, cache_rows, v_scale,
+                                packed_rows(seq_start), seqlens, nullptr, lse, status_word, (cudaStream_t)stream, o_hat);
 }
 
 gqla_status gqla_decode_gqa_fp8(const gqla_dims* d, int32_t B, int32_t s_q, float scale, int32_t num_splits,

@@ -436,7 +436,8 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
 inline gqla_status tc_decode_absorb_fp8(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S, const uint8_t* q8,
                                         const float* q_scale, const uint8_t* cache8, int64_t cache_row_stride,
                                         int64_t cache_rows, float v_scale, const RowMap& rows, const int32_t* seqlens,
-                                        float* o_part, float* lse_part, int32_t* status, cudaStream_t st) {
+                                        float* o_part, float* lse_part, int32_t* status, cudaStream_t st,
+                                        void* o_final = nullptr) {
     if (!tc_covers(d, GQLA_BF16, s_q, 0) || cache_row_stride % 16 != 0 || cache_rows > 0x7fffffffLL || cache_rows < 1)
         return GQLA_ERR_UNSUPPORTED;
     const int rows_total = s_q * d.h_q;
@@ -466,7 +467,8 @@ inline gqla_status tc_decode_absorb_fp8(const gqla_dims& d, int32_t B, int32_t s
     p.balanced = balanced ? 1 : 0; p.W = workers;
     p.scale_log2 = scale * 1.4426950408889634f; p.v_scale = v_scale; p.q_scale = q_scale;
     p.rows = rows; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
-    p.o_final = nullptr;
+    p.o_final = (__nv_bfloat16*)o_final;
+    if (o_final != nullptr && (balanced || S != 1)) return GQLA_ERR_UNSUPPORTED;
     auto kern = tc::decode_absorb_fp8_tc_kernel<0>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AbsorbFp8Smem::kTotal) != cudaSuccess)
         return GQLA_ERR_CUDA;

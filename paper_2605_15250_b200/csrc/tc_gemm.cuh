@@ -81,10 +81,41 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    pdl_wait();  // set-up done; the inputs may come from the previous kernel of the stream
-
     const CUtensorMap* tmB = (MODE == kGemmExpand && grp >= p.g) ? &tmB1 : &tmB0;
     const int j = (MODE == kGemmExpand) ? grp % p.g : grp;
+
+    // The projection weights are constants of the model, never outputs of the previous kernel of the stream: their
+    // tiles for the first ring stages are requested BEFORE the wait on that kernel and travel while it drains.
+    // (The activations, which it may have written, are requested after the wait.)
+    const int n_pre = (MODE == kGemmExpand) ? 0 : (p.k_blocks < L::kStages ? p.k_blocks : L::kStages);
+    auto load_b = [&](int kb, int s) {
+        uint8_t* b_dst = tiles + s * L::kStageBytes + L::kABytes;
+        if (B_MN && MODE == kGemmExpand) {
+            // rows = j * K + k, columns = d; one 64x64 box per 64 output columns, two per group
+#pragma unroll
+            for (int nb = 0; nb < BN / 64; ++nb)
+                tma_load_2d(b_dst + nb * 8192, tmB, (nb & 1) * 64, (j + (nb >> 1)) * p.k_blocks * 64 + kb * 64, &full[s]);
+        } else if (B_MN) {
+            // rows = j * K + k, columns = output feature; one 64x64 box per 64 output columns
+#pragma unroll
+            for (int nb = 0; nb < BN / 64; ++nb)
+                tma_load_2d(b_dst + nb * 8192, tmB, n_tile * BN + nb * 64, j * p.k_blocks * 64 + kb * 64, &full[s]);
+        } else {
+            // rows = j * r_kv + output feature, columns = k
+            tma_load_2d(b_dst, tmB, kb * 64, j * p.r_kv + n_tile * BN, &full[s]);
+        }
+    };
+    if (warp == 0 && n_pre > 0) {
+        if (elect_one()) {
+            tma_prefetch_desc(tmB);
+            for (int kb = 0; kb < n_pre; ++kb) {  // the ring is empty: no wait needed for its first round
+                mbar_expect_tx(&full[kb], L::kStageBytes);
+                load_b(kb, kb);
+            }
+        }
+        __syncwarp();
+    }
+    pdl_wait();  // set-up done; the activations may come from the previous kernel of the stream
 
     if (warp == 0) {
         if (elect_one()) {
@@ -95,8 +126,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
                 const uint32_t ph = (kb / L::kStages) & 1;
                 if (!mbar_wait(&empty[s], ph ^ 1, ab, 1)) break;
                 uint8_t* a_dst = tiles + s * L::kStageBytes;
-                uint8_t* b_dst = a_dst + L::kABytes;
-                mbar_expect_tx(&full[s], L::kStageBytes);
+                if (kb >= n_pre) mbar_expect_tx(&full[s], L::kStageBytes);  // stages [0, n_pre) were armed before the wait
                 if (MODE == kGemmExpand) {
                     tma_load_2d(a_dst, &tmA, kb * 64, m_tile * 128, &full[s]);
                 } else {
@@ -109,22 +139,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
                         "r"(m_tile * (128 / p.hpb))
                         : "memory");
                 }
-                if (B_MN && MODE == kGemmExpand) {
-                    // rows = j * K + k, columns = d; one 64x64 box per 64 output columns, two per group
-#pragma unroll
-                    for (int nb = 0; nb < BN / 64; ++nb)
-                        tma_load_2d(b_dst + nb * 8192, tmB, (nb & 1) * 64, (j + (nb >> 1)) * p.k_blocks * 64 + kb * 64,
-                                    &full[s]);
-                } else if (B_MN) {
-                    // rows = j * K + k, columns = output feature; one 64x64 box per 64 output columns
-#pragma unroll
-                    for (int nb = 0; nb < BN / 64; ++nb)
-                        tma_load_2d(b_dst + nb * 8192, tmB, n_tile * BN + nb * 64, j * p.k_blocks * 64 + kb * 64,
-                                    &full[s]);
-                } else {
-                    // rows = j * r_kv + output feature, columns = k
-                    tma_load_2d(b_dst, tmB, kb * 64, j * p.r_kv + n_tile * BN, &full[s]);
-                }
+                if (kb >= n_pre) load_b(kb, s);
             }
         }
     } else if (warp == 1) {

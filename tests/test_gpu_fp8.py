@@ -97,6 +97,15 @@ def test_fp8_decode_both_paths(dims, policy, s_q):
     assert_close(o_part.cpu().numpy(), op_ref, "decode_absorb_fp8 o_part", rel, abs_)
     assert_close(lse_part.cpu().numpy(), lp_ref, "decode_absorb_fp8 lse_part", 1e-2, 1e-3)
 
+    if tc:  # the whole-sequence call: bf16 o_hat in one pass (tensor-core shapes only)
+        o_hat = torch.full((Bn, s_q, w.h_q, w.r_kv), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((Bn, s_q, w.h_q), float("nan"), dtype=torch.float32, device="cuda")
+        B.gqla_decode_absorb_fp8_final(bd, q8, qs, cache8, sc, dev["seq_start"], dev["seqlens"], w.scale, o_hat, lse, status)
+        o1, l1 = O.decode_absorb_fp8_partials(od, q8.cpu().numpy(), qs.cpu().numpy(), cache8.cpu().numpy(), sc, ss, sl, s_q,
+                                              w.scale, 1)
+        assert_close(o_hat.float().cpu().numpy(), o1[:, 0], "decode_absorb_fp8_final o_hat", rel, abs_)
+        assert_close(lse.cpu().numpy(), l1[:, 0], "decode_absorb_fp8_final lse", 1e-2, 1e-3)
+
     # ---- GQA path: expand in bf16, quantise the three planes and q, attend
     k_c = torch.empty((N, w.g, w.d_h), dtype=torch.bfloat16, device="cuda")
     v = torch.empty_like(k_c)
