@@ -532,7 +532,11 @@ gqla_status gqla_quantize_rows_e4m3(gqla_dtype src_dtype, int64_t rows, int32_t 
     if (blocks > 0x7fffffffLL) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e;
-    if (src_dtype == GQLA_BF16)
+    if (src_dtype == GQLA_BF16 && width % 8 == 0 && split % 8 == 0 && width <= 8 * 32 * kQuantChunksPerLane && aligned16(src) &&
+        (reinterpret_cast<uintptr_t>(dst) & 7u) == 0)
+        e = tc::launch_pdl(quantize_rows_bf16_vec_kernel, dim3((unsigned)blocks), dim3(128), 0, st, rows, width, split, pre_a,
+                           pre_b, (const __nv_bfloat16*)src, dst, row_scale);
+    else if (src_dtype == GQLA_BF16)
         e = tc::launch_pdl(quantize_rows_kernel<__nv_bfloat16>, dim3((unsigned)blocks), dim3(128), 0, st, rows, width, split,
                            pre_a, pre_b, (const __nv_bfloat16*)src, dst, row_scale);
     else
