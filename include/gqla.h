@@ -82,7 +82,8 @@ typedef enum {
     GQLA_ERR_UNSUPPORTED = 5, /* valid but no kernel covers it                  */
     GQLA_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed            */
     GQLA_ERR_TIMEOUT = 7,     /* value written to *status_word by a bounded wait */
-    GQLA_ERR_CAPACITY = 8     /* the call needs more built-in scratch than the library holds */
+    GQLA_ERR_CAPACITY = 8,    /* the call needs more built-in scratch than the library holds */
+    GQLA_ERR_DEBUG_CHECK = 9  /* value written to *status_word by an index check of a -DGQLA_DEBUG build */
 } gqla_status;
 
 typedef enum { GQLA_BF16 = 0, GQLA_F32 = 1 } gqla_dtype;
@@ -284,8 +285,10 @@ gqla_status gqla_up_proj(const gqla_dims* dims, gqla_dtype dtype, int32_t B, int
  *   gqla_decode_gqa_dv     v [N, g, d_v]        ->  o_part [B, S, s_q, h_q, d_v]
  *   gqla_up_proj_dv        w_uv [g, r_kv, d_v]  ->  o [B, s_q, h_q, d_v]
  * The absorb path needs nothing else (its attention runs in the latent space), and gqla_combine_splits
- * takes the output width as d_out already.  With d_v == d_h they are the calls without the suffix; other
- * values run on the generic kernels (d_v <= 512 for gqla_decode_gqa_dv). */
+ * takes the output width as d_out already.  With d_v == d_h they are the calls without the suffix.
+ * gqla_decode_gqa_dv runs on the tensor-core kernel when d_h = 128, d_r = 64 and d_v is a multiple of 128 up to
+ * 512 (one CTA per 128-column block of V; the blocks of a group share its K tiles through L2), on the generic
+ * kernel otherwise (d_v <= 512); the other two run on the generic kernels whenever d_v != d_h. */
 gqla_status gqla_expand_cache_dv(const gqla_dims* dims, int32_t d_v, gqla_dtype dtype, int64_t N, const void* cache,
                                  int64_t cache_row_stride, const void* w_uk, const void* w_uv, void* k_c, void* v,
                                  void* k_r, void* stream);

@@ -13,7 +13,8 @@ from ctypes import c_char_p, c_float, c_int32, c_int64, c_void_p
 import torch
 
 _PKG_DIR = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG_DIR, "libgqla.so")
+# GQLA_LIB_PATH selects another build of the same library (e.g. the -DGQLA_DEBUG one, libgqla_debug.so)
+LIB_PATH = os.environ.get("GQLA_LIB_PATH") or os.path.join(_PKG_DIR, "libgqla.so")
 
 GQLA_BF16, GQLA_F32 = 0, 1
 POLICY_AUTO, POLICY_GENERIC = 0, 1

@@ -72,6 +72,7 @@ const char* gqla_status_str(gqla_status s) {
         case GQLA_ERR_CUDA: return "CUDA error";
         case GQLA_ERR_TIMEOUT: return "device wait timed out";
         case GQLA_ERR_CAPACITY: return "call exceeds the library's built-in scratch capacity";
+        case GQLA_ERR_DEBUG_CHECK: return "index check of a debug build failed";
     }
     return "unknown status";
 }
@@ -418,9 +419,9 @@ static gqla_status decode_gqa_any(const gqla_dims* d, int32_t d_v, gqla_dtype dt
     if (!aligned16(q) || !aligned16(k_c) || !aligned16(v) || !aligned16(k_r)) return GQLA_ERR_ALIGN;
     if ((d->d_r > 0 && k_r_row_stride < d->d_r) || n_rows < 0 || d_v < 1) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
-    if (g_policy.load() == GQLA_POLICY_AUTO && d_v == d->d_h && tc_covers(*d, dtype, s_q, 1)) {
+    if (g_policy.load() == GQLA_POLICY_AUTO && tc_covers(*d, dtype, s_q, 1)) {
         s = tc_decode_gqa(*d, B, s_q, scale, num_splits, q, k_c, v, k_r, k_r_row_stride, n_rows, rows, seqlens, o_part,
-                          lse_part, status_word, st);
+                          lse_part, status_word, st, d_v);
         if (s != GQLA_ERR_UNSUPPORTED) return s;
     }
     DecodeArgs a{};

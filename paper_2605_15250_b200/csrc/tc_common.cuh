@@ -69,6 +69,20 @@ struct Abort {
     }
 };
 
+// Index checks of a debug build (-DGQLA_DEBUG; the pool offers no compute-sanitizer): a violated check records
+// kStatusDebug | (where << 8) in the status word and execution goes on -- nothing traps.  Compiled out otherwise.
+constexpr int32_t kStatusDebug = 9;  // == GQLA_ERR_DEBUG_CHECK
+#ifdef GQLA_DEBUG
+#define GQLA_DEBUG_CHECK(cond, status_ptr, where)                                                     \
+    do {                                                                                              \
+        if (!(cond) && (status_ptr) != nullptr) atomicCAS((status_ptr), 0, kStatusDebug | ((where) << 8)); \
+    } while (0)
+#else
+#define GQLA_DEBUG_CHECK(cond, status_ptr, where) \
+    do {                                          \
+    } while (0)
+#endif
+
 // Waits for phase `parity` of `bar`; false if aborted or timed out (and raises the abort).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const Abort& ab, int32_t where) {
     for (uint32_t it = 0; it < kWaitSpins; ++it) {

@@ -337,8 +337,14 @@ decode_absorb_fp8_tc_kernel(const AbsorbFp8Params p, const __grid_constant__ CUt
         int ec = 0;  // completed phases of the `epi` barrier
 
         while (walk.next(pc)) {
+            GQLA_DEBUG_CHECK(pc.b >= 0 && pc.b < p.B, p.status, 32);  // a piece names a sequence of the batch
             const int32_t T = p.seqlens[pc.b];
             const int64_t slot0 = (int64_t)pc.b * p.S;
+            GQLA_DEBUG_CHECK(pc.n_tiles == 0 || (pc.k >= 0 && pc.k < p.S), p.status, 33);  // ... and one of its S slots
+            GQLA_DEBUG_CHECK(pc.tok_begin >= 0 && pc.tok_begin <= pc.tok_end && pc.tok_end <= (T > 0 ? T : 0), p.status, 34);
+            GQLA_DEBUG_CHECK(pc.n_tiles == (pc.tok_end > pc.tok_begin ? (pc.tok_end - pc.tok_begin + 127) / 128 : 0), p.status, 35);
+            GQLA_DEBUG_CHECK(!p.balanced || pc.tok_begin % 128 == 0, p.status, 36);  // balanced pieces start on tile boundaries
+            GQLA_DEBUG_CHECK(pc.fill_begin >= 0 && pc.fill_begin <= pc.fill_end && pc.fill_end <= p.S || pc.fill_end == 0, p.status, 37);
             // split slots this worker marks empty
             if (part == 0 && row_valid && p.lse_part != nullptr)
                 for (int kk = pc.fill_begin; kk < pc.fill_end; ++kk) p.lse_part[(slot0 + kk) * p.rows_total + rho] = -INFINITY;

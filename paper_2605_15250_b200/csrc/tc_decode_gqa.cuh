@@ -28,11 +28,13 @@ namespace tc {
 
 struct GqaParams {
     int32_t B, S, s_q, h_q, g, hpg, hpg_box;
-    int32_t balanced, W;  // balanced plan: W workers per group, grid = W * g
+    int32_t balanced, W;  // balanced plan: W workers per (group, value block), grid = W * g * v_blocks
+    int32_t v_blocks, d_v;  // value head dim d_v = 128 * v_blocks: a CTA computes one 128-column block of the output
+                            // (v_blocks = 1 unless the value head dim differs from d_h, Sec. 3.2)
     float scale_log2;
     RowMap rows;  // packed or paged (pages a multiple of 128 rows, pieces starting on tile boundaries)
     const int32_t* seqlens;
-    float* o_part;    // [B, S, s_q, h_q, 128]
+    float* o_part;    // [B, S, s_q, h_q, d_v]
     float* lse_part;  // [B, S, s_q, h_q]
     int32_t* status;
 };
@@ -117,14 +119,16 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
     pdl_launch_dependents();
     pdl_wait();  // barriers and TMEM are set up; everything below reads the caller's tensors
     // the plan of this CTA: group j, and either one (sequence, split) piece or worker w's share
-    const int j = blockIdx.x % p.g;
+    // consecutive CTAs: the value blocks of a group, then the groups of the same rows (they share k_R and K_C tiles
+    // through L2)
+    const int vb = blockIdx.x % p.v_blocks;
+    const int j = (blockIdx.x / p.v_blocks) % p.g;
+    const int unit = blockIdx.x / (p.v_blocks * p.g);
     Walker walk;
     if (p.balanced) {
-        const BalancedStart st = balanced_prepass(p.seqlens, p.B, p.S, blockIdx.x / p.g, p.W,
-                                                  reinterpret_cast<int32_t*>(merge), L::kThreads);
-        walk.init_balanced(p.seqlens, p.B, p.S, blockIdx.x / p.g, p.W, st);
+        const BalancedStart st = balanced_prepass(p.seqlens, p.B, p.S, unit, p.W, reinterpret_cast<int32_t*>(merge), L::kThreads);
+        walk.init_balanced(p.seqlens, p.B, p.S, unit, p.W, st);
     } else {
-        const int unit = blockIdx.x / p.g;
         walk.init_fixed(p.seqlens, p.B, p.S, unit / p.S, unit % p.S);
     }
     tc_fence_before();
@@ -172,8 +176,8 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
                     tma_load_2d(st + L::kKcBytes, &tmR, 0, row, &kfull[s]);
                     if (!(ok = mbar_wait(&vempty[s], ph ^ 1, ab, 2))) break;
                     mbar_expect_tx(&vfull[s], L::kVBytes);
-                    tma_load_3d(st + L::kKcBytes + L::kKrBytes, &tmV, 0, j, row, &vfull[s]);
-                    tma_load_3d(st + L::kKcBytes + L::kKrBytes + 16384, &tmV, 64, j, row, &vfull[s]);
+                    tma_load_3d(st + L::kKcBytes + L::kKrBytes, &tmV, vb * 128, j, row, &vfull[s]);
+                    tma_load_3d(st + L::kKcBytes + L::kKrBytes + 16384, &tmV, vb * 128 + 64, j, row, &vfull[s]);
                 }
                 ++pi;
             }
@@ -257,10 +261,16 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
         }
 
         while (walk.next(pc)) {
+            GQLA_DEBUG_CHECK(pc.b >= 0 && pc.b < p.B, p.status, 32);  // a piece names a sequence of the batch
             const int32_t T = p.seqlens[pc.b];
             const int64_t slot0 = (int64_t)pc.b * p.S;
+            GQLA_DEBUG_CHECK(pc.n_tiles == 0 || (pc.k >= 0 && pc.k < p.S), p.status, 33);  // ... and one of its S slots
+            GQLA_DEBUG_CHECK(pc.tok_begin >= 0 && pc.tok_begin <= pc.tok_end && pc.tok_end <= (T > 0 ? T : 0), p.status, 34);
+            GQLA_DEBUG_CHECK(pc.n_tiles == (pc.tok_end > pc.tok_begin ? (pc.tok_end - pc.tok_begin + 127) / 128 : 0), p.status, 35);
+            GQLA_DEBUG_CHECK(!p.balanced || pc.tok_begin % 128 == 0, p.status, 36);  // balanced pieces start on tile boundaries
+            GQLA_DEBUG_CHECK(pc.fill_begin >= 0 && pc.fill_begin <= pc.fill_end && pc.fill_end <= p.S || pc.fill_end == 0, p.status, 37);
             // split slots this worker marks empty
-            if (f == 0 && row_valid)
+            if (f == 0 && row_valid && vb == 0)
                 for (int kk = pc.fill_begin; kk < pc.fill_end; ++kk)
                     p.lse_part[((slot0 + kk) * p.s_q + pq) * p.h_q + (int64_t)j * p.hpg + il] = -INFINITY;
             if (pc.n_tiles == 0 && p.balanced) continue;  // an empty sequence: its slots were marked above
@@ -390,11 +400,12 @@ decode_gqa_tc_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ,
                         const float4 x = *reinterpret_cast<const float4*>(merge + (ff * R + rr) * L::kMergePitch + 4 * mcg);
                         acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
                     }
-                    *reinterpret_cast<float4*>(p.o_part + (out_row0 + (int64_t)pp * p.h_q + ii) * 128 + c4 * 32 + 4 * mcg) = acc;
+                    *reinterpret_cast<float4*>(p.o_part + (out_row0 + (int64_t)pp * p.h_q + ii) * p.d_v + vb * 128 + c4 * 32 +
+                                               4 * mcg) = acc;
                 }
                 named_bar_sync(1, 128);
             }
-            if (f == 0 && row_valid)
+            if (f == 0 && row_valid && vb == 0)
                 p.lse_part[out_row0 + (int64_t)pq * p.h_q + il] = live ? (M + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
             gt += pc.n_tiles;
             if (pc.n_tiles > 0) ++pi;

@@ -377,19 +377,24 @@ inline cudaError_t gqa_launch(const tc::GqaParams& p, const CUtensorMap& q, cons
     return tc::launch_pdl(kern, dim3(grid), dim3(tc::GqaSmem::kThreads), tc::GqaSmem::kTotal, st, p, q, k, r, v);
 }
 
+// d_v: value head dim, a multiple of 128 up to 512 (d_h when the shapes of Sec. 3.1 apply).  With d_v > 128 every
+// (rows, group) unit is served by d_v / 128 CTAs, one per 128-column block of V and of the output; each of them
+// computes the scores itself (the K tiles are shared through L2), which is the price of keeping one kernel.
 inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S, const void* q,
                                  const void* k_c, const void* v, const void* k_r, int64_t k_r_row_stride,
                                  int64_t n_rows, const RowMap& rows, const int32_t* seqlens, float* o_part,
-                                 float* lse_part, int32_t* status, cudaStream_t st) {
-    if (!tc_covers(d, GQLA_BF16, s_q, 1) || !stride_ok(k_r_row_stride) || n_rows > 0x7fffffffLL || n_rows < 1)
+                                 float* lse_part, int32_t* status, cudaStream_t st, int32_t d_v = 128) {
+    if (!tc_covers(d, GQLA_BF16, s_q, 1) || !stride_ok(k_r_row_stride) || n_rows > 0x7fffffffLL || n_rows < 1 ||
+        d_v % 128 != 0 || d_v < 128 || d_v > 512)
         return GQLA_ERR_UNSUPPORTED;
+    const int v_blocks = d_v / 128;
     if (rows.paged() && rows.page_size % kTileRows != 0) return GQLA_ERR_UNSUPPORTED;  // a tile must not straddle pages
-    // S < 0: balanced plan with -S slots per sequence, W persistent CTAs per group
-    const int32_t workers = S < 0 ? tc_balanced_workers(d, s_q, 1) : 0;
+    // S < 0: balanced plan with -S slots per sequence, W persistent CTAs per (group, value block)
+    const int32_t workers = S < 0 ? tc_balanced_workers(d, s_q, 1) / v_blocks : 0;
     const bool balanced = S < 0 && workers > 0;
     if (S < 0) S = -S;
     if (rows.paged() && !balanced && S != 1) return GQLA_ERR_UNSUPPORTED;  // see tc_decode_absorb
-    const int64_t units = balanced ? (int64_t)workers * d.g : (int64_t)B * S * d.g;
+    const int64_t units = (balanced ? (int64_t)workers * d.g : (int64_t)B * S * d.g) * v_blocks;
     if (units > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     const int hpg = d.h_q / d.g;
     int hpg_box = 0, sq_box = 0;
@@ -405,9 +410,11 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
     {
         const uint64_t dims[3] = {(uint64_t)d.d_h, (uint64_t)d.g, (uint64_t)n_rows};
         const uint64_t str[2] = {(uint64_t)d.d_h * 2, (uint64_t)d.g * d.d_h * 2};
+        const uint64_t vdims[3] = {(uint64_t)d_v, (uint64_t)d.g, (uint64_t)n_rows};
+        const uint64_t vstr[2] = {(uint64_t)d_v * 2, (uint64_t)d.g * d_v * 2};
         const uint32_t box[3] = {64, 1, 128};
         if (!tc::make_tmap_bf16(&tmK, k_c, 3, dims, str, box)) return GQLA_ERR_CUDA;
-        if (!tc::make_tmap_bf16(&tmV, v, 3, dims, str, box)) return GQLA_ERR_CUDA;
+        if (!tc::make_tmap_bf16(&tmV, v, 3, vdims, vstr, box)) return GQLA_ERR_CUDA;
     }
     {
         const uint64_t dims[2] = {(uint64_t)d.d_r, (uint64_t)n_rows};
@@ -416,6 +423,7 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
         if (!tc::make_tmap_bf16(&tmR, k_r, 2, dims, str, box)) return GQLA_ERR_CUDA;
     }
     tc::GqaParams p{};
+    p.v_blocks = v_blocks; p.d_v = d_v;
     p.B = B; p.S = S; p.s_q = s_q; p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpg_box = hpg_box;
     p.balanced = balanced ? 1 : 0; p.W = workers;
     p.scale_log2 = scale * 1.4426950408889634f;

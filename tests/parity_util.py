@@ -30,6 +30,24 @@ def assert_close(got, ref, what: str, rel: float = REL, abs_: float = ABS) -> fl
     return float(err)
 
 
+class Canaried:
+    """A device tensor with guard regions before and behind it (the pool offers no compute-sanitizer): `t` is the
+    tensor a kernel writes, check() fails if a single guard byte has changed."""
+
+    PAD = 4096  # bytes on each side
+    BYTE = 0xA5
+
+    def __init__(self, shape, dtype):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        self.raw = torch.full((self.PAD + n + self.PAD,), self.BYTE, dtype=torch.uint8, device="cuda")
+        self.t = self.raw[self.PAD:self.PAD + n].view(dtype).view(*shape)
+        self.n = n
+
+    def check(self, what: str) -> None:
+        head, tail = self.raw[:self.PAD], self.raw[self.PAD + self.n:]
+        assert bool((head == self.BYTE).all()) and bool((tail == self.BYTE).all()), f"{what}: wrote outside its buffer"
+
+
 def dims_of(w: synth.Workload):
     return O.Dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r), B.make_dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)
 

@@ -508,6 +508,75 @@ def test_determinism_run_to_run():
     dec.check_status()
 
 
+# ------------------------------------------------------------------ overruns and index checks
+
+
+def test_outputs_do_not_overrun_their_buffers():
+    """Every output of the tensor-core kernels sits between guard regions: bulk and TMA stores clipped at ragged
+    ends (N not a multiple of the 128 / 256-row tiles, h_q not a multiple of the row block), partial slots, final rows."""
+    from tests.parity_util import Canaried
+    w = _wl("canary", 3, 2, 211, **dict(h_q=28, g=4, d_h=128, r_kv=512, d_r=64))
+    seqlens = np.array([333, 1, 1291], dtype=np.int32)
+    x = synth.make_inputs(w, seqlens=seqlens)
+    bd = B.make_dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)
+    dev = {k: t.cuda() for k, t in x.items()}
+    N, Bn, s_q = x["cache"].shape[0], w.batch, w.s_q
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    bf, f32 = torch.bfloat16, torch.float32
+    q_hat = Canaried((Bn, s_q, w.h_q, w.d_abs), bf)
+    B.gqla_absorb_q(bd, dev["q_c"], dev["q_r"], dev["w_uk"], q_hat.t)
+    k_c, v, k_r = Canaried((N, w.g, w.d_h), bf), Canaried((N, w.g, w.d_h), bf), Canaried((N, w.d_r), bf)
+    B.gqla_expand_cache(bd, dev["cache"], dev["w_uk"], dev["w_uv"], k_c.t, v.t, k_r.t)
+    outs = [(q_hat, "absorb_q"), (k_c, "expand k_c"), (v, "expand v"), (k_r, "expand k_r")]
+    q = torch.cat([x["q_c"], x["q_r"]], -1).contiguous().cuda()
+    for S in (1, 3, -3):
+        sl = abs(S)
+        oa, la = Canaried((Bn, sl, s_q, w.h_q, w.r_kv), f32), Canaried((Bn, sl, s_q, w.h_q), f32)
+        B.gqla_decode_absorb(bd, q_hat.t, dev["cache"], dev["seq_start"], dev["seqlens"], w.scale, S, oa.t, la.t, status)
+        og, lg = Canaried((Bn, sl, s_q, w.h_q, w.d_h), f32), Canaried((Bn, sl, s_q, w.h_q), f32)
+        B.gqla_decode_gqa(bd, q, k_c.t, v.t, k_r.t, dev["seq_start"], dev["seqlens"], w.scale, S, og.t, lg.t, status)
+        o_f, l_f = Canaried((Bn, s_q, w.h_q, w.d_h), bf), Canaried((Bn, s_q, w.h_q), f32)
+        B.gqla_combine_up_proj(bd, oa.t, la.t, dev["w_uv"], o_f.t, l_f.t)
+        o_c = Canaried((Bn, s_q, w.h_q, w.d_h), bf)
+        B.gqla_combine_splits(og.t, lg.t, o_c.t, None)
+        outs += [(oa, f"absorb o_part S={S}"), (la, f"absorb lse_part S={S}"), (og, f"gqa o_part S={S}"), (lg, f"gqa lse_part S={S}"),
+                 (o_f, f"combine_up_proj S={S}"), (l_f, f"combine_up_proj lse S={S}"), (o_c, f"combine_splits S={S}")]
+    o_hat, lse = Canaried((Bn, s_q, w.h_q, w.r_kv), bf), Canaried((Bn, s_q, w.h_q), f32)
+    B.gqla_decode_absorb_final(bd, q_hat.t, dev["cache"], dev["seq_start"], dev["seqlens"], w.scale, o_hat.t, lse.t, status)
+    o = Canaried((Bn, s_q, w.h_q, w.d_h), bf)
+    B.gqla_up_proj(bd, o_hat.t, dev["w_uv"], o.t)
+    B.gqla_append_expand(bd, s_q, dev["cache"], dev["seq_start"], dev["seqlens"], dev["w_uk"], dev["w_uv"], k_c.t, v.t, k_r.t)
+    outs += [(o_hat, "decode_absorb_final"), (lse, "decode_absorb_final lse"), (o, "up_proj"), (k_c, "append k_c"), (v, "append v"),
+             (k_r, "append k_r")]
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for c, what in outs:
+        c.check(what)
+
+
+def test_debug_build_index_checks_stay_silent():
+    """The -DGQLA_DEBUG build (piece and tile index checks that record a code instead of trapping) runs the ragged
+    parity case in a process of its own: outputs within tolerance, status word 0."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    lib = gbuild.build(debug=True)
+    code = (
+        "import numpy as np, torch\n"
+        "from paper_2605_15250_b200 import binding as B, synth\n"
+        "from tests.parity_util import end_to_end\n"
+        "assert B.LIB_PATH.endswith('libgqla_debug.so')\n"
+        "w = synth.Workload('dbg', 128, 8, 128, 512, 64, batch=5, s_q=2, dtype='bf16', seed=5)\n"
+        "sl = np.array([700, 0, 129, 2050, 64], dtype=np.int32)\n"
+        "for S in (1, 3, -3):\n"
+        "    end_to_end(w, sl, S, q_gain=4.0)\n"
+        "print('debug-ok')\n")
+    env = dict(os.environ, GQLA_LIB_PATH=lib, PYTHONPATH=root)
+    res = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, env=env, cwd=root, timeout=600)
+    assert res.returncode == 0 and "debug-ok" in res.stdout, res.stdout[-2000:] + res.stderr[-4000:]
+
+
 # ------------------------------------------------------------------ a value head dimension of its own
 
 
