@@ -2,16 +2,25 @@
 // GQLA_ERR_UNSUPPORTED when the shape is outside what those kernels cover, in which case
 // the caller falls through to the generic SIMT kernels.
 #pragma once
+#include <stdlib.h>
+
 #include "../../include/gqla.h"
 #include "common.cuh"
 #include "tc_decode_absorb.cuh"
 #include "tc_decode_gqa.cuh"
+#include "tc_decode_gqa_t.cuh"
 #include "tc_decode_gqa_fp8.cuh"
 #include "tc_decode_absorb_fp8.cuh"
 #include "tc_append.cuh"
 #include "tc_combine_up.cuh"
 #include "tc_expand.cuh"
 #include "tc_gemm.cuh"
+
+// Largest (padded) query-row count per group served by the tokens-on-M GQA kernel when the environment does not
+// say otherwise; beyond it the row-replicating kernel runs (its replication factor 128/R is then 2 or 1).
+#ifndef GQLA_GQA_TOKENS_MAX_ROWS
+#define GQLA_GQA_TOKENS_MAX_ROWS 32
+#endif
 
 namespace gqla {
 
@@ -368,6 +377,40 @@ inline int absorb_resident_pairs() {
     return cached[dev];
 }
 
+// Rows of the tokens-on-M GQA kernel's query block: heads per group and query positions each padded to a power of
+// two, at least 16 rows in all (the smallest N of an M = 128 MMA).
+inline int gqa_rows_t(const gqla_dims& d, int32_t s_q, int* hpg_box, int* sq_box) {
+    const int sb = next_pow2(s_q);
+    int hb = next_pow2(d.h_q / d.g);
+    if (hb * sb < 16) hb = 16 / sb;
+    if (hpg_box != nullptr) *hpg_box = hb;
+    if (sq_box != nullptr) *sq_box = sb;
+    return hb * sb;
+}
+
+// Which GQA kernel serves a shape both cover: the tokens-on-M kernel (tc_decode_gqa_t.cuh) for few query rows per
+// group, the row-replicating one beyond.  GQLA_GQA_KERNEL=rows|tokens in the environment overrides the choice for
+// shapes both cover (read once per process; a tuning aid).
+inline bool gqa_prefers_tokens(int rows_t) {
+    static const int forced = []() {
+        const char* e = getenv("GQLA_GQA_KERNEL");
+        if (e == nullptr) return 0;
+        return e[0] == 't' ? 1 : (e[0] == 'r' ? 2 : 0);
+    }();
+    if (rows_t > 64) return false;
+    if (forced != 0) return forced == 1;
+    return rows_t <= GQLA_GQA_TOKENS_MAX_ROWS;
+}
+
+template <int R>
+inline cudaError_t gqa_t_launch(const tc::GqaParams& p, const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& r,
+                                const CUtensorMap& v, unsigned grid, cudaStream_t st) {
+    auto kern = tc::decode_gqa_t_kernel<R>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::GqaTSmem<R>::kTotal);
+    if (e != cudaSuccess) return e;
+    return tc::launch_pdl(kern, dim3(grid), dim3(tc::GqaTSmem<R>::kThreads), tc::GqaTSmem<R>::kTotal, st, p, q, k, r, v);
+}
+
 template <int R>
 inline cudaError_t gqa_launch(const tc::GqaParams& p, const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& r,
                               const CUtensorMap& v, unsigned grid, cudaStream_t st) {
@@ -398,7 +441,9 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
     if (units > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     const int hpg = d.h_q / d.g;
     int hpg_box = 0, sq_box = 0;
-    const int R = gqa_rows(d, s_q, &hpg_box, &sq_box);
+    int R = gqa_rows(d, s_q, &hpg_box, &sq_box);
+    const bool tokens_on_m = gqa_prefers_tokens(gqa_rows_t(d, s_q, nullptr, nullptr));
+    if (tokens_on_m) R = gqa_rows_t(d, s_q, &hpg_box, &sq_box);
     CUtensorMap tmQ, tmK, tmR, tmV;
     {
         const int feat = d.d_h + d.d_r;
@@ -429,6 +474,15 @@ inline gqla_status tc_decode_gqa(const gqla_dims& d, int32_t B, int32_t s_q, flo
     p.scale_log2 = scale * 1.4426950408889634f;
     p.rows = rows; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
     cudaError_t e;
+    if (tokens_on_m) {
+        switch (R) {
+            case 16: e = gqa_t_launch<16>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
+            case 32: e = gqa_t_launch<32>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
+            case 64: e = gqa_t_launch<64>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
+            default: return GQLA_ERR_UNSUPPORTED;
+        }
+        return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
+    }
     switch (R) {
         case 8: e = gqa_launch<8>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
         case 16: e = gqa_launch<16>(p, tmQ, tmK, tmR, tmV, (unsigned)units, st); break;
