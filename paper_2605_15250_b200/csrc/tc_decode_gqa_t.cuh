@@ -10,8 +10,8 @@
 // so the tensor core does exactly the method's FLOPs (N = R instead of 128).  The price is in the softmax: a
 // TMEM lane is now a TOKEN and holds one score of every query row, so a row's maximum and sum live across the
 // 128 softmax threads.  They are kept out of the loop:
-//   * eight softmax warps, two per TMEM lane quadrant: a thread owns one token of the tile and half of the query
-//     rows.  Every thread holds the same reference m_ref[r] for its rows and checks its own token's scores against
+//   * R/8 softmax warps per TMEM lane quadrant (8 or 16 in all): a thread owns one token of the tile and eight of
+//     the query rows, so the softmax of a tile is spread over up to 512 threads.  Every thread holds the same reference m_ref[r] for its rows and checks its own token's scores against
 //     it; a bar.red.or tells the warps whether any score outgrew its reference by more than 2^8.  Only
 //     then (and on a piece's first tile) are the true row maxima of the tile reduced (redux over a warp, shared
 //     memory across warps), the references raised and O^T rescaled column by column;
@@ -48,10 +48,11 @@ struct GqaTSmem {
     static constexpr int kOffP = kOffStage + kStages * kStageBytes;
     static constexpr int kOffRed = kOffP + 2 * kPBuf;        // [4 warps][R] floats: row maxima / sums across warps
     static constexpr int kRedBytes = 4 * R * 4;
-    static constexpr int kTileBytes = kOffRed + (kRedBytes > 2048 ? kRedBytes : 2048);
+    static constexpr int kTileBytes = kOffRed + (kRedBytes > 3072 ? kRedBytes : 3072);  // also the plan scratch
     // q_full q_empty o_free kfull[2] vfull[2] kempty[2] vempty[2] s_full[2] p_ready[2] pv_done[2]
     static constexpr int kNumBars = 17;
-    static constexpr int kSoftmaxWarps = 8;  // two per TMEM lane quadrant: each takes half of the query rows of its tokens
+    static constexpr int kRowsPerThread = R <= 32 ? 8 : 16;           // query rows a softmax thread takes of its token
+    static constexpr int kSoftmaxWarps = 4 * (R / kRowsPerThread);  // R / kRowsPerThread warps per TMEM lane quadrant
     static constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
     static constexpr int kTotal = kTileBytes + kNumBars * 8 + 16;
     static_assert(R == 16 || R == 32 || R == 64, "query rows are padded to a power of two in [16, 64]");
@@ -70,13 +71,13 @@ __device__ __forceinline__ uint64_t desc_mnmajor_rows(uint32_t smem_addr, uint32
 
 constexpr float kTRescaleThreshold = 8.0f;  // log2 units: P may grow to 2^8 before the references are raised
 
-// OR over the 256 softmax threads (named barrier 1).
-__device__ __forceinline__ bool bar_or_256(bool v) {
+// OR over the `nthreads` softmax threads (named barrier 1).
+__device__ __forceinline__ bool bar_or(bool v, int nthreads) {
     uint32_t r;
     asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\tbarrier.cta.red.or.pred q, 1, 256, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\tbarrier.cta.red.or.pred q, 1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
         : "=r"(r)
-        : "r"((uint32_t)v)
+        : "r"((uint32_t)v), "r"(nthreads)
         : "memory");
     return r != 0;
 }
@@ -102,9 +103,10 @@ __global__ void __launch_bounds__(GqaTSmem<R>::kThreads, 1)
 decode_gqa_t_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmV) {
     using L = GqaTSmem<R>;
-    constexpr int RW = R / 2;                // query rows per softmax thread (the other half belongs to the partner warp)
-    constexpr int CH = RW < 16 ? RW : 16;    // rows handled per pass (TMEM columns per load): keeps the live registers low
+    constexpr int RW = L::kRowsPerThread;    // query rows per softmax thread (the others belong to its partner warps)
+    constexpr int CH = RW;                   // rows handled per pass (TMEM columns per load)
     constexpr int NCH = RW / CH;
+    constexpr int kSmT = 32 * L::kSoftmaxWarps;  // softmax threads
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* tiles = smem_raw;
     if ((smem_u32(tiles) & 1023u) != 0) {  // swizzled tiles need 1 KB alignment
@@ -263,7 +265,7 @@ decode_gqa_t_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ, 
     } else {
         // ------------------------------------------------------------------ softmax: one TMEM lane = one token per thread
         const int q = warp & 3;
-        const int half = (warp - 2) >> 2;  // which half of the query rows this warp takes: rows [half * RW, +RW)
+        const int half = (warp - 2) >> 2;  // which part of the query rows this warp takes: rows [half * RW, +RW)
         const int r0 = half * RW;
         const int tl = q * 32 + lane;  // token within the tile == TMEM lane (and value column in the epilogue)
         const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -321,7 +323,7 @@ decode_gqa_t_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ, 
                         xs[c] = vis ? __uint_as_float(x[c]) * p.scale_log2 : -INFINITY;
                         grow |= xs[c] > m_ref[rl] + kTRescaleThreshold;
                     }
-                    if (bar_or_256(grow || !okl)) {
+                    if (bar_or(grow || !okl, kSmT)) {
                         if (ab.raised()) { ok = false; break; }  // same answer in every thread: the flag was set before the barrier
                         // raise the references of this chunk's rows to the tile's true maxima and rescale O^T
                         float* redw = red + q * R + r0 + ch * CH;
@@ -330,7 +332,7 @@ decode_gqa_t_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ, 
                             const float wm = warp_max_redux(xs[c]);
                             if (lane == 0) redw[c] = wm;
                         }
-                        named_bar_sync(1, 256);
+                        named_bar_sync(1, kSmT);
                         float factor[CH];
                         bool any = false;
 #pragma unroll
@@ -343,7 +345,7 @@ decode_gqa_t_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ, 
                             l[rl] *= factor[c];
                             m_ref[rl] = mn;
                         }
-                        named_bar_sync(1, 256);  // red may be rewritten by the next chunk / tile
+                        named_bar_sync(1, kSmT);  // red may be rewritten by the next chunk / tile
                         // (`any` is the same in the threads of a warp -- they hold the same rows -- but not across the two
                         // halves, which rescale their own columns of O^T; no barrier follows inside this branch)
                         if (any && t > 0) {
@@ -399,7 +401,7 @@ decode_gqa_t_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ, 
                     const float ws = warp_sum(l[ch * CH + c]);
                     if (lane == 0) redw[c] = ws;
                 }
-                named_bar_sync(1, 256);
+                named_bar_sync(1, kSmT);
                 uint32_t o[CH];
                 if (pc.n_tiles > 0 && ok) {  // warp-uniform
                     tmem_ld_n(lane_base + kColO + r0 + ch * CH, o, CH);
@@ -417,7 +419,7 @@ decode_gqa_t_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ, 
                     p.o_part[orow * p.d_v + vb * 128 + tl] = live ? __uint_as_float(o[c]) / Lt : 0.f;
                     if (vb == 0 && tl == 0) p.lse_part[orow] = live ? (m_ref[rl] + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
                 }
-                named_bar_sync(1, 256);
+                named_bar_sync(1, kSmT);
             }
             // O^T has been read: the next piece's first P.V may overwrite it
             tc_fence_before();
