@@ -184,10 +184,31 @@ def run(names, steps: int, warmup: int):
         torch.cuda.empty_cache()
 
 
+def markdown(path: str) -> None:
+    """Prints the JSON lines of an earlier run as the table the benchmark spec carries."""
+    print("| config | path | s_q | split plan | pieces/seq | decode kernel µs | path µs | tokens/s (path) | GB/s | TFLOP/s | "
+          "of measured roofline | of nominal roofline |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+    with open(path) as fh:
+        for line in fh:
+            r = json.loads(line)
+            if "layout" in r:
+                continue
+            plan = f"{r['plan']}, {'S=' if r['plan'] == 'fixed' else ''}{r['slots']}{'' if r['plan'] == 'fixed' else ' slots'}"
+            meas = r.get("frac_of_measured_roofline", r.get("frac_of_fallback_roofline"))
+            print(f"| {r['workload']} | {r['path']} | {r['s_q']} | {plan} | {r['pieces_per_sequence']:.2f} | {r['kernel_us']} | "
+                  f"{r['path_us']} | {r['tokens_per_s']:,} | {r['gbs']:.0f} | {r['tflops']:.0f} | {meas:.3f} | "
+                  f"{r['frac_of_nominal_roofline']:.3f} |")
+
+
 if __name__ == "__main__":
     ap = argparse.ArgumentParser()
     ap.add_argument("--workloads", default="C1,C2,C3,C4")
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--markdown", default="", help="print the JSON lines of an earlier run (a file) as a markdown table and exit")
     a = ap.parse_args()
-    run(a.workloads.split(","), a.steps, a.warmup)
+    if a.markdown:
+        markdown(a.markdown)
+    else:
+        run(a.workloads.split(","), a.steps, a.warmup)
