@@ -7,6 +7,7 @@
 #include "../../include/gqla.h"
 #include "common.cuh"
 #include "tc_decode_absorb.cuh"
+#include "tc_decode_absorb_t.cuh"
 #include "tc_decode_gqa.cuh"
 #include "tc_decode_gqa_t.cuh"
 #include "tc_decode_gqa_fp8.cuh"
@@ -20,6 +21,10 @@
 // say otherwise; beyond it the row-replicating kernel runs (its replication factor 128/R is then 2 or 1).
 #ifndef GQLA_GQA_TOKENS_MAX_ROWS
 #define GQLA_GQA_TOKENS_MAX_ROWS 32
+#endif
+// Likewise for the absorb path: largest (padded) h_q * s_q served by its tokens-on-M kernel by default.
+#ifndef GQLA_ABSORB_TOKENS_MAX_ROWS
+#define GQLA_ABSORB_TOKENS_MAX_ROWS 32
 #endif
 
 namespace gqla {
@@ -83,6 +88,26 @@ inline int sm_count() {
 
 inline int absorb_resident_pairs();
 
+// Query rows of the absorb path's tokens-on-M kernel (tc_decode_absorb_t.cuh): h_q * s_q padded to 16 or 32.
+inline int absorb_rows_t(const gqla_dims& d, int32_t s_q) {
+    const int r = next_pow2(d.h_q * s_q);
+    return r < 16 ? 16 : r;
+}
+// Which absorb kernel serves a shape: the tokens-on-M kernel up to 32 query rows (a quarter of the pair kernel's
+// tile), the pair kernel beyond.  GQLA_ABSORB_KERNEL=rows|tokens overrides the choice for the shapes both cover,
+// h_q * s_q <= 32 (read once per process; a tuning aid).
+inline bool absorb_prefers_tokens(const gqla_dims& d, int32_t s_q) {
+    static const int forced = []() {
+        const char* e = getenv("GQLA_ABSORB_KERNEL");
+        if (e == nullptr) return 0;
+        return e[0] == 't' ? 1 : (e[0] == 'r' ? 2 : 0);
+    }();
+    const int rows_t = absorb_rows_t(d, s_q);
+    if (rows_t > 32) return false;  // 16 rows per softmax thread spill: the pair kernel is faster there
+    if (forced != 0) return forced == 1;
+    return rows_t <= GQLA_ABSORB_TOKENS_MAX_ROWS;
+}
+
 // Workers of the balanced plan: the GQA path runs one CTA per SM and keeps the cut points of all g
 // groups identical (so the CTAs of the g groups read one k_R tile together): W = SMs / g workers per
 // group.  The absorb path runs one CTA pair per two SMs: W = (SMs / 2) / row_blocks per row block.
@@ -91,6 +116,7 @@ inline int32_t tc_balanced_workers(const gqla_dims& d, int32_t s_q, int32_t path
     const int sms = sm_count();
     if (sms <= 0) return 0;
     if (path == 1) return sms / d.g > 0 ? sms / d.g : 0;
+    if (absorb_prefers_tokens(d, s_q)) return sms;  // one persistent CTA per SM
     const int row_blocks = (s_q * d.h_q + 127) / 128;
     const int pairs = absorb_resident_pairs();
     return pairs / row_blocks > 0 ? pairs / row_blocks : 0;
@@ -296,6 +322,15 @@ inline gqla_status tc_combine_up_proj(const gqla_dims& d, gqla_dtype dtype, int3
                : GQLA_ERR_CUDA;
 }
 
+template <int R>
+inline cudaError_t absorb_t_launch(const tc::AbsorbParams& p, const CUtensorMap& q, const CUtensorMap& c, unsigned grid,
+                                   cudaStream_t st) {
+    auto kern = tc::decode_absorb_t_kernel<R>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AbsorbTSmem<R>::kTotal);
+    if (e != cudaSuccess) return e;
+    return tc::launch_pdl(kern, dim3(grid), dim3(tc::AbsorbTSmem<R>::kThreads), tc::AbsorbTSmem<R>::kTotal, st, p, q, c);
+}
+
 inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, float scale, int32_t S,
                                     const void* q_hat, const void* cache, int64_t cache_row_stride,
                                     int64_t cache_rows, const RowMap& rows, const int32_t* seqlens,
@@ -315,11 +350,13 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
     if (rows.paged() && !balanced && S != 1) return GQLA_ERR_UNSUPPORTED;
     const int64_t pairs = balanced ? (int64_t)workers * row_blocks : (int64_t)B * S * row_blocks;
     if (2 * pairs > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
+    const bool tokens_on_m = absorb_prefers_tokens(d, s_q);
+    const int rows_t = absorb_rows_t(d, s_q);
     CUtensorMap tmQ, tmC;
     {
         const uint64_t dims[2] = {(uint64_t)(d.r_kv + d.d_r), (uint64_t)B * rows_total};
         const uint64_t str[1] = {(uint64_t)(d.r_kv + d.d_r) * 2};
-        const uint32_t box[2] = {64, 64};
+        const uint32_t box[2] = {64, tokens_on_m ? (uint32_t)rows_t : 64u};  // beyond the last row: zero fill
         if (!tc::make_tmap_bf16(&tmQ, q_hat, 2, dims, str, box)) return GQLA_ERR_CUDA;
     }
     {
@@ -335,6 +372,12 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
     p.rows = rows; p.seqlens = seqlens; p.o_part = o_part; p.lse_part = lse_part; p.status = status;
     p.o_final = (__nv_bfloat16*)o_final;
     if (o_final != nullptr && (balanced || S != 1)) return GQLA_ERR_UNSUPPORTED;
+    if (tokens_on_m) {
+        const unsigned grid = (unsigned)(balanced ? workers : B * S);  // single CTAs: W of them, or one per piece
+        const cudaError_t e = rows_t == 16 ? absorb_t_launch<16>(p, tmQ, tmC, grid, st)
+                                           : absorb_t_launch<32>(p, tmQ, tmC, grid, st);
+        return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
+    }
     auto kern = tc::decode_absorb_tc_kernel<0>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::AbsorbSmem::kTotal) != cudaSuccess)
         return GQLA_ERR_CUDA;

@@ -581,6 +581,37 @@ def test_both_gqa_kernels_on_the_shapes_both_cover(kernel):
     assert res.returncode == 0 and "kernel-ok" in res.stdout, res.stdout[-2000:] + res.stderr[-4000:]
 
 
+@pytest.mark.parametrize("kernel", ["rows", "tokens"])
+def test_both_absorb_kernels_on_the_shapes_both_cover(kernel):
+    """Two tensor-core kernels serve the absorb path: tokens on the MMA's M axis for h_q * s_q <= 32 (every cache tile
+    fetched once and used as K and as V; the default there) and the CTA-pair kernel with the query rows on M.
+    GQLA_ABSORB_KERNEL forces either one where both apply; the choice is read once per process, so each runs the
+    ragged parity cases (fixed, balanced and whole-sequence plans) in a process of its own."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = (
+        "import numpy as np, torch\n"
+        "from paper_2605_15250_b200 import binding as B, synth\n"
+        "from tests.parity_util import end_to_end, stagewise\n"
+        "sl = np.array([700, 0, 129, 2050, 64, 1, 63, 65], dtype=np.int32)\n"
+        "for dims, s_q in ((dict(h_q=32, g=8, d_h=128, r_kv=512, d_r=64), 1), (dict(h_q=16, g=8, d_h=128, r_kv=512, d_r=64), 2),\n"
+        "                  (dict(h_q=28, g=4, d_h=128, r_kv=512, d_r=64), 1), (dict(h_q=8, g=8, d_h=128, r_kv=512, d_r=64), 2),\n"
+        "                  (dict(h_q=8, g=4, d_h=128, r_kv=512, d_r=64), 3)):\n"
+        "    w = synth.Workload('k', batch=8, s_q=s_q, dtype='bf16', seed=9, **dims)\n"
+        "    d = B.make_dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)\n"
+        "    sms = torch.cuda.get_device_properties(0).multi_processor_count\n"
+        "    assert B.gqla_balanced_workers(d, torch.bfloat16, s_q, 'absorb') == (sms if '%s' == 'tokens' else sms // 2)\n"
+        "    stagewise(w, sl, 3, q_gain=4.0)\n"
+        "    for S in (1, 4, -3):\n"
+        "        end_to_end(w, sl, S, q_gain=4.0, paths=('absorb',))\n"
+        "print('kernel-ok')\n") % kernel
+    env = dict(os.environ, GQLA_ABSORB_KERNEL=kernel, PYTHONPATH=root)
+    res = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, env=env, cwd=root, timeout=900)
+    assert res.returncode == 0 and "kernel-ok" in res.stdout, res.stdout[-2000:] + res.stderr[-4000:]
+
+
 def test_debug_build_index_checks_stay_silent():
     """The -DGQLA_DEBUG build (piece and tile index checks that record a code instead of trapping) runs the ragged
     parity case in a process of its own: outputs within tolerance, status word 0."""
