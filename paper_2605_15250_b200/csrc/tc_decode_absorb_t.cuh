@@ -12,8 +12,9 @@
 // the first product and, its first eight boxes, as the V operand of the second: every cache byte enters shared memory
 // once.  Two tile stages; a stage is released when the tile's P.V has completed.  M = 64 keeps two tiles resident
 // beside Qh (with 128-token tiles one stage alone takes 144 KB); its accumulator sits in TMEM lanes 0-15 of each of
-// the four lane quadrants (row i of the tile -> lane 32 * (i / 16) + i % 16), so softmax thread `lane` < 16 of a warp
-// in quadrant q owns token 16 q + lane.  The softmax follows tc_decode_gqa_t.cuh: references shared by all threads,
+// the four lane quadrants (row i of the tile -> lane 32 * (i / 16) + i % 16); the softmax warps read it with
+// tcgen05.ld.16x256b, which spreads those 16 lanes over all 32 threads (two tokens x two query rows per thread and
+// eight-column load).  The softmax follows tc_decode_gqa_t.cuh: references shared by all threads,
 // one barrier.red.or per tile, true row maxima only when a score outgrows its reference by 2^8, row sums met once
 // per piece.  O^T has four blocks of R TMEM columns (latent columns [128 m, 128 m + 128) in the lanes); every row
 // leaves as 4 x 128 consecutive values, as fp32 partials or, for a whole-sequence call, as the final bf16 row.
@@ -253,14 +254,16 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
         }
     } else {
         // ------------------------------------------------------------------ softmax
+        // An M = 64 accumulator occupies lanes 0-15 of each TMEM lane quadrant.  tcgen05.ld.16x256b hands those 16 lanes
+        // x 8 columns to all 32 threads of the warp: thread t gets the scores of tokens t/4 and t/4 + 8 of its quadrant
+        // for the two query rows 2 (t % 4), 2 (t % 4) + 1 of the warp's eight -- every lane works.
         const int q = warp & 3;
-        const int half = (warp - 2) >> 2;    // rows [half * RW, +RW) of the R query rows
+        const int half = (warp - 2) >> 2;    // the warp's rows: [half * RW, +RW) of the R query rows
         const int r0 = half * RW;
-        const bool has_token = lane < 16;    // an M = 64 accumulator uses lanes 0-15 of each quadrant
-        const int tk = q * 16 + lane;        // token within the tile (lanes < 16)
+        const int c2 = 2 * (lane & 3);       // the thread's rows: r0 + c2, r0 + c2 + 1
         const int tl = q * 32 + lane;        // TMEM lane == latent column within a block in the epilogue
         const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
-        float m_ref[RW], l[RW];
+        float m_ref[2], l[2];
 
         while (walk.next(pc)) {
             const int32_t T = p.seqlens[pc.b];
@@ -271,96 +274,98 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
                 for (int kk = pc.fill_begin; kk < pc.fill_end; ++kk) p.lse_part[(slot0 + kk) * p.rows_total + tl] = -INFINITY;
             if (pc.n_tiles == 0 && p.balanced) continue;
             const int nt = pc.n_tiles == 0 ? 0 : (pc.tok_end - pc.tok_begin + TK - 1) / TK;
-#pragma unroll
-            for (int r = 0; r < RW; ++r) { m_ref[r] = -INFINITY; l[r] = 0.f; }
+            m_ref[0] = m_ref[1] = -INFINITY;
+            l[0] = l[1] = 0.f;
             bool ok = true;
 
             for (int t = 0; t < nt && ok; ++t) {
                 const int n = gt + t;
                 const int s = n & 1;
-                const int pbi = n % L::kPBufs;
                 // a failed wait raises the CTA's abort flag; the warps agree on leaving at the barrier below
                 bool okl = __all_sync(0xffffffffu, mbar_wait_fast(&s_full[s], (n >> 1) & 1, ab, 7));
                 tc_fence_after();
                 // (the P^T buffer was last read by P.V(n-2), which the issuer queued before S^T(n): MMAs complete in
                 // issue order, so S^T(n) having landed means that P.V(n-2) has read it)
-                // query row r = pq * h_q + head; position pq sees the tokens below T - (s_q - 1 - pq)
-                const int ta = pc.tok_begin + t * TK + tk;
-                const int pq_min = p.s_q - (T - ta) > 0 ? p.s_q - (T - ta) : 0;
-                const int r_lo = (has_token && ta < pc.tok_end) ? pq_min * p.h_q : R;
-                const int r_hi = p.rows_total;
-                uint8_t* prow = p_smem + pbi * L::kPBuf + tk * L::kPRow;
-                const uint32_t pswz = ((uint32_t)(tk * L::kPRow) >> 7) & ((1u << L::kPSwzBits) - 1);
-                uint32_t x[RW];
-                float xs[RW];
-                bool grow = false;
+                uint32_t x[4] = {0u, 0u, 0u, 0u};
                 if (okl) {
-                    tmem_ld_n(lane_base + kColS + (uint32_t)s * R + r0, x, RW);
+                    tmem_ld_16x256b(lane_base + kColS + (uint32_t)s * R + r0, x);
                     tmem_wait_ld();
                 }
+                // query row r = pq * h_q + head; position pq sees the tokens below T - (s_q - 1 - pq)
+                float xs[4];  // [token A row 0, token A row 1, token B row 0, token B row 1]
+                bool grow = false;
 #pragma unroll
-                for (int c = 0; c < RW; ++c) {
-                    const int r = r0 + c;
-                    const bool vis = okl && r >= r_lo && r < r_hi;
-                    xs[c] = vis ? __uint_as_float(x[c]) * p.scale_log2 : -INFINITY;
-                    grow |= xs[c] > m_ref[c] + kTRescaleThreshold;
+                for (int h = 0; h < 2; ++h) {
+                    const int ta = pc.tok_begin + t * TK + q * 16 + (lane >> 2) + 8 * h;
+                    const int pq_min = p.s_q - (T - ta) > 0 ? p.s_q - (T - ta) : 0;
+                    const int r_lo = ta < pc.tok_end ? pq_min * p.h_q : R;
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const int r = r0 + c2 + j;
+                        const bool vis = okl && r >= r_lo && r < p.rows_total;
+                        xs[2 * h + j] = vis ? __uint_as_float(x[2 * h + j]) * p.scale_log2 : -INFINITY;
+                        grow |= xs[2 * h + j] > m_ref[j] + kTRescaleThreshold;
+                    }
                 }
                 if (bar_or(grow || !okl, kSmT)) {
                     if (ab.raised()) { ok = false; break; }  // same answer in every thread: the flag was set before the barrier
-                    float* redw = red + q * R + r0;
-#pragma unroll
-                    for (int c = 0; c < RW; ++c) {
-                        const float wm = warp_max_redux(xs[c]);
-                        if (lane == 0) redw[c] = wm;
-                    }
-                    named_bar_sync(1, kSmT);
-                    float factor[RW];
+                    float factor[2];
                     bool any = false;
 #pragma unroll
-                    for (int c = 0; c < RW; ++c) {
-                        const int r = r0 + c;
+                    for (int j = 0; j < 2; ++j) {  // the row's maximum over the warp's 16 tokens: lanes with equal t % 4
+                        float mx = fmaxf(xs[j], xs[2 + j]);
+                        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                        if (lane < 4) red[q * R + r0 + c2 + j] = mx;
+                    }
+                    named_bar_sync(1, kSmT);
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const int r = r0 + c2 + j;
                         const float tm = fmaxf(fmaxf(red[r], red[R + r]), fmaxf(red[2 * R + r], red[3 * R + r]));
-                        const float mn = fmaxf(m_ref[c], tm);
-                        factor[c] = mn > m_ref[c] ? ex2(m_ref[c] - mn) : 1.f;  // ex2(-inf) = 0 on first use
-                        any |= mn > m_ref[c];
-                        l[c] *= factor[c];
-                        m_ref[c] = mn;
+                        const float mn = fmaxf(m_ref[j], tm);
+                        factor[j] = mn > m_ref[j] ? ex2(m_ref[j] - mn) : 1.f;  // ex2(-inf) = 0 on first use
+                        any |= mn > m_ref[j];
+                        l[j] *= factor[j];
+                        m_ref[j] = mn;
                     }
                     named_bar_sync(1, kSmT);  // red may be rewritten by the next tile
-                    if (any && t > 0) {
+                    if (__any_sync(0xffffffffu, any) && t > 0) {
                         // O^T may be rescaled only between P.V(n-1) completing and P.V(n) being issued
                         if (!__all_sync(0xffffffffu, mbar_wait(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, ab, 8))) {
                             okl = false;  // noticed by everybody at the next barrier
                         } else {
                             tc_fence_after();
+                            float f8[RW];  // factors of the warp's eight rows: row c is held by lanes with t % 4 == c / 2
+#pragma unroll
+                            for (int c = 0; c < RW; ++c) f8[c] = __shfl_sync(0xffffffffu, factor[c & 1], c >> 1);
 #pragma unroll
                             for (int m = 0; m < 4; ++m) {
                                 uint32_t o[RW];
                                 tmem_ld_n(lane_base + kColO + m * R + r0, o, RW);
                                 tmem_wait_ld();
 #pragma unroll
-                                for (int c = 0; c < RW; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * factor[c]);
+                                for (int c = 0; c < RW; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f8[c]);
                                 tmem_st_n(lane_base + kColO + m * R + r0, o, RW);
                             }
                             tmem_wait_st();
                         }
                     }
                 }
-                // probabilities of this token for the thread's rows -> its row of P^T, eight rows per 16-byte store
-                uint32_t pk[RW / 2];
+                // probabilities: a bf16 pair (the thread's two rows) into each of its two tokens' rows of P^T
+                const int pbi = n % L::kPBufs;
 #pragma unroll
-                for (int c = 0; c < RW; c += 2) {
-                    const float e0 = xs[c] > -INFINITY ? ex2(xs[c] - m_ref[c]) : 0.f;
-                    const float e1 = xs[c + 1] > -INFINITY ? ex2(xs[c + 1] - m_ref[c + 1]) : 0.f;
-                    l[c] += e0;
-                    l[c + 1] += e1;
-                    pk[c / 2] = pack_bf16(e0, e1);
-                }
-                if (has_token) {
-#pragma unroll
-                    for (int i = 0; i < RW / 8; ++i)
-                        *reinterpret_cast<uint4*>(prow + ((((uint32_t)(r0 / 8 + i)) ^ pswz) << 4)) =
-                            make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                for (int h = 0; h < 2; ++h) {
+                    const float e0 = xs[2 * h] > -INFINITY ? ex2(xs[2 * h] - m_ref[0]) : 0.f;
+                    const float e1 = xs[2 * h + 1] > -INFINITY ? ex2(xs[2 * h + 1] - m_ref[1]) : 0.f;
+                    l[0] += e0;
+                    l[1] += e1;
+                    const uint32_t off = (uint32_t)(q * 16 + (lane >> 2) + 8 * h) * L::kPRow;  // the token's row of P^T
+                    const uint32_t pswz = (off >> 7) & ((1u << L::kPSwzBits) - 1);             // XOR of its 16-byte chunks
+                    const uint32_t col = (uint32_t)(r0 + c2) * 2;                              // byte of row r0 + c2 in it
+                    *reinterpret_cast<uint32_t*>(p_smem + pbi * L::kPBuf + off + (((col >> 4) ^ pswz) << 4) + (col & 15)) =
+                        pack_bf16(e0, e1);
                 }
                 fence_proxy_async_smem();  // generic-proxy writes of P^T -> visible to the tensor core
                 tc_fence_before();
@@ -372,25 +377,32 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
             const int n_last = gt + nt - 1;
             if (nt > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[n_last & 1], (n_last >> 1) & 1, ab, 9));
             tc_fence_after();
-            float* redw = red + q * R + r0;
 #pragma unroll
-            for (int c = 0; c < RW; ++c) {
-                const float ws = warp_sum(l[c]);
-                if (lane == 0) redw[c] = ws;
+            for (int j = 0; j < 2; ++j) {  // the row's sum over the warp's tokens: lanes with equal t % 4
+                float ws = l[j];
+                ws += __shfl_xor_sync(0xffffffffu, ws, 4);
+                ws += __shfl_xor_sync(0xffffffffu, ws, 8);
+                ws += __shfl_xor_sync(0xffffffffu, ws, 16);
+                if (lane < 4) red[q * R + r0 + c2 + j] = ws;
             }
             named_bar_sync(1, kSmT);
-            float inv[RW];
+            const int64_t out_row0 = (p.o_final != nullptr ? (int64_t)pc.b : slot0 + pc.k) * p.rows_total;
+            if (q == 0 && lane < 4 && p.lse_part != nullptr) {
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int r = r0 + c2 + j;
+                    const float Lt = (red[r] + red[R + r]) + (red[2 * R + r] + red[3 * R + r]);
+                    const bool live = ok && nt > 0 && Lt > 0.f && m_ref[j] > -INFINITY;
+                    if (r < p.rows_total) p.lse_part[out_row0 + r] = live ? (m_ref[j] + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
+                }
+            }
+            float inv[RW];  // of the warp's eight rows (a lane is a latent column of all of them)
 #pragma unroll
             for (int c = 0; c < RW; ++c) {
                 const int r = r0 + c;
                 const float Lt = (red[r] + red[R + r]) + (red[2 * R + r] + red[3 * R + r]);
-                const bool live = ok && nt > 0 && Lt > 0.f && m_ref[c] > -INFINITY;
-                inv[c] = live ? 1.f / Lt : 0.f;
-                if (tl == 0 && r < p.rows_total && p.lse_part != nullptr)
-                    p.lse_part[(p.o_final != nullptr ? (int64_t)pc.b : slot0 + pc.k) * p.rows_total + r] =
-                        live ? (m_ref[c] + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
+                inv[c] = (ok && nt > 0 && Lt > 0.f) ? 1.f / Lt : 0.f;
             }
-            const int64_t out_row0 = (p.o_final != nullptr ? (int64_t)pc.b : slot0 + pc.k) * p.rows_total;
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
                 uint32_t o[RW];

@@ -149,7 +149,7 @@ def time_case(dec: GqlaDecoder, w: synth.Workload, x: dict, path: str, S: int, s
     return out
 
 
-def run(names, steps: int, warmup: int):
+def run(names, steps: int, warmup: int, paths=("absorb", "gqa")):
     gbuild.build()
     B.lib()
     assert torch.cuda.is_available(), "the sweep needs a CUDA device"
@@ -164,13 +164,14 @@ def run(names, steps: int, warmup: int):
     for name in names:
         base = synth.WORKLOADS[name]
         dec = None
-        for path, s_q, plans in cases[name]:
+        todo = [c for c in cases[name] if c[0] in paths]
+        for path, s_q, plans in todo:
             w = base.with_(s_q=s_q)
             x = synth.make_inputs(w)
             if dec is None:
                 dec = GqlaDecoder(w.h_q, w.g, w.d_h, w.r_kv, w.d_r, x["w_uk"].to(dev), x["w_uv"].to(dev),
                                   x["cache"].to(dev), x["seq_start"].to(dev), x["seqlens"].to(dev), w.scale)
-                if any(p == "gqa" for p, _, _ in cases[name]):
+                if any(p == "gqa" for p, _, _ in todo):
                     dec.expand_cache()
             for S in plans:
                 res = time_case(dec, w, x, path, S, steps, warmup)
@@ -206,9 +207,10 @@ if __name__ == "__main__":
     ap.add_argument("--workloads", default="C1,C2,C3,C4")
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--paths", default="absorb,gqa", help="decode paths to time (the GQA path expands the cache first)")
     ap.add_argument("--markdown", default="", help="print the JSON lines of an earlier run (a file) as a markdown table and exit")
     a = ap.parse_args()
     if a.markdown:
         markdown(a.markdown)
     else:
-        run(a.workloads.split(","), a.steps, a.warmup)
+        run(a.workloads.split(","), a.steps, a.warmup, tuple(a.paths.split(",")))
