@@ -319,7 +319,9 @@ gqla_status gqla_split_plan(int32_t seqlen, int32_t num_splits, int32_t* begin, 
 gqla_status gqla_balanced_plan(const int32_t* seqlens, int32_t B, int32_t s_cap, int32_t workers, int32_t* begin,
                                int32_t* end, int32_t* worker);
 /* Number of workers W a balanced decode call of this shape is cut for on the CURRENT device
- * (path: 0 = absorb, 1 = GQA); 0 if such a call falls back to the fixed plan; -1 on error. */
+ * (path: 0 = absorb, 1 = GQA); 0 if such a call falls back to the fixed plan; -1 on error.  The figure is that of
+ * the bf16 / f32 calls; gqla_decode_absorb_fp8 always runs on CTA pairs and cuts for half the SMs per 128 query
+ * rows, where the bf16 call of a shape with at most 64 query rows cuts for one worker per SM. */
 int32_t gqla_balanced_workers(const gqla_dims* dims, gqla_dtype dtype, int32_t s_q, int32_t path);
 /* Rows visible to query p of an s_q-token step: max(0, seqlen - (s_q-1-p)). */
 int32_t gqla_visible_limit(int32_t seqlen, int32_t s_q, int32_t p);

@@ -222,6 +222,13 @@ __device__ __forceinline__ void tmem_ld_16x256b(uint32_t taddr, uint32_t* r) {
                  : "r"(taddr)
                  : "memory");
 }
+// Sixteen columns: r[4..7] are r[0..3] of the columns 8 further on.
+__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t* r) {
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_st4(uint32_t taddr, const uint32_t* r) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
                  "r"(r[2]), "r"(r[3])
@@ -361,6 +368,16 @@ __device__ __forceinline__ void umma_ss2_lo(uint32_t d_tmem, uint32_t a_lo, uint
         "mov.b64 da, {%1, %4};\n\tmov.b64 db, {%2, %4};\n\tsetp.ne.b32 p, %5, 0;\n\t"
         "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem),
         "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(kDescHiSw128), "n"(ACCUMULATE ? 1 : 0)
+        : "memory");
+}
+// The same for one CTA, with the two constant high words given and the accumulate flag a run-time value.
+__device__ __forceinline__ void umma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                           uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
+        "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\tsetp.ne.b32 p, %6, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // Arrives (once every MMA issued so far has finished) on the barrier at the same offset in every CTA of `mask`.

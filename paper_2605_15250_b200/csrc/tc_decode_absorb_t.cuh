@@ -1,5 +1,5 @@
 // Absorb-path split-KV flash decoding on tcgen05 with the TOKENS on the MMA's M axis (Eq. (mqa)), for models whose
-// h_q * s_q query rows fill only part of a 128-row MMA tile (the LLaMA-shaped setup of Sec. 5: h_q = 32).
+// h_q * s_q <= 64 query rows fill at most half of a 128-row MMA tile (the LLaMA-shaped setup of Sec. 5: h_q = 32).
 //
 // tc_decode_absorb.cuh pads the query rows to 128, so at h_q = 32 three quarters of its tensor work is padding and
 // the kernel runs at the pace of its MMAs, not of the cache stream.  Here both products are transposed, as in
@@ -19,12 +19,13 @@
 // per piece.  O^T has four blocks of R TMEM columns (latent columns [128 m, 128 m + 128) in the lanes); every row
 // leaves as 4 x 128 consecutive values, as fp32 partials or, for a whole-sequence call, as the final bf16 row.
 //
-// What it buys is power, not burst speed.  A tile fetched once has to stay in shared memory from its first product
-// until its second, i.e. through the softmax, so of the two 72 KB stages at most one is in flight while the other
-// is held: in a burst the cache streams no faster than under the pair kernel (h_q = 32, 128 sequences of 8-32 K
-// tokens, balanced plan: 583 us against 575 us on the same GPU).  Launched back to back for seconds under the power
-// cap, a quarter of the tensor work leaves the clocks at 1.80 GHz where the pair kernel's drop to 1.0 GHz: 622 us
-// against 707 us per launch.
+// Shared memory holds two tiles and one of them is always held by the softmax (a tile fetched once has to stay from its
+// first product until its second), so the producer also asks a later tile into L2 when it issues a load, and the held time
+// is kept short: the issuer polls instead of blocking, the softmax uses every lane.  Measured (h_q = 32, s_q = 1, 128
+// sequences of 8-32 K tokens, balanced plan, one GPU): 477 us in a burst against 523-539 us for the pair kernel; launched
+// back to back for seconds under the power cap, a quarter of the tensor work leaves the clocks at 1.79 GHz where the pair
+// kernel's drop to 1.26 GHz: 524 us against 620 us per launch.  With 64 rows (sixteen per softmax warp, one P^T buffer):
+// 566 against 582 us in a burst.
 #pragma once
 #include "common.cuh"
 #include "sched.cuh"
@@ -44,22 +45,22 @@ struct AbsorbTSmem {
     static constexpr int kStageBytes = 9 * kBox;              // 64 tokens x 576
     static constexpr int kStages = 2;
     static constexpr int kPRow = 2 * R;                       // one token's R probabilities (bf16)
-    static constexpr int kPSwzBits = R == 32 ? 2 : 1;         // swizzle span = row length (64 / 32 bytes)
+    static constexpr int kPSwzBits = R == 64 ? 3 : (R == 32 ? 2 : 1);  // swizzle span = row length (128 / 64 / 32 bytes)
     static constexpr int kPBuf = (kTile * kPRow + 1023) / 1024 * 1024;
-    static constexpr int kPBufs = 2;                          // P^T buffers: writing P(n) waits only for P.V(n-2)
+    static constexpr int kPBufs = R == 64 ? 1 : 2;            // P^T buffers (one where Qh takes 72 KB: P(n) waits for P.V(n-1))
     static constexpr int kGroup = 3 * kBox;                   // boxes land in groups of three, one barrier each
     static constexpr int kOffStage = kQBytes;
     static constexpr int kOffP = kOffStage + kStages * kStageBytes;
     static constexpr int kOffRed = kOffP + kPBufs * kPBuf;    // [4 quadrants][R] floats; also the plan scratch
-    static constexpr int kRowsPerThread = 8;
-    static constexpr int kSoftmaxWarps = 4 * (R / kRowsPerThread);
+    static constexpr int kRowsPerWarp = R == 64 ? 16 : 8;    // query rows (score columns) a softmax warp takes of its 16 tokens
+    static constexpr int kSoftmaxWarps = 4 * (R / kRowsPerWarp);
     static constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
     static constexpr int kRedBytes = 4 * R * 4 > (kThreads + 4) * 4 ? 4 * R * 4 : (kThreads + 4) * 4;
     static constexpr int kTileBytes = kOffRed + (kRedBytes + 15) / 16 * 16;
     // q_full q_empty o_free full[2][3] empty[2] s_full[2] p_ready[2] pv_done[2]
     static constexpr int kNumBars = 17;
     static constexpr int kTotal = kTileBytes + kNumBars * 8 + 16;
-    static_assert(R == 16 || R == 32, "query rows are padded to 16 or 32");
+    static_assert(R == 16 || R == 32 || R == 64, "query rows are padded to 16, 32 or 64");
     static_assert(kQBytes % 1024 == 0, "swizzled tiles start on 1 KB boundaries");
     static_assert(kTotal <= 232448, "shared memory budget of one CTA");
     static_assert(OneCtaPerSM<kTotal>::value, "");
@@ -75,7 +76,8 @@ template <int R>
 __global__ void __launch_bounds__(AbsorbTSmem<R>::kThreads, 1)
 decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmC) {
     using L = AbsorbTSmem<R>;
-    constexpr int RW = L::kRowsPerThread;
+    constexpr int RW = L::kRowsPerWarp;
+    constexpr int NJ = RW / 4;  // query rows per softmax thread
     constexpr int kSmT = 32 * L::kSoftmaxWarps;
     constexpr int TK = L::kTile;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -102,7 +104,7 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
 
     // TMEM columns: two score buffers of R columns, then four output blocks of R columns
     constexpr uint32_t kColS = 0, kColO = 2 * R;
-    constexpr uint32_t kTmemCols = 6 * R <= 128 ? 128 : 256;
+    constexpr uint32_t kTmemCols = 6 * R <= 128 ? 128 : (6 * R <= 256 ? 256 : 512);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const Abort ab{abort_flag, p.status};
@@ -199,14 +201,17 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
                                 tc_fence_after();
                                 const uint32_t v_addr = smem_u32(stage0 + s * L::kStageBytes);
                                 const uint32_t pb = p_addr0 + (n % L::kPBufs) * L::kPBuf;
+                                // descriptors stepped through their low words (the high words are constants): the
+                                // issuer's instructions per MMA are part of the time a tile stays held
+                                const uint64_t vd = desc_mnmajor_sw128(v_addr, L::kBox), pd = desc_mnmajor_rows(pb, L::kPRow);
+                                const uint32_t v_lo = (uint32_t)vd, v_hi = (uint32_t)(vd >> 32);
+                                const uint32_t p_lo = (uint32_t)pd, p_hi = (uint32_t)(pd >> 32);
 #pragma unroll
                                 for (int m = 0; m < 4; ++m)      // latent columns [128 m, +128): boxes 2m and 2m + 1
 #pragma unroll
                                     for (int ks = 0; ks < 4; ++ks)  // 16 tokens per step
-                                        umma_ss(tmem_base + kColO + m * R,
-                                                desc_mnmajor_sw128(v_addr + 2 * m * L::kBox + ks * 2048, L::kBox),
-                                                desc_mnmajor_rows(pb + ks * 16 * L::kPRow, L::kPRow), idesc_pv,
-                                                (pv_tile | ks) != 0);
+                                        umma_ss_lo(tmem_base + kColO + m * R, v_lo + ((2 * m * L::kBox + ks * 2048) >> 4), v_hi,
+                                                   p_lo + ((ks * 16 * L::kPRow) >> 4), p_hi, idesc_pv, (pv_tile | ks) != 0);
                                 umma_commit(&empty[s]);
                                 umma_commit(&pv_done[s]);
                                 ++pv_tile;
@@ -221,14 +226,15 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
                             tc_fence_after();
                             const uint32_t st = smem_u32(stage0 + s * L::kStageBytes);
                             const uint32_t d = tmem_base + kColS + (uint32_t)s * R;
+                            const uint32_t k_lo = desc_lo(desc_kmajor_sw128(st + 3 * s_grp * L::kBox));
+                            const uint32_t q_lo = desc_lo(desc_kmajor_sw128(q_addr + 3 * s_grp * L::kQBlock));
 #pragma unroll
-                            for (int kk = 0; kk < 3; ++kk) {
-                                const int kb = 3 * s_grp + kk;
+                            for (int kk = 0; kk < 3; ++kk)
 #pragma unroll
                                 for (int ks = 0; ks < 4; ++ks)
-                                    umma_ss(d, desc_kmajor_sw128(st + kb * L::kBox + ks * 32),
-                                            desc_kmajor_sw128(q_addr + kb * L::kQBlock + ks * 32), idesc_qk, (kb | ks) != 0);
-                            }
+                                    umma_ss_lo(d, k_lo + ((kk * L::kBox + ks * 32) >> 4), kDescHiSw128,
+                                               q_lo + ((kk * L::kQBlock + ks * 32) >> 4), kDescHiSw128, idesc_qk,
+                                               (uint32_t)(s_grp | kk | ks));
                             if (++s_grp == 3) {
                                 umma_commit(&s_full[s]);
                                 s_grp = 0;
@@ -256,14 +262,16 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
         // ------------------------------------------------------------------ softmax
         // An M = 64 accumulator occupies lanes 0-15 of each TMEM lane quadrant.  tcgen05.ld.16x256b hands those 16 lanes
         // x 8 columns to all 32 threads of the warp: thread t gets the scores of tokens t/4 and t/4 + 8 of its quadrant
-        // for the two query rows 2 (t % 4), 2 (t % 4) + 1 of the warp's eight -- every lane works.
+        // for the query rows 2 (t % 4), 2 (t % 4) + 1 of the warp's eight (and, with sixteen rows per warp, the same two of
+        // the second eight) -- every lane works.
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;    // the warp's rows: [half * RW, +RW) of the R query rows
         const int r0 = half * RW;
-        const int c2 = 2 * (lane & 3);       // the thread's rows: r0 + c2, r0 + c2 + 1
+        const int c2 = 2 * (lane & 3);       // the thread's rows: r0 + rj(j), rj(j) = c2 + (j & 1) + 8 (j >> 1)
         const int tl = q * 32 + lane;        // TMEM lane == latent column within a block in the epilogue
         const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
-        float m_ref[2], l[2];
+        float m_ref[NJ], l[NJ];
+        auto rj = [&](int j) -> int { return c2 + (j & 1) + 8 * (j >> 1); };
 
         while (walk.next(pc)) {
             const int32_t T = p.seqlens[pc.b];
@@ -274,8 +282,8 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
                 for (int kk = pc.fill_begin; kk < pc.fill_end; ++kk) p.lse_part[(slot0 + kk) * p.rows_total + tl] = -INFINITY;
             if (pc.n_tiles == 0 && p.balanced) continue;
             const int nt = pc.n_tiles == 0 ? 0 : (pc.tok_end - pc.tok_begin + TK - 1) / TK;
-            m_ref[0] = m_ref[1] = -INFINITY;
-            l[0] = l[1] = 0.f;
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) { m_ref[j] = -INFINITY; l[j] = 0.f; }
             bool ok = true;
 
             for (int t = 0; t < nt && ok; ++t) {
@@ -286,13 +294,14 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
                 tc_fence_after();
                 // (the P^T buffer was last read by P.V(n-2), which the issuer queued before S^T(n): MMAs complete in
                 // issue order, so S^T(n) having landed means that P.V(n-2) has read it)
-                uint32_t x[4] = {0u, 0u, 0u, 0u};
+                uint32_t x[2 * NJ];  // x[4 (j >> 1) + 2 h + (j & 1)]: token h (0: t/4, 1: t/4 + 8), row j of the thread
                 if (okl) {
-                    tmem_ld_16x256b(lane_base + kColS + (uint32_t)s * R + r0, x);
+                    if (NJ == 2) tmem_ld_16x256b(lane_base + kColS + (uint32_t)s * R + r0, x);
+                    else tmem_ld_16x256b_x2(lane_base + kColS + (uint32_t)s * R + r0, x);
                     tmem_wait_ld();
                 }
                 // query row r = pq * h_q + head; position pq sees the tokens below T - (s_q - 1 - pq)
-                float xs[4];  // [token A row 0, token A row 1, token B row 0, token B row 1]
+                float xs[2 * NJ];  // same order
                 bool grow = false;
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
@@ -300,29 +309,29 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
                     const int pq_min = p.s_q - (T - ta) > 0 ? p.s_q - (T - ta) : 0;
                     const int r_lo = ta < pc.tok_end ? pq_min * p.h_q : R;
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const int r = r0 + c2 + j;
+                    for (int j = 0; j < NJ; ++j) {
+                        const int r = r0 + rj(j), i = 4 * (j >> 1) + 2 * h + (j & 1);
                         const bool vis = okl && r >= r_lo && r < p.rows_total;
-                        xs[2 * h + j] = vis ? __uint_as_float(x[2 * h + j]) * p.scale_log2 : -INFINITY;
-                        grow |= xs[2 * h + j] > m_ref[j] + kTRescaleThreshold;
+                        xs[i] = vis ? __uint_as_float(x[i]) * p.scale_log2 : -INFINITY;
+                        grow |= xs[i] > m_ref[j] + kTRescaleThreshold;
                     }
                 }
                 if (bar_or(grow || !okl, kSmT)) {
                     if (ab.raised()) { ok = false; break; }  // same answer in every thread: the flag was set before the barrier
-                    float factor[2];
+                    float factor[NJ];
                     bool any = false;
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {  // the row's maximum over the warp's 16 tokens: lanes with equal t % 4
-                        float mx = fmaxf(xs[j], xs[2 + j]);
+                    for (int j = 0; j < NJ; ++j) {  // the row's maximum over the warp's 16 tokens: lanes with equal t % 4
+                        float mx = fmaxf(xs[4 * (j >> 1) + (j & 1)], xs[4 * (j >> 1) + 2 + (j & 1)]);
                         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
                         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
                         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-                        if (lane < 4) red[q * R + r0 + c2 + j] = mx;
+                        if (lane < 4) red[q * R + r0 + rj(j)] = mx;
                     }
                     named_bar_sync(1, kSmT);
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const int r = r0 + c2 + j;
+                    for (int j = 0; j < NJ; ++j) {
+                        const int r = r0 + rj(j);
                         const float tm = fmaxf(fmaxf(red[r], red[R + r]), fmaxf(red[2 * R + r], red[3 * R + r]));
                         const float mn = fmaxf(m_ref[j], tm);
                         factor[j] = mn > m_ref[j] ? ex2(m_ref[j] - mn) : 1.f;  // ex2(-inf) = 0 on first use
@@ -337,17 +346,20 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
                             okl = false;  // noticed by everybody at the next barrier
                         } else {
                             tc_fence_after();
-                            float f8[RW];  // factors of the warp's eight rows: row c is held by lanes with t % 4 == c / 2
 #pragma unroll
-                            for (int c = 0; c < RW; ++c) f8[c] = __shfl_sync(0xffffffffu, factor[c & 1], c >> 1);
+                            for (int cc = 0; cc < RW; cc += 8) {  // eight rows at a time
+                                float f8[8];  // row cc + c is row (c & 1) + 2 (cc >> 3) of the lanes with t % 4 == c / 2
 #pragma unroll
-                            for (int m = 0; m < 4; ++m) {
-                                uint32_t o[RW];
-                                tmem_ld_n(lane_base + kColO + m * R + r0, o, RW);
-                                tmem_wait_ld();
+                                for (int c = 0; c < 8; ++c) f8[c] = __shfl_sync(0xffffffffu, factor[(c & 1) + 2 * (cc >> 3)], c >> 1);
 #pragma unroll
-                                for (int c = 0; c < RW; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f8[c]);
-                                tmem_st_n(lane_base + kColO + m * R + r0, o, RW);
+                                for (int m = 0; m < 4; ++m) {
+                                    uint32_t o[8];
+                                    tmem_ld8(lane_base + kColO + m * R + r0 + cc, o);
+                                    tmem_wait_ld();
+#pragma unroll
+                                    for (int c = 0; c < 8; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f8[c]);
+                                    tmem_st8(lane_base + kColO + m * R + r0 + cc, o);
+                                }
                             }
                             tmem_wait_st();
                         }
@@ -355,17 +367,31 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
                 }
                 // probabilities: a bf16 pair (the thread's two rows) into each of its two tokens' rows of P^T
                 const int pbi = n % L::kPBufs;
+                uint32_t pk[NJ];  // [2 h + pair]: the bf16 pair of token h for the thread's row pair
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int jp = 0; jp < NJ; jp += 2) {
+                        const int i = 4 * (jp >> 1) + 2 * h;
+                        const float e0 = xs[i] > -INFINITY ? ex2(xs[i] - m_ref[jp]) : 0.f;
+                        const float e1 = xs[i + 1] > -INFINITY ? ex2(xs[i + 1] - m_ref[jp + 1]) : 0.f;
+                        l[jp] += e0;
+                        l[jp + 1] += e1;
+                        pk[(NJ / 2) * h + (jp >> 1)] = pack_bf16(e0, e1);
+                    }
+                // a single P^T buffer is still being read by P.V(n-1)
+                if (L::kPBufs == 1 && t > 0 && okl)
+                    okl = __all_sync(0xffffffffu, mbar_wait(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, ab, 8));
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const float e0 = xs[2 * h] > -INFINITY ? ex2(xs[2 * h] - m_ref[0]) : 0.f;
-                    const float e1 = xs[2 * h + 1] > -INFINITY ? ex2(xs[2 * h + 1] - m_ref[1]) : 0.f;
-                    l[0] += e0;
-                    l[1] += e1;
                     const uint32_t off = (uint32_t)(q * 16 + (lane >> 2) + 8 * h) * L::kPRow;  // the token's row of P^T
                     const uint32_t pswz = (off >> 7) & ((1u << L::kPSwzBits) - 1);             // XOR of its 16-byte chunks
-                    const uint32_t col = (uint32_t)(r0 + c2) * 2;                              // byte of row r0 + c2 in it
-                    *reinterpret_cast<uint32_t*>(p_smem + pbi * L::kPBuf + off + (((col >> 4) ^ pswz) << 4) + (col & 15)) =
-                        pack_bf16(e0, e1);
+#pragma unroll
+                    for (int jp = 0; jp < NJ; jp += 2) {
+                        const uint32_t col = (uint32_t)(r0 + rj(jp)) * 2;                      // byte of that row pair in it
+                        *reinterpret_cast<uint32_t*>(p_smem + pbi * L::kPBuf + off + (((col >> 4) ^ pswz) << 4) + (col & 15)) =
+                            pk[(NJ / 2) * h + (jp >> 1)];
+                    }
                 }
                 fence_proxy_async_smem();  // generic-proxy writes of P^T -> visible to the tensor core
                 tc_fence_before();
@@ -378,46 +404,49 @@ decode_absorb_t_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMap
             if (nt > 0 && ok) ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[n_last & 1], (n_last >> 1) & 1, ab, 9));
             tc_fence_after();
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {  // the row's sum over the warp's tokens: lanes with equal t % 4
+            for (int j = 0; j < NJ; ++j) {  // the row's sum over the warp's tokens: lanes with equal t % 4
                 float ws = l[j];
                 ws += __shfl_xor_sync(0xffffffffu, ws, 4);
                 ws += __shfl_xor_sync(0xffffffffu, ws, 8);
                 ws += __shfl_xor_sync(0xffffffffu, ws, 16);
-                if (lane < 4) red[q * R + r0 + c2 + j] = ws;
+                if (lane < 4) red[q * R + r0 + rj(j)] = ws;
             }
             named_bar_sync(1, kSmT);
             const int64_t out_row0 = (p.o_final != nullptr ? (int64_t)pc.b : slot0 + pc.k) * p.rows_total;
             if (q == 0 && lane < 4 && p.lse_part != nullptr) {
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const int r = r0 + c2 + j;
+                for (int j = 0; j < NJ; ++j) {
+                    const int r = r0 + rj(j);
                     const float Lt = (red[r] + red[R + r]) + (red[2 * R + r] + red[3 * R + r]);
                     const bool live = ok && nt > 0 && Lt > 0.f && m_ref[j] > -INFINITY;
                     if (r < p.rows_total) p.lse_part[out_row0 + r] = live ? (m_ref[j] + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
                 }
             }
-            float inv[RW];  // of the warp's eight rows (a lane is a latent column of all of them)
 #pragma unroll
-            for (int c = 0; c < RW; ++c) {
-                const int r = r0 + c;
-                const float Lt = (red[r] + red[R + r]) + (red[2 * R + r] + red[3 * R + r]);
-                inv[c] = (ok && nt > 0 && Lt > 0.f) ? 1.f / Lt : 0.f;
-            }
+            for (int cc = 0; cc < RW; cc += 8) {  // eight rows at a time (a lane is a latent column of all of them)
+                float inv[8];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                uint32_t o[RW];
-                if (nt > 0 && ok) {  // warp-uniform
-                    tmem_ld_n(lane_base + kColO + m * R + r0, o, RW);
-                    tmem_wait_ld();
+                for (int c = 0; c < 8; ++c) {
+                    const int r = r0 + cc + c;
+                    const float Lt = (red[r] + red[R + r]) + (red[2 * R + r] + red[3 * R + r]);
+                    inv[c] = (ok && nt > 0 && Lt > 0.f) ? 1.f / Lt : 0.f;
                 }
 #pragma unroll
-                for (int c = 0; c < RW; ++c) {
-                    const int r = r0 + c;
-                    if (r >= p.rows_total) continue;  // padding rows are computed and dropped
-                    const float val = inv[c] > 0.f ? __uint_as_float(o[c]) * inv[c] : 0.f;
-                    // lane tl holds latent column 128 m + tl of every row: 128 consecutive values per row and block
-                    if (p.o_final != nullptr) p.o_final[(out_row0 + r) * 512 + m * 128 + tl] = __float2bfloat16(val);
-                    else p.o_part[(out_row0 + r) * 512 + m * 128 + tl] = val;
+                for (int m = 0; m < 4; ++m) {
+                    uint32_t o[8];
+                    if (nt > 0 && ok) {  // warp-uniform
+                        tmem_ld8(lane_base + kColO + m * R + r0 + cc, o);
+                        tmem_wait_ld();
+                    }
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const int r = r0 + cc + c;
+                        if (r >= p.rows_total) continue;  // padding rows are computed and dropped
+                        const float val = inv[c] > 0.f ? __uint_as_float(o[c]) * inv[c] : 0.f;
+                        // lane tl holds latent column 128 m + tl of every row: 128 consecutive values per row and block
+                        if (p.o_final != nullptr) p.o_final[(out_row0 + r) * 512 + m * 128 + tl] = __float2bfloat16(val);
+                        else p.o_part[(out_row0 + r) * 512 + m * 128 + tl] = val;
+                    }
                 }
             }
             named_bar_sync(1, kSmT);  // red is rewritten by the next piece

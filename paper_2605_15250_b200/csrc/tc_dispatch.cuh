@@ -24,7 +24,7 @@
 #endif
 // Likewise for the absorb path: largest (padded) h_q * s_q served by its tokens-on-M kernel by default.
 #ifndef GQLA_ABSORB_TOKENS_MAX_ROWS
-#define GQLA_ABSORB_TOKENS_MAX_ROWS 32
+#define GQLA_ABSORB_TOKENS_MAX_ROWS 64
 #endif
 
 namespace gqla {
@@ -88,14 +88,14 @@ inline int sm_count() {
 
 inline int absorb_resident_pairs();
 
-// Query rows of the absorb path's tokens-on-M kernel (tc_decode_absorb_t.cuh): h_q * s_q padded to 16 or 32.
+// Query rows of the absorb path's tokens-on-M kernel (tc_decode_absorb_t.cuh): h_q * s_q padded to 16, 32 or 64.
 inline int absorb_rows_t(const gqla_dims& d, int32_t s_q) {
     const int r = next_pow2(d.h_q * s_q);
     return r < 16 ? 16 : r;
 }
-// Which absorb kernel serves a shape: the tokens-on-M kernel up to 32 query rows (a quarter of the pair kernel's
-// tile), the pair kernel beyond.  GQLA_ABSORB_KERNEL=rows|tokens overrides the choice for the shapes both cover,
-// h_q * s_q <= 32 (read once per process; a tuning aid).
+// Which absorb kernel serves a shape: the tokens-on-M kernel up to 64 query rows (half the pair kernel's tile), the
+// pair kernel beyond.  GQLA_ABSORB_KERNEL=rows|tokens overrides the choice for the shapes both cover, h_q * s_q <= 64
+// (read once per process; a tuning aid).
 inline bool absorb_prefers_tokens(const gqla_dims& d, int32_t s_q) {
     static const int forced = []() {
         const char* e = getenv("GQLA_ABSORB_KERNEL");
@@ -103,9 +103,17 @@ inline bool absorb_prefers_tokens(const gqla_dims& d, int32_t s_q) {
         return e[0] == 't' ? 1 : (e[0] == 'r' ? 2 : 0);
     }();
     const int rows_t = absorb_rows_t(d, s_q);
-    if (rows_t > 32) return false;  // 16 rows per softmax thread spill: the pair kernel is faster there
+    if (rows_t > 64) return false;
     if (forced != 0) return forced == 1;
     return rows_t <= GQLA_ABSORB_TOKENS_MAX_ROWS;
+}
+
+// Workers of the balanced plan on the absorb path's CTA-pair kernels (bf16 and E4M3): pairs resident at once per
+// block of 128 query rows.
+inline int32_t pair_balanced_workers(const gqla_dims& d, int32_t s_q) {
+    const int row_blocks = (s_q * d.h_q + 127) / 128;
+    const int pairs = absorb_resident_pairs();
+    return pairs / row_blocks > 0 ? pairs / row_blocks : 0;
 }
 
 // Workers of the balanced plan: the GQA path runs one CTA per SM and keeps the cut points of all g
@@ -117,9 +125,7 @@ inline int32_t tc_balanced_workers(const gqla_dims& d, int32_t s_q, int32_t path
     if (sms <= 0) return 0;
     if (path == 1) return sms / d.g > 0 ? sms / d.g : 0;
     if (absorb_prefers_tokens(d, s_q)) return sms;  // one persistent CTA per SM
-    const int row_blocks = (s_q * d.h_q + 127) / 128;
-    const int pairs = absorb_resident_pairs();
-    return pairs / row_blocks > 0 ? pairs / row_blocks : 0;
+    return pair_balanced_workers(d, s_q);
 }
 
 inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t N, const void* cache,
@@ -374,8 +380,9 @@ inline gqla_status tc_decode_absorb(const gqla_dims& d, int32_t B, int32_t s_q, 
     if (o_final != nullptr && (balanced || S != 1)) return GQLA_ERR_UNSUPPORTED;
     if (tokens_on_m) {
         const unsigned grid = (unsigned)(balanced ? workers : B * S);  // single CTAs: W of them, or one per piece
-        const cudaError_t e = rows_t == 16 ? absorb_t_launch<16>(p, tmQ, tmC, grid, st)
-                                           : absorb_t_launch<32>(p, tmQ, tmC, grid, st);
+        const cudaError_t e = rows_t == 16   ? absorb_t_launch<16>(p, tmQ, tmC, grid, st)
+                              : rows_t == 32 ? absorb_t_launch<32>(p, tmQ, tmC, grid, st)
+                                             : absorb_t_launch<64>(p, tmQ, tmC, grid, st);
         return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
     }
     auto kern = tc::decode_absorb_tc_kernel<0>;
@@ -547,7 +554,7 @@ inline gqla_status tc_decode_absorb_fp8(const gqla_dims& d, int32_t B, int32_t s
         return GQLA_ERR_UNSUPPORTED;
     const int rows_total = s_q * d.h_q;
     const int row_blocks = (rows_total + 127) / 128;
-    const int32_t workers = S < 0 ? tc_balanced_workers(d, s_q, 0) : 0;
+    const int32_t workers = S < 0 ? pair_balanced_workers(d, s_q) : 0;
     const bool balanced = S < 0 && workers > 0;
     if (S < 0) S = -S;
     const int64_t pairs = balanced ? (int64_t)workers * row_blocks : (int64_t)B * S * row_blocks;

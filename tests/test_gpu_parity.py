@@ -583,8 +583,8 @@ def test_both_gqa_kernels_on_the_shapes_both_cover(kernel):
 
 @pytest.mark.parametrize("kernel", ["rows", "tokens"])
 def test_both_absorb_kernels_on_the_shapes_both_cover(kernel):
-    """Two tensor-core kernels serve the absorb path: tokens on the MMA's M axis for h_q * s_q <= 32 (every cache tile
-    fetched once and used as K and as V; the default there) and the CTA-pair kernel with the query rows on M.
+    """Two tensor-core kernels serve the absorb path: tokens on the MMA's M axis for h_q * s_q <= 64 (every cache tile
+    fetched once and used as K and as V) and the CTA-pair kernel with the query rows on M.
     GQLA_ABSORB_KERNEL forces either one where both apply; the choice is read once per process, so each runs the
     ragged parity cases (fixed, balanced and whole-sequence plans) in a process of its own."""
     import os
@@ -598,7 +598,8 @@ def test_both_absorb_kernels_on_the_shapes_both_cover(kernel):
         "sl = np.array([700, 0, 129, 2050, 64, 1, 63, 65], dtype=np.int32)\n"
         "for dims, s_q in ((dict(h_q=32, g=8, d_h=128, r_kv=512, d_r=64), 1), (dict(h_q=16, g=8, d_h=128, r_kv=512, d_r=64), 2),\n"
         "                  (dict(h_q=28, g=4, d_h=128, r_kv=512, d_r=64), 1), (dict(h_q=8, g=8, d_h=128, r_kv=512, d_r=64), 2),\n"
-        "                  (dict(h_q=8, g=4, d_h=128, r_kv=512, d_r=64), 3)):\n"
+        "                  (dict(h_q=8, g=4, d_h=128, r_kv=512, d_r=64), 3), (dict(h_q=32, g=8, d_h=128, r_kv=512, d_r=64), 2),\n"
+        "                  (dict(h_q=20, g=4, d_h=128, r_kv=512, d_r=64), 3)):\n"
         "    w = synth.Workload('k', batch=8, s_q=s_q, dtype='bf16', seed=9, **dims)\n"
         "    d = B.make_dims(w.h_q, w.g, w.d_h, w.r_kv, w.d_r)\n"
         "    sms = torch.cuda.get_device_properties(0).multi_processor_count\n"
