@@ -22,10 +22,10 @@
 // Shared memory holds two tiles and one of them is always held by the softmax (a tile fetched once has to stay from its
 // first product until its second), so the producer also asks a later tile into L2 when it issues a load, and the held time
 // is kept short: the issuer polls instead of blocking, the softmax uses every lane.  Measured (h_q = 32, s_q = 1, 128
-// sequences of 8-32 K tokens, balanced plan, one GPU): 477 us in a burst against 523-539 us for the pair kernel; launched
-// back to back for seconds under the power cap, a quarter of the tensor work leaves the clocks at 1.79 GHz where the pair
-// kernel's drop to 1.26 GHz: 524 us against 620 us per launch.  With 64 rows (sixteen per softmax warp, one P^T buffer):
-// 566 against 582 us in a burst.
+// sequences of 8-32 K tokens, balanced plan, one GPU): 437 us in a burst against 541 us for the pair kernel; launched
+// back to back for seconds under the power cap, a quarter of the tensor work leaves the clocks at 1.70 GHz where the pair
+// kernel's drop to 1.21 GHz: 505 us against 633 us per launch.  With 64 rows (sixteen per softmax warp, one P^T buffer):
+// 502 against 554 us in a burst.
 #pragma once
 #include "common.cuh"
 #include "sched.cuh"

@@ -220,12 +220,14 @@ decode_gqa_t_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ, 
                 tc_fence_after();
                 const uint32_t st = smem_u32(stage0 + s * L::kStageBytes);
                 const uint32_t d = tmem_base + kColS + (uint32_t)s * R;
+                // descriptors stepped through their low words (the high words are constants): fewer instructions per MMA
+                const uint32_t k_lo = desc_lo(desc_kmajor_sw128(st)), q_lo = desc_lo(desc_kmajor_sw128(q_addr));
 #pragma unroll
                 for (int kb = 0; kb < 3; ++kb)
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        umma_ss(d, desc_kmajor_sw128(st + kb * 16384 + ks * 32),
-                                desc_kmajor_sw128(q_addr + kb * L::kQBlock + ks * 32), idesc_qk, (kb | ks) != 0);
+                        umma_ss_lo(d, k_lo + ((kb * 16384 + ks * 32) >> 4), kDescHiSw128, q_lo + ((kb * L::kQBlock + ks * 32) >> 4),
+                                   kDescHiSw128, idesc_qk, (uint32_t)(kb | ks));
                 umma_commit(&s_full[s]);
                 umma_commit(&kempty[s]);
                 return true;
@@ -251,10 +253,11 @@ decode_gqa_t_kernel(const GqaParams p, const __grid_constant__ CUtensorMap tmQ, 
                     tc_fence_after();
                     const uint32_t v_addr = smem_u32(stage0 + s * L::kStageBytes + L::kKcBytes + L::kKrBytes);
                     const uint32_t pb = p_addr0 + s * L::kPBuf;
+                    const uint64_t vd = desc_mnmajor_sw128(v_addr, 16384), pd = desc_mnmajor_rows(pb, L::kPRow);
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)  // 16 tokens per step: rows [16 ks, +16) of the V boxes and of P^T
-                        umma_ss(tmem_base + kColO, desc_mnmajor_sw128(v_addr + ks * 2048, 16384),
-                                desc_mnmajor_rows(pb + ks * 16 * L::kPRow, L::kPRow), idesc_pv, (t | ks) != 0);
+                        umma_ss_lo(tmem_base + kColO, (uint32_t)vd + ((ks * 2048) >> 4), (uint32_t)(vd >> 32),
+                                   (uint32_t)pd + ((ks * 16 * L::kPRow) >> 4), (uint32_t)(pd >> 32), idesc_pv, (uint32_t)(t | ks));
                     umma_commit(&vempty[s]);
                     umma_commit(&pv_done[s]);
                 }
