@@ -574,7 +574,7 @@ def run_ours(args):
             "clocks": clocks, "e2e": e2e, "gpu_launches": 3 * steps, "roofline": roof, "cpu_baseline": cpu,
             # the two targets as their statement defines them: fractions of the NOMINAL roofline
             # min(2.25 PFLOP/s, bytes / 8 TB/s), not of the peaks measured on this GPU
-            "north_star": {"absorb_frac_of_nominal_roofline": roof["frac_of_nominal_roofline"], "absorb_target": 0.60,
+            "targets": {"absorb_frac_of_nominal_roofline": roof["frac_of_nominal_roofline"], "absorb_target": 0.60,
                            "gqa_frac_of_8tbs": g_gbs / 8000.0, "gqa_target": 0.75},
             "paths": paths,
         }

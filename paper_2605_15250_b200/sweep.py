@@ -186,7 +186,7 @@ def run(names, steps: int, warmup: int, paths=("absorb", "gqa")):
 
 
 def markdown(path: str) -> None:
-    """Prints the JSON lines of an earlier run as the table the benchmark spec carries."""
+    """Prints the JSON lines of an earlier run as a markdown table."""
     print("| config | path | s_q | split plan | pieces/seq | decode kernel µs | path µs | tokens/s (path) | GB/s | TFLOP/s | "
           "of measured roofline | of nominal roofline |")
     print("|---|---|---|---|---|---|---|---|---|---|---|---|")
