@@ -626,10 +626,11 @@ def test_debug_build_index_checks_stay_silent():
         "from paper_2605_15250_b200 import binding as B, synth\n"
         "from tests.parity_util import end_to_end\n"
         "assert B.LIB_PATH.endswith('libgqla_debug.so')\n"
-        "w = synth.Workload('dbg', 128, 8, 128, 512, 64, batch=5, s_q=2, dtype='bf16', seed=5)\n"
         "sl = np.array([700, 0, 129, 2050, 64], dtype=np.int32)\n"
-        "for S in (1, 3, -3):\n"
-        "    end_to_end(w, sl, S, q_gain=4.0)\n"
+        "for h_q in (128, 32):  # query rows on the MMA's M axis / tokens on M, on both paths\n"
+        "    w = synth.Workload('dbg', h_q, 8, 128, 512, 64, batch=5, s_q=2, dtype='bf16', seed=5)\n"
+        "    for S in (1, 3, -3):\n"
+        "        end_to_end(w, sl, S, q_gain=4.0)\n"
         "print('debug-ok')\n")
     env = dict(os.environ, GQLA_LIB_PATH=lib, PYTHONPATH=root)
     res = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, env=env, cwd=root, timeout=600)
