@@ -4,7 +4,7 @@
 //   up_proj      :  o[row, d]         = sum_r o_hat[row, r] W_UV[j][r][d] (Eq. (mqa), line 6)
 // One CTA computes a 128 x BN output tile: warp 0 streams A/B tiles with TMA through a ring of
 // shared-memory stages, warp 1 issues tcgen05.mma into a TMEM accumulator, warps 2-5 read the
-// accumulator back (tcgen05.ld) and store bf16 rows.
+// accumulator back (tcgen05.ld), stage their bf16 rows in the idle stage ring and ship each row as one bulk store.
 #pragma once
 #include "tc_common.cuh"
 
@@ -28,10 +28,12 @@ struct GemmParams {
 
 template <int BN, bool B_MN>
 struct GemmSmem {
-    static constexpr int kStages = 4;
+    static constexpr int kStages = BN <= 128 ? 6 : 4;  // 32 KB or 48 KB per stage: 192 KB of tiles in flight
     static constexpr int kABytes = 128 * 128;  // 128 rows x 64 bf16
     static constexpr int kBBytes = BN * 128;   // K-major: BN rows x 64 k;  MN-major: (BN/64) boxes of 64 k-rows x 64 n
     static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kOutPitch = BN * 2 + 16;  // output staging of the epilogue (reuses the stage ring)
+    static_assert(128 * kOutPitch <= kStages * kStageBytes, "output staging must fit in the stage ring");
     static constexpr int kTotal = kStages * kStageBytes + 1024 /*align slack*/ + 256 /*barriers*/;
     static_assert(OneCtaPerSM<kTotal>::value, "");
 };
@@ -169,8 +171,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
         // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32)
         const int q = warp & 3;
         const int row = q * 32 + lane;  // row of the tile == TMEM lane
-        const bool ok = mbar_wait(acc_full, 0, ab, 3);
-        tc_fence_after();
+        // (output addresses and the side copies first: they overlap the main loop instead of following it)
         __nv_bfloat16* dst = nullptr;
         if (MODE == kGemmExpand) {
             const int64_t n = (int64_t)m_tile * 128 + row;
@@ -204,24 +205,37 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
                 }
             }
         }
+        const bool ok = mbar_wait(acc_full, 0, ab, 3);
+        tc_fence_after();
         if (ok) {
+            // The thread's output row leaves through shared memory as ONE bulk store (BN * 2 contiguous bytes): 16-byte
+            // stores of 32 threads to 32 different rows made the epilogue the longest part of these kernels.  The
+            // stage ring is idle here (the accumulator is complete, so every load has landed and been multiplied);
+            // the padded pitch keeps the 16-byte stores of a quarter warp on distinct banks.  A thread stages and
+            // ships only its own row, so no barrier is needed in between.
+            uint8_t* srow = tiles + row * L::kOutPitch;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t v[32];
+            for (int c0 = 0; c0 < BN; c0 += 64) {  // two loads in flight per wait
+                uint32_t v[64];
                 tmem_ld32(tmem_addr(tmem_base, q * 32, c0), v);
+                tmem_ld32(tmem_addr(tmem_base, q * 32, c0 + 32), v + 32);
                 tmem_wait_ld();
-                if (dst != nullptr) {
-                    uint4* d4 = reinterpret_cast<uint4*>(dst + c0);
+                uint4* d4 = reinterpret_cast<uint4*>(srow + c0 * 2);
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(v[8 * t + 0]), __uint_as_float(v[8 * t + 1]));
-                        o.y = pack_bf16(__uint_as_float(v[8 * t + 2]), __uint_as_float(v[8 * t + 3]));
-                        o.z = pack_bf16(__uint_as_float(v[8 * t + 4]), __uint_as_float(v[8 * t + 5]));
-                        o.w = pack_bf16(__uint_as_float(v[8 * t + 6]), __uint_as_float(v[8 * t + 7]));
-                        d4[t] = o;
-                    }
+                for (int t = 0; t < 8; ++t) {
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(v[8 * t + 0]), __uint_as_float(v[8 * t + 1]));
+                    o.y = pack_bf16(__uint_as_float(v[8 * t + 2]), __uint_as_float(v[8 * t + 3]));
+                    o.z = pack_bf16(__uint_as_float(v[8 * t + 4]), __uint_as_float(v[8 * t + 5]));
+                    o.w = pack_bf16(__uint_as_float(v[8 * t + 6]), __uint_as_float(v[8 * t + 7]));
+                    d4[t] = o;
                 }
+            }
+            fence_proxy_async_smem();  // staged row -> visible to the bulk-copy engine
+            if (dst != nullptr) {
+                bulk_store(dst, srow, BN * 2);
+                bulk_commit();
+                bulk_wait_read();  // shared memory must outlive the copy's reads
             }
         }
     }
