@@ -165,7 +165,9 @@ __device__ __forceinline__ float4 ld_stream4(const float* p) {  // read once: do
                  : "l"(p));
     return v;
 }
-template <typename TO>
+// V = 4 or 8 output columns per thread (8 where d_out allows: half the threads, i.e. one wave of them on the shapes
+// of the decode chains, and 16-byte stores of bf16).
+template <typename TO, int V>
 __global__ void __launch_bounds__(256) combine_vec_kernel(int64_t rows, int32_t rows_per_seq, int32_t S, int32_t d_out,
                                                           const float* __restrict__ o_part,
                                                           const float* __restrict__ lse_part, TO* __restrict__ out,
@@ -173,11 +175,11 @@ __global__ void __launch_bounds__(256) combine_vec_kernel(int64_t rows, int32_t 
     // (dependent-launch instructions; no-ops when the kernel is launched the ordinary way)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int32_t vec_per_row = d_out >> 2;
+    const int32_t vec_per_row = d_out / V;
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t r = idx / vec_per_row;
     if (r >= rows) return;
-    const int c = (int)(idx % vec_per_row) << 2;
+    const int c = (int)(idx % vec_per_row) * V;
     const int64_t b = r / rows_per_seq;
     const int rr = (int)(r % rows_per_seq);
     const float* lp = lse_part + b * S * rows_per_seq + rr;
@@ -186,20 +188,41 @@ __global__ void __launch_bounds__(256) combine_vec_kernel(int64_t rows, int32_t 
     const bool dead = !(mx > -INFINITY);
     const float* op = o_part + (b * S * rows_per_seq + rr) * d_out + c;
     const int64_t kstride = (int64_t)rows_per_seq * d_out;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 acc[V / 4];
+#pragma unroll
+    for (int u = 0; u < V / 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
     float den = 0.f;
     for (int k = 0; k < S; ++k) {
         const float wk = dead ? 0.f : expf(__ldg(lp + (int64_t)k * rows_per_seq) - mx);
         den += wk;
         if (wk == 0.f) continue;  // an empty split's partial is never read
-        const float4 x = ld_stream4(op + k * kstride);
-        acc.x = fmaf(wk, x.x, acc.x);
-        acc.y = fmaf(wk, x.y, acc.y);
-        acc.z = fmaf(wk, x.z, acc.z);
-        acc.w = fmaf(wk, x.w, acc.w);
+#pragma unroll
+        for (int u = 0; u < V / 4; ++u) {
+            const float4 x = ld_stream4(op + k * kstride + 4 * u);
+            acc[u].x = fmaf(wk, x.x, acc[u].x);
+            acc[u].y = fmaf(wk, x.y, acc[u].y);
+            acc[u].z = fmaf(wk, x.z, acc[u].z);
+            acc[u].w = fmaf(wk, x.w, acc[u].w);
+        }
     }
     const float inv = den > 0.f ? 1.f / den : 0.f;
-    store4(out + r * d_out + c, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
+#pragma unroll
+    for (int u = 0; u < V / 4; ++u) {
+        acc[u].x *= inv; acc[u].y *= inv; acc[u].z *= inv; acc[u].w *= inv;
+    }
+    if constexpr (V == 8 && sizeof(TO) == 2) {  // eight bf16: one 16-byte store
+        __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[0].x, acc[0].y), h1 = __floats2bfloat162_rn(acc[0].z, acc[0].w);
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[1].x, acc[1].y), h3 = __floats2bfloat162_rn(acc[1].z, acc[1].w);
+        uint4 u4;
+        u4.x = *reinterpret_cast<uint32_t*>(&h0);
+        u4.y = *reinterpret_cast<uint32_t*>(&h1);
+        u4.z = *reinterpret_cast<uint32_t*>(&h2);
+        u4.w = *reinterpret_cast<uint32_t*>(&h3);
+        *reinterpret_cast<uint4*>(out + r * d_out + c) = u4;
+    } else {
+#pragma unroll
+        for (int u = 0; u < V / 4; ++u) store4(out + r * d_out + c + 4 * u, acc[u]);
+    }
     if (lse != nullptr && c == 0) lse[r] = dead ? -INFINITY : mx + logf(den);
 }
 
