@@ -9,14 +9,21 @@
 //     this CTA's 128 of every 256 latent columns) is two boxes.  A tile is 36 KB of K and 32 KB of V per CTA
 //     instead of 72 + 64, so both rings are two tiles deep in less shared memory than the bf16 kernel needs for one.
 //   * Scores are scaled per query row (q_scale, which folds the cache planes' scales in), outputs by v_scale.
-//   * P is rounded to E4M3; the softmax reference is held kAF8Bias binades below the running maximum and follows
-//     it as soon as it has grown by more than one binade, so that P <= 2^8 and terms down to 2^-16 of the largest
-//     one still count (the format's smallest positive value is 2^-9).
+//   * P is rounded to E4M3 (smallest positive value 2^-9, largest 448): a row's softmax reference is put kAF8Bias = 5
+//     binades below the row maximum that raised it and is raised again when a score exceeds it by more than 8.75, so
+//     that P <= 430 and terms down to 2^-14 of the largest one count right after a raise (2^-17.75 before the next).
+//   * With half the bytes and half the MMA time per tile the softmax warps set the pace, so their per-tile chain is
+//     kept short: whether any score of the CTA outgrew its row's reference is ONE barrier.red (the row maxima, whose
+//     four parts live in four warps, are exchanged through shared memory only when it says yes -- raises are rare by
+//     the choice of the two constants above), and barriers that have usually completed are probed before a suspending
+//     wait.  The exchange of every tile's maxima and a reference that followed the maximum within one binade (O
+//     rescaled on 40 % of the tiles) cost a quarter of the kernel.
 #pragma once
 #include "common.cuh"
 #include "sched.cuh"
 #include "tc_common.cuh"
 #include "tc_decode_gqa_fp8.cuh"  // E4M3 descriptors, packing
+#include "tc_decode_gqa_t.cuh"    // bar_or
 
 namespace gqla {
 namespace tc {
@@ -67,8 +74,8 @@ struct AbsorbFp8Smem {
 
 constexpr uint32_t kA8ColO = 0;    // O: MMA m (latent columns [256m, 256m+256)) at TMEM columns [128m, 128m+128)
 constexpr uint32_t kA8ColS = 256;  // two 64-column score buffers
-constexpr float kAF8Bias = 7.0f;     // log2 units the softmax reference sits below the running maximum
-constexpr float kAF8Refresh = 1.0f;  // the reference follows the maximum once it has grown by this much
+constexpr float kAF8Bias = 5.0f;   // log2 units a raised softmax reference sits below the row maximum that raised it
+constexpr float kAF8Grow = 8.75f;  // a score this far above its row's reference raises it (2^8.75 = 430 < 448)
 constexpr uint32_t kDescHiSw64 = (uint32_t)(((1ull << 46) | (4ull << 61) | ((uint64_t)(512 >> 4) << 32)) >> 32);
 // cta_group::2 MMA of kind::f8f6f4; descriptors as (low word, constant high word of their swizzle mode).
 template <bool ACCUMULATE>
@@ -105,7 +112,7 @@ decode_absorb_fp8_tc_kernel(const AbsorbFp8Params p, const __grid_constant__ CUt
     uint64_t* s_full = epi_done + 1;   // [2]
     uint64_t* p_ready = s_full + 2;    // [2] leader only: one arrival per softmax warp of the pair
     uint64_t* pv_done = p_ready + 2;   // [2]
-    uint64_t* xch = pv_done + 2;       // [2] softmax warps of this CTA: per-tile max exchange
+    uint64_t* xch = pv_done + 2;       // [2] (not used by this kernel: the maxima are exchanged behind a named barrier)
     uint64_t* fin = xch + 2;           //     the final partial-sum exchange of a piece
     uint64_t* epi = fin + 1;           //     and the steps of the output staging
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + L::kNumBars);
@@ -355,6 +362,9 @@ decode_absorb_fp8_tc_kernel(const AbsorbFp8Params p, const __grid_constant__ CUt
             if (!row_valid) lim = 0;
             // the row's score scale: softmax scale x log2(e) x the query row's quantisation scale
             const float sl2 = p.scale_log2 * (row_valid ? p.q_scale[(int64_t)pc.b * p.rows_total + rho] : 1.f);
+            // m_used: the row's softmax REFERENCE (log2 units), the same in the four threads of the row.  P = 2^(x - m_used)
+            // is rounded to E4M3 (smallest positive value 2^-9, largest 448): a raise puts the reference kAF8Bias binades
+            // below the row's maximum so far, and the next raise comes when a score exceeds it by more than kAF8Grow.
             float m_used = -INFINITY, l = 0.f;
             bool ok = true;
 
@@ -362,58 +372,78 @@ decode_absorb_fp8_tc_kernel(const AbsorbFp8Params p, const __grid_constant__ CUt
                 const int n = gt + t;
                 const int sb = n & 1;
                 const uint32_t nph = (n >> 1) & 1;
-                ok = __all_sync(0xffffffffu, mbar_wait(&s_full[sb], nph, ab, 7));
-                if (!ok) break;
+                // a failed wait raises the CTA's abort flag; the warps agree on leaving at the barrier below
+                bool okl = __all_sync(0xffffffffu, mbar_wait_fast(&s_full[sb], nph, ab, 7));
                 tc_fence_after();
                 const int tok0 = t * 128 + hf * 64 + ch * 32;
                 uint32_t x[32];
-                tmem_ld32(lane_base + kA8ColS + (uint32_t)sb * 64 + ch * 32, x);
-                tmem_wait_ld();
+                if (okl) {
+                    tmem_ld32(lane_base + kA8ColS + (uint32_t)sb * 64 + ch * 32, x);
+                    tmem_wait_ld();
+                }
                 const bool full = tok0 + 32 <= lim;  // every score of this thread is visible
                 float mx = -INFINITY;
+                if (okl) {
+                    if (full) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(x[c]));
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (tok0 + c < lim) mx = fmaxf(mx, __uint_as_float(x[c]));
+                    }
+                }
+                // Does any score of the CTA outgrow its row's reference?  One barrier.red instead of an exchange of the
+                // row maxima (the other three parts of a row live in other warps); only then are the maxima exchanged.
+                const float m_t = mx * sl2;
+                float factor = 1.f;
+                bool need = false;
+                if (bar_or(m_t > m_used + kAF8Grow || !okl, L::kSoftmaxWarps * 32)) {
+                    if (ab.raised()) { ok = false; break; }  // same answer in every thread: the flag was set before the barrier
+                    float* mxs = sm_max;
+                    mxs[part * 64 + r] = m_t;
+                    named_bar_sync(1, L::kSoftmaxWarps * 32);
+                    const float row_max = fmaxf(fmaxf(mxs[r], mxs[64 + r]), fmaxf(mxs[128 + r], mxs[192 + r]));
+                    const float m_new = fmaxf(m_used, row_max - kAF8Bias);
+                    need = m_new > m_used;
+                    factor = need ? ex2(m_used - m_new) : 1.f;  // ex2(-inf) = 0 on first use
+                    if (need) {
+                        l *= factor;
+                        m_used = m_new;
+                    }
+                    named_bar_sync(1, L::kSoftmaxWarps * 32);  // the maxima may be rewritten by the next raise
+                }
+                const float m_sub = m_used == -INFINITY ? 0.f : m_used;
+                uint32_t pk[8];
                 if (full) {
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(x[c]));
+                    for (int c = 0; c < 32; c += 4) {
+                        float e[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            e[i] = ex2(fmaf(__uint_as_float(x[c + i]), sl2, -m_sub));
+                            l += e[i];
+                        }
+                        pk[c / 4] = pack_e4m3x4(e[0], e[1], e[2], e[3]);
+                    }
                 } else {
 #pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (tok0 + c < lim) mx = fmaxf(mx, __uint_as_float(x[c]));
-                }
-                // the other three parts of this row live in other warps
-                float* mxs = sm_max + sb * 256;
-                mxs[part * 64 + r] = mx;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&xch[sb]);
-                ok = __all_sync(0xffffffffu, mbar_wait(&xch[sb], nph, ab, 10));
-                if (!ok) break;
-                mx = fmaxf(fmaxf(mxs[r], mxs[64 + r]), fmaxf(mxs[128 + r], mxs[192 + r]));
-                const float m_t = mx * sl2;
-                const bool need = m_t > m_used + kAF8Refresh;
-                const float factor = need ? ex2(m_used - m_t) : 1.f;
-                if (need) {
-                    l *= factor;
-                    m_used = m_t;
-                }
-                // exponent offset: the reference sits kAF8Bias binades below the (lazily tracked) maximum
-                const float m_sub = m_used == -INFINITY ? 0.f : m_used - kAF8Bias;
-                uint32_t pk[8];
+                    for (int c = 0; c < 32; c += 4) {
+                        float e[4];
 #pragma unroll
-                for (int c = 0; c < 32; c += 4) {
-                    float e[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        e[i] = (full || tok0 + c + i < lim) ? ex2(fmaf(__uint_as_float(x[c + i]), sl2, -m_sub)) : 0.f;
-                        l += e[i];
+                        for (int i = 0; i < 4; ++i) {
+                            e[i] = (okl && tok0 + c + i < lim) ? ex2(fmaf(__uint_as_float(x[c + i]), sl2, -m_sub)) : 0.f;
+                            l += e[i];
+                        }
+                        pk[c / 4] = pack_e4m3x4(e[0], e[1], e[2], e[3]);
                     }
-                    pk[c / 4] = pack_e4m3x4(e[0], e[1], e[2], e[3]);
                 }
                 // O may be rescaled, and the P buffer rewritten, only once P.V(n-1) has completed
-                if (t > 0) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, ab, 8));
-                    if (!ok) break;
+                if (t > 0 && okl) {
+                    okl = __all_sync(0xffffffffu, mbar_wait_fast(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, ab, 8));
                     tc_fence_after();
                 }
-                if (__any_sync(0xffffffffu, need) && t > 0) {
+                if (__any_sync(0xffffffffu, need) && t > 0 && okl) {
                     // this thread's share of the lane's O: columns [128m + 64ch, +64) for m = 0, 1
 #pragma unroll 1
                     for (int c = 0; c < 4; ++c) {
@@ -437,7 +467,7 @@ decode_absorb_fp8_tc_kernel(const AbsorbFp8Params p, const __grid_constant__ CUt
                 fence_proxy_async_smem();  // generic-proxy writes of P -> visible to the tensor core
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(p_ready_l[sb]);
+                if (lane == 0 && okl) mbar_arrive_cluster(p_ready_l[sb]);  // withheld after a failed wait: the next vote ends the loop
             }
 
             // -------------------------------------------------------------- epilogue: normalise and store
@@ -541,7 +571,7 @@ decode_absorb_fp8_tc_kernel(const AbsorbFp8Params p, const __grid_constant__ CUt
             if (!__all_sync(0xffffffffu, mbar_wait(epi_done, pi & 1, ab, 12))) ok = false;
             if (row_valid && part == 0 && p.lse_part != nullptr)
                 p.lse_part[(slot0 + pc.k) * p.rows_total + rho] =
-                    live ? (m_used - kAF8Bias + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
+                    live ? (m_used + log2f(Lt)) * 0.6931471805599453f : -INFINITY;
             gt += pc.n_tiles;
             ++pi;
         }
