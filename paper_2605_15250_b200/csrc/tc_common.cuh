@@ -257,6 +257,16 @@ __device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t* r) {
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
+// OR of a predicate over the `nthreads` threads that call it (named barrier 1).
+__device__ __forceinline__ bool bar_or(bool v, int nthreads) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\tbarrier.cta.red.or.pred q, 1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)v), "r"(nthreads)
+        : "memory");
+    return r != 0;
+}
 
 // ----------------------------------------------------------------------------- UMMA descriptors
 // Shared-memory matrix descriptor (64-bit):

@@ -9,9 +9,9 @@
 //     this CTA's 128 of every 256 latent columns) is two boxes.  A tile is 36 KB of K and 32 KB of V per CTA
 //     instead of 72 + 64, so both rings are two tiles deep in less shared memory than the bf16 kernel needs for one.
 //   * Scores are scaled per query row (q_scale, which folds the cache planes' scales in), outputs by v_scale.
-//   * P is rounded to E4M3 (smallest positive value 2^-9, largest 448): a row's softmax reference is put kAF8Bias = 5
+//   * P is rounded to E4M3 (smallest positive value 2^-9, largest 448): a row's softmax reference is put kAF8Bias = 6
 //     binades below the row maximum that raised it and is raised again when a score exceeds it by more than 8.75, so
-//     that P <= 430 and terms down to 2^-14 of the largest one count right after a raise (2^-17.75 before the next).
+//     that P <= 430 and terms down to 2^-15 of the largest one count right after a raise (2^-17.75 before the next).
 //   * With half the bytes and half the MMA time per tile the softmax warps set the pace, so their per-tile chain is
 //     kept short: whether any score of the CTA outgrew its row's reference is ONE barrier.red (the row maxima, whose
 //     four parts live in four warps, are exchanged through shared memory only when it says yes -- raises are rare by
@@ -23,7 +23,6 @@
 #include "sched.cuh"
 #include "tc_common.cuh"
 #include "tc_decode_gqa_fp8.cuh"  // E4M3 descriptors, packing
-#include "tc_decode_gqa_t.cuh"    // bar_or
 
 namespace gqla {
 namespace tc {
@@ -74,7 +73,7 @@ struct AbsorbFp8Smem {
 
 constexpr uint32_t kA8ColO = 0;    // O: MMA m (latent columns [256m, 256m+256)) at TMEM columns [128m, 128m+128)
 constexpr uint32_t kA8ColS = 256;  // two 64-column score buffers
-constexpr float kAF8Bias = 5.0f;   // log2 units a raised softmax reference sits below the row maximum that raised it
+constexpr float kAF8Bias = 6.0f;   // log2 units a raised softmax reference sits below the row maximum that raised it
 constexpr float kAF8Grow = 8.75f;  // a score this far above its row's reference raises it (2^8.75 = 430 < 448)
 constexpr uint32_t kDescHiSw64 = (uint32_t)(((1ull << 46) | (4ull << 61) | ((uint64_t)(512 >> 4) << 32)) >> 32);
 // cta_group::2 MMA of kind::f8f6f4; descriptors as (low word, constant high word of their swizzle mode).

@@ -11,9 +11,11 @@
 //     half as large.  The 64-byte rows of the k_R and q^R tiles use the 64-byte swizzle, everything else the
 //     128-byte one.
 //   * Scores are scaled per query row (q_scale folds the key planes' scales in), outputs by v_scale.
-//   * P is rounded to E4M3 (4 significant bits).  Its smallest positive value is 2^-9, so the softmax reference is
-//     held kBias = 7 binades BELOW the running maximum and refreshed as soon as the maximum grows by more than
-//     one binade: P <= 2^8 (the format ends at 448) and terms down to 2^-16 of the largest one still count.
+//   * P is rounded to E4M3 (4 significant bits; smallest positive value 2^-9, largest 448).  A replica's softmax
+//     reference is put kF8Bias = 6 binades BELOW the tile maximum that raised it and raised again when a tile's
+//     maximum exceeds it by more than 8.75: P <= 430, and terms down to 2^-15 of the largest one count right after a
+//     raise (2^-17.75 before the next).  A raise rescales O and has to wait for the previous tile's P.V, so it is
+//     kept rare; following the maximum within one binade rescaled on a large share of the tiles.
 #pragma once
 #include "common.cuh"
 #include "sched.cuh"
@@ -59,8 +61,8 @@ struct GqaFp8Smem {
 constexpr uint32_t kF8ColS = 0;    // two 128-column score buffers
 constexpr uint32_t kF8ColP = 256;  // two 32-column E4M3 probability buffers (four per 32-bit column)
 constexpr uint32_t kF8ColO = 384;  // 128-column output accumulator
-constexpr float kF8Bias = 7.0f;    // log2 units the reference sits below the running maximum
-constexpr float kF8Refresh = 1.0f; // the reference follows the maximum once it has grown by this much
+constexpr float kF8Bias = 6.0f;    // log2 units a raised softmax reference sits below the maximum that raised it
+constexpr float kF8Grow = 8.75f;   // a score this far above its reference raises it (2^8.75 = 430 < 448)
 
 // K-major operand tile with 64-byte swizzle: rows of 64 bytes, 8-row groups 512 B apart.
 __device__ __forceinline__ uint64_t desc_kmajor_sw64(uint32_t smem_addr) {
@@ -310,7 +312,7 @@ decode_gqa_fp8_tc_kernel(const GqaFp8Params p, const __grid_constant__ CUtensorM
             for (int t = 0; t < pc.n_tiles && ok; ++t) {
                 const int n = gt + t;
                 const int sb = n & 1;
-                ok = __all_sync(0xffffffffu, mbar_wait(&s_full[sb], (n >> 1) & 1, ab, 7));
+                ok = __all_sync(0xffffffffu, mbar_wait_fast(&s_full[sb], (n >> 1) & 1, ab, 7));
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t s_addr = lane_base + kF8ColS + (uint32_t)sb * 128 + col0;
@@ -325,11 +327,14 @@ decode_gqa_fp8_tc_kernel(const GqaFp8Params p, const __grid_constant__ CUtensorM
                     for (int c = 0; c < CH; ++c)
                         if (owns(c) && tok0 + ch * CH + c < lim) mx = fmaxf(mx, __uint_as_float(x[c]));
                 }
+                // m_used is the replica's softmax REFERENCE: raised to kF8Bias below the tile maximum that exceeded it by
+                // more than kF8Grow (a raise rescales O and has to wait for the previous tile's P.V: it is made rare)
                 const float m_t = mx * sl2;
-                const bool need = m_t > m_used + kF8Refresh;
-                const float factor = need ? ex2(m_used - m_t) : 1.f;
+                const bool need = m_t > m_used + kF8Grow;
+                const float m_new = m_t - kF8Bias;
+                const float factor = need ? ex2(m_used - m_new) : 1.f;
                 if (__any_sync(0xffffffffu, need) && t > 0) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, ab, 8));
+                    ok = __all_sync(0xffffffffu, mbar_wait_fast(&pv_done[(n - 1) & 1], ((n - 1) >> 1) & 1, ab, 8));
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll 1
@@ -345,10 +350,9 @@ decode_gqa_fp8_tc_kernel(const GqaFp8Params p, const __grid_constant__ CUtensorM
                 }
                 if (need) {
                     l *= factor;
-                    m_used = m_t;
+                    m_used = m_new;
                 }
-                // exponent offset: the reference sits kF8Bias binades below the (lazily tracked) maximum
-                const float m_sub = m_used == -INFINITY ? 0.f : m_used - kF8Bias;
+                const float m_sub = m_used == -INFINITY ? 0.f : m_used;
                 const uint32_t p_addr = lane_base + kF8ColP + (uint32_t)sb * 32 + col0 / 4;
 #pragma unroll
                 for (int ch = 0; ch < NCH; ++ch) {
@@ -382,7 +386,7 @@ decode_gqa_fp8_tc_kernel(const GqaFp8Params p, const __grid_constant__ CUtensorM
             if (pc.n_tiles > 0 && ok)
                 ok = __all_sync(0xffffffffu, mbar_wait(&pv_done[n_last & 1], (n_last >> 1) & 1, ab, 9));
             tc_fence_after();
-            const float m_eff = m_used - kF8Bias;  // -inf stays -inf
+            const float m_eff = m_used;  // the reference the replica's sums are relative to (-inf: nothing seen)
             merge[Lr * L::kMergePitch + 32] = m_eff;
             merge[Lr * L::kMergePitch + 33] = l;
             named_bar_sync(1, 128);

@@ -71,16 +71,6 @@ __device__ __forceinline__ uint64_t desc_mnmajor_rows(uint32_t smem_addr, uint32
 
 constexpr float kTRescaleThreshold = 8.0f;  // log2 units: P may grow to 2^8 before the references are raised
 
-// OR over the `nthreads` softmax threads (named barrier 1).
-__device__ __forceinline__ bool bar_or(bool v, int nthreads) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\tbarrier.cta.red.or.pred q, 1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r)
-        : "r"((uint32_t)v), "r"(nthreads)
-        : "memory");
-    return r != 0;
-}
 // Maximum of a float over the warp with one redux: floats are mapped to integers of the same order.
 __device__ __forceinline__ float warp_max_redux(float x) {
     int i = __float_as_int(x);
