@@ -245,7 +245,7 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
                 const uint32_t d = tmem_base + kAColS + (uint32_t)(n & 1) * 64;
 #pragma unroll 1
                 for (int g3 = 0; g3 < 3; ++g3) {
-                    if (!mbar_wait(&kfull[ks], kph, ab, 3)) return false;
+                    if (!mbar_wait_fast(&kfull[ks], kph, ab, 3)) return false;
                     tc_fence_after();
                     // descriptors as low words: the high word is a constant, stepping is one 32-bit add
                     const uint32_t kd = desc_lo(desc_kmajor_sw128(smem_u32(tiles + L::kOffK + ks * L::kKGroup)));
@@ -280,13 +280,13 @@ decode_absorb_tc_kernel(const AbsorbParams p, const __grid_constant__ CUtensorMa
                     } else {
                         umma_commit2(q_empty, 3);  // every Qh Kh^T of this piece has been issued
                     }
-                    if (!(ok = mbar_wait(&p_ready[n & 1], (n >> 1) & 1, ab, 5))) break;
+                    if (!(ok = mbar_wait_fast(&p_ready[n & 1], (n >> 1) & 1, ab, 5))) break;
                     // the first P.V of a piece overwrites O: the previous piece's O must have been read
                     if (t == 0 && pi > 0 && !(ok = mbar_wait(o_free, (pi - 1) & 1, ab, 14))) break;
                     tc_fence_after();
 #pragma unroll 1
                     for (int h = 0; h < 2; ++h) {
-                        if (!(ok = mbar_wait(&vfull[vs], vph, ab, 6))) break;
+                        if (!(ok = mbar_wait_fast(&vfull[vs], vph, ab, 6))) break;
                         tc_fence_after();
                         const uint32_t vd = desc_lo(desc_mnmajor_sw128(smem_u32(tiles + L::kOffV + vs * L::kVGroup), L::kBox));
                         const uint32_t pd = desc_lo(p_desc) + ((h * L::kBox) >> 4);
