@@ -130,8 +130,35 @@ def test_fp8_decode_both_paths(dims, policy, s_q):
     assert_close(og_part.cpu().numpy(), og_ref, "decode_gqa_fp8 o_part", rel, abs_)
     assert_close(lg_part.cpu().numpy(), lg_ref, "decode_gqa_fp8 lse_part", 1e-2, 1e-3)
     assert int(status.item()) == 0
+
     # the two quantised paths still describe the same attention: against the unquantised oracle within the input
     # rounding (two E4M3 roundings per product in the scores, one per value)
     ref = O.decode_gqa_partials(od, synth.to_f64(q), synth.to_f64(k_c), synth.to_f64(v), synth.to_f64(dev["cache"][:, w.r_kv:]),
                                 ss, sl, s_q, w.scale, S)[0]
     assert np.abs(og_part.cpu().numpy() - ref).max() <= 0.3 * np.abs(ref).max()
+
+    # ---- the balanced plan (num_splits < 0) cuts the sequences differently; what it must reproduce is the merged
+    # attention output, which no plan changes: both calls, merged, against the oracle's merged partials
+    o_ref, l_ref = O.combine_splits(op_ref, lp_ref)
+    g_ref, gl_ref = O.combine_splits(og_ref, lg_ref)
+    for slots in (2, 4):
+        o_part = torch.full((Bn, slots, s_q, w.h_q, w.r_kv), float("nan"), dtype=torch.float32, device="cuda")
+        lse_part = torch.full((Bn, slots, s_q, w.h_q), float("nan"), dtype=torch.float32, device="cuda")
+        B.gqla_decode_absorb_fp8(bd, q8, qs, cache8, sc, dev["seq_start"], dev["seqlens"], w.scale, -slots, o_part, lse_part,
+                                 status)
+        o_m = torch.empty((Bn, s_q, w.h_q, w.r_kv), dtype=torch.float32, device="cuda")
+        l_m = torch.empty((Bn, s_q, w.h_q), dtype=torch.float32, device="cuda")
+        B.gqla_combine_splits(o_part, lse_part, o_m, l_m)
+        assert_close(o_m.cpu().numpy(), o_ref, "balanced decode_absorb_fp8, merged", rel, abs_)
+        assert_close(l_m.cpu().numpy(), l_ref, "balanced decode_absorb_fp8, merged lse", 1e-2, 1e-3)
+        og_part = torch.full((Bn, slots, s_q, w.h_q, w.d_h), float("nan"), dtype=torch.float32, device="cuda")
+        lg_part = torch.full((Bn, slots, s_q, w.h_q), float("nan"), dtype=torch.float32, device="cuda")
+        B.gqla_decode_gqa_fp8(bd, q8g, qsg, kc8, v8, kr8, sv, dev["seq_start"], dev["seqlens"], w.scale, -slots, og_part,
+                              lg_part, status)
+        g_m = torch.empty((Bn, s_q, w.h_q, w.d_h), dtype=torch.float32, device="cuda")
+        gl_m = torch.empty((Bn, s_q, w.h_q), dtype=torch.float32, device="cuda")
+        B.gqla_combine_splits(og_part, lg_part, g_m, gl_m)
+        assert_close(g_m.cpu().numpy(), g_ref, "balanced decode_gqa_fp8, merged", rel, abs_)
+        assert_close(gl_m.cpu().numpy(), gl_ref, "balanced decode_gqa_fp8, merged lse", 1e-2, 1e-3)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
