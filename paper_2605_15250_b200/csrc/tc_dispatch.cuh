@@ -193,11 +193,12 @@ inline gqla_status tc_expand_cache(const gqla_dims& d, gqla_dtype dtype, int64_t
 }
 
 // 4-D view of a [B*s_q, h_q, feat] activation: (feat, head-in-group, group, position).
-inline bool make_grouped_act_map(CUtensorMap* m, const void* base, const gqla_dims& d, int feat, int64_t positions) {
+inline bool make_grouped_act_map(CUtensorMap* m, const void* base, const gqla_dims& d, int feat, int64_t positions,
+                                 int tile_rows = 128) {
     const int hpg = d.h_q / d.g, hpb = next_pow2(hpg);
     const uint64_t dims[4] = {(uint64_t)feat, (uint64_t)hpg, (uint64_t)d.g, (uint64_t)positions};
     const uint64_t str[3] = {(uint64_t)feat * 2, (uint64_t)hpg * feat * 2, (uint64_t)d.h_q * feat * 2};
-    const uint32_t box[4] = {64, (uint32_t)hpb, 1, (uint32_t)(128 / hpb)};  // beyond the hpg heads: zero fill
+    const uint32_t box[4] = {64, (uint32_t)hpb, 1, (uint32_t)(tile_rows / hpb)};  // beyond the hpg heads: zero fill
     return tc::make_tmap_bf16(m, base, 4, dims, str, box);
 }
 
@@ -232,10 +233,13 @@ inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, i
     if (!tc_gemm_covers(d, dtype)) return GQLA_ERR_UNSUPPORTED;
     const int hpg = d.h_q / d.g, hpb = next_pow2(hpg);
     const int64_t positions = (int64_t)B * s_q;
-    const int64_t m_tiles = (positions + 128 / hpb - 1) / (128 / hpb);
+    // 64-row tiles where a group's head slots allow: this kernel is bound by what one CTA pulls of o_hat (r_kv columns
+    // per row), and the 128-row tiling leaves more than half of the SMs idle at the shapes of a decode step
+    const int bm = hpb <= 64 ? 64 : 128;
+    const int64_t m_tiles = (positions + bm / hpb - 1) / (bm / hpb);
     if (m_tiles > 0x7fffffffLL) return GQLA_ERR_UNSUPPORTED;
     CUtensorMap tmA, tmB;
-    if (!make_grouped_act_map(&tmA, o_hat, d, d.r_kv, positions)) return GQLA_ERR_CUDA;
+    if (!make_grouped_act_map(&tmA, o_hat, d, d.r_kv, positions, bm)) return GQLA_ERR_CUDA;
     {
         // W_UV[j] as an MN-major B operand: rows = (j, r) (contraction), columns = d (output)
         const uint64_t dims[2] = {(uint64_t)d.d_h, (uint64_t)d.g * d.r_kv};
@@ -248,8 +252,9 @@ inline gqla_status tc_up_proj(const gqla_dims& d, gqla_dtype dtype, int32_t B, i
     p.m_total = positions;
     p.h_q = d.h_q; p.g = d.g; p.hpg = hpg; p.hpb = hpb; p.d_h = d.d_h; p.r_kv = d.r_kv; p.d_r = d.d_r;
     p.out0 = o; p.status = projection_status_word();
-    cudaError_t e =
-        tc::gemm_launch<tc::kGemmUpProj, 128, true>(p, tmA, tmB, tmB, dim3((unsigned)m_tiles, (unsigned)d.g, 1), st);
+    const dim3 grid((unsigned)m_tiles, (unsigned)d.g, 1);
+    cudaError_t e = bm == 64 ? tc::gemm_launch<tc::kGemmUpProj, 128, true, 64>(p, tmA, tmB, tmB, grid, st)
+                             : tc::gemm_launch<tc::kGemmUpProj, 128, true, 128>(p, tmA, tmB, tmB, grid, st);
     return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
 }
 

@@ -17,7 +17,7 @@ struct GemmParams {
     int32_t k_blocks;   // K / 64
     int64_t m_total;    // expand: cache rows N;  others: B * s_q (query positions)
     int32_t h_q, g, hpg, d_h, r_kv, d_r;
-    int32_t hpb;        // heads per group padded to a power of two: a tile is 128/hpb positions x hpb head slots
+    int32_t hpb;        // heads per group padded to a power of two: a tile is BM/hpb positions x hpb head slots
     void* out0;         // expand: k_c;  absorb_q: q_hat;  up_proj: o
     void* out1;         // expand: v
     const void* aux_in; // absorb_q: q_r (copied into q_hat's tail);  expand: cache (for the k_R copy)
@@ -26,23 +26,26 @@ struct GemmParams {
     int32_t* status;
 };
 
-template <int BN, bool B_MN>
+template <int BN, bool B_MN, int BM = 128>
 struct GemmSmem {
-    static constexpr int kStages = BN <= 128 ? 6 : 4;  // 32 KB or 48 KB per stage: 192 KB of tiles in flight
-    static constexpr int kABytes = 128 * 128;  // 128 rows x 64 bf16
+    static constexpr int kABytes = BM * 128;   // BM rows x 64 bf16
+    static constexpr int kStages = 196608 / (kABytes + BN * 128);  // 192 KB of tiles in flight: 4, 6 or 8 stages
     static constexpr int kBBytes = BN * 128;   // K-major: BN rows x 64 k;  MN-major: (BN/64) boxes of 64 k-rows x 64 n
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kOutPitch = BN * 2 + 16;  // output staging of the epilogue (reuses the stage ring)
-    static_assert(128 * kOutPitch <= kStages * kStageBytes, "output staging must fit in the stage ring");
+    static_assert(BM * kOutPitch <= kStages * kStageBytes, "output staging must fit in the stage ring");
+    static_assert(BM == 64 || BM == 128, "an MMA tile has 64 or 128 rows");
+    static_assert(2 * kStages + 1 <= 24, "barriers must fit in the 256 bytes behind the tiles");
     static constexpr int kTotal = kStages * kStageBytes + 1024 /*align slack*/ + 256 /*barriers*/;
     static_assert(OneCtaPerSM<kTotal>::value, "");
 };
 
-template <int MODE, int BN, bool B_MN>
+template <int MODE, int BN, bool B_MN, int BM = 128>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1) {
-    using L = GemmSmem<BN, B_MN>;
+    using L = GemmSmem<BN, B_MN, BM>;
+    static_assert(BM == 128 || MODE != kGemmExpand, "the expansion uses 128-row tiles");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + L::kStages * L::kStageBytes);
@@ -138,7 +141,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
                         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], "
                         "[%1, {%3, %4, %5, %6}], [%2];" ::"r"(smem_u32(a_dst)),
                         "l"(reinterpret_cast<uint64_t>(&tmA)), "r"(smem_u32(&full[s])), "r"(kb * 64), "r"(0), "r"(j),
-                        "r"(m_tile * (128 / p.hpb))
+                        "r"(m_tile * (BM / p.hpb))
                         : "memory");
                 }
                 if (kb >= n_pre) load_b(kb, s);
@@ -146,7 +149,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
         }
     } else if (warp == 1) {
         if (elect_one()) {
-            constexpr uint32_t idesc = idesc_bf16(128, BN, 0, B_MN ? 1 : 0);
+            constexpr uint32_t idesc = idesc_bf16(BM, BN, 0, B_MN ? 1 : 0);
             bool ok = true;
             for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
                 const int s = kb % L::kStages;
@@ -170,7 +173,9 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
     } else {
         // epilogue: warp w may touch TMEM lanes [32 * (w % 4), +32)
         const int q = warp & 3;
-        const int row = q * 32 + lane;  // row of the tile == TMEM lane
+        // row of the tile: the TMEM lane for 128-row tiles; a 64-row accumulator sits in lanes 0-15 of each quadrant
+        const int row = BM == 128 ? q * 32 + lane : q * 16 + (lane & 15);
+        const bool has_row = BM == 128 || lane < 16;
         // (output addresses and the side copies first: they overlap the main loop instead of following it)
         __nv_bfloat16* dst = nullptr;
         if (MODE == kGemmExpand) {
@@ -186,10 +191,10 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
                 }
             }
         } else {
-            const int64_t bp = (int64_t)m_tile * (128 / p.hpb) + row / p.hpb;
+            const int64_t bp = (int64_t)m_tile * (BM / p.hpb) + row / p.hpb;
             const int il = row % p.hpb;
             const int i = j * p.hpg + il;
-            if (bp < p.m_total && il < p.hpg) {
+            if (has_row && bp < p.m_total && il < p.hpg) {
                 const int64_t r = bp * p.h_q + i;
                 if (MODE == kGemmAbsorbQ) {
                     __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out0) + r * (p.r_kv + p.d_r);
@@ -221,6 +226,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
                 tmem_ld32(tmem_addr(tmem_base, q * 32, c0 + 32), v + 32);
                 tmem_wait_ld();
                 uint4* d4 = reinterpret_cast<uint4*>(srow + c0 * 2);
+                if (has_row)  // (lanes 16-31 of a 64-row accumulator hold nothing)
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
                     uint4 o;
@@ -246,11 +252,11 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmA, cons
 
 // ----------------------------------------------------------------------------- host launchers
 
-template <int MODE, int BN, bool B_MN>
+template <int MODE, int BN, bool B_MN, int BM = 128>
 inline cudaError_t gemm_launch(const GemmParams& p, const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1,
                                dim3 grid, cudaStream_t st) {
-    using L = GemmSmem<BN, B_MN>;
-    auto kern = gemm_tc_kernel<MODE, BN, B_MN>;
+    using L = GemmSmem<BN, B_MN, BM>;
+    auto kern = gemm_tc_kernel<MODE, BN, B_MN, BM>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
