@@ -165,8 +165,9 @@ __device__ __forceinline__ float4 ld_stream4(const float* p) {  // read once: do
                  : "l"(p));
     return v;
 }
-// V = 4 or 8 output columns per thread (8 where d_out allows: half the threads, i.e. one wave of them on the shapes
-// of the decode chains, and 16-byte stores of bf16).
+// V = 4, 8 or 16 output columns per thread (as many as d_out allows: the kernel's CTAs wait, resident beside those of
+// the decode kernel, for it to finish, and only a grid small enough to be resident as a whole runs as one wave;
+// 16-byte stores of bf16).
 template <typename TO, int V>
 __global__ void __launch_bounds__(256) combine_vec_kernel(int64_t rows, int32_t rows_per_seq, int32_t S, int32_t d_out,
                                                           const float* __restrict__ o_part,
@@ -210,15 +211,19 @@ __global__ void __launch_bounds__(256) combine_vec_kernel(int64_t rows, int32_t 
     for (int u = 0; u < V / 4; ++u) {
         acc[u].x *= inv; acc[u].y *= inv; acc[u].z *= inv; acc[u].w *= inv;
     }
-    if constexpr (V == 8 && sizeof(TO) == 2) {  // eight bf16: one 16-byte store
-        __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[0].x, acc[0].y), h1 = __floats2bfloat162_rn(acc[0].z, acc[0].w);
-        __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[1].x, acc[1].y), h3 = __floats2bfloat162_rn(acc[1].z, acc[1].w);
-        uint4 u4;
-        u4.x = *reinterpret_cast<uint32_t*>(&h0);
-        u4.y = *reinterpret_cast<uint32_t*>(&h1);
-        u4.z = *reinterpret_cast<uint32_t*>(&h2);
-        u4.w = *reinterpret_cast<uint32_t*>(&h3);
-        *reinterpret_cast<uint4*>(out + r * d_out + c) = u4;
+    if constexpr (V >= 8 && sizeof(TO) == 2) {  // eight bf16 per 16-byte store
+#pragma unroll
+        for (int u = 0; u < V / 8; ++u) {
+            __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[2 * u].x, acc[2 * u].y), h1 = __floats2bfloat162_rn(acc[2 * u].z, acc[2 * u].w);
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[2 * u + 1].x, acc[2 * u + 1].y),
+                           h3 = __floats2bfloat162_rn(acc[2 * u + 1].z, acc[2 * u + 1].w);
+            uint4 u4;
+            u4.x = *reinterpret_cast<uint32_t*>(&h0);
+            u4.y = *reinterpret_cast<uint32_t*>(&h1);
+            u4.z = *reinterpret_cast<uint32_t*>(&h2);
+            u4.w = *reinterpret_cast<uint32_t*>(&h3);
+            *reinterpret_cast<uint4*>(out + r * d_out + c + 8 * u) = u4;
+        }
     } else {
 #pragma unroll
         for (int u = 0; u < V / 4; ++u) store4(out + r * d_out + c + 4 * u, acc[u]);

@@ -474,24 +474,20 @@ gqla_status gqla_combine_splits(int32_t B, int32_t rows_per_seq, int32_t num_spl
     if (rows > 0x7fffffffLL) return GQLA_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (d_out % 4 == 0) {
-        const int vec = d_out % 8 == 0 ? 8 : 4;  // output columns per thread
+        const int vec = d_out % 16 == 0 ? 16 : (d_out % 8 == 0 ? 8 : 4);  // output columns per thread
         const int64_t items = rows * (d_out / vec);
         const int64_t nblk = (items + 255) / 256;
         if (nblk > 0x7fffffffLL) return GQLA_ERR_SHAPE;
-        const unsigned blocks = (unsigned)nblk;
+        const dim3 blocks((unsigned)nblk), threads(256);
+        const bool bf = out_dtype == GQLA_BF16;
         cudaError_t e;
-        if (out_dtype == GQLA_BF16 && vec == 8)
-            e = tc::launch_pdl(combine_vec_kernel<__nv_bfloat16, 8>, dim3(blocks), dim3(256), 0, st, rows, rows_per_seq,
-                               num_splits, d_out, o_part, lse_part, (__nv_bfloat16*)out, lse);
-        else if (out_dtype == GQLA_BF16)
-            e = tc::launch_pdl(combine_vec_kernel<__nv_bfloat16, 4>, dim3(blocks), dim3(256), 0, st, rows, rows_per_seq,
-                               num_splits, d_out, o_part, lse_part, (__nv_bfloat16*)out, lse);
-        else if (vec == 8)
-            e = tc::launch_pdl(combine_vec_kernel<float, 8>, dim3(blocks), dim3(256), 0, st, rows, rows_per_seq, num_splits,
-                               d_out, o_part, lse_part, (float*)out, lse);
-        else
-            e = tc::launch_pdl(combine_vec_kernel<float, 4>, dim3(blocks), dim3(256), 0, st, rows, rows_per_seq, num_splits,
-                               d_out, o_part, lse_part, (float*)out, lse);
+#define GQLA_COMBINE(TO, V)                                                                                              \
+    e = tc::launch_pdl(combine_vec_kernel<TO, V>, blocks, threads, 0, st, rows, rows_per_seq, num_splits, d_out, o_part, \
+                       lse_part, (TO*)out, lse)
+        if (vec == 16) { if (bf) GQLA_COMBINE(__nv_bfloat16, 16); else GQLA_COMBINE(float, 16); }
+        else if (vec == 8) { if (bf) GQLA_COMBINE(__nv_bfloat16, 8); else GQLA_COMBINE(float, 8); }
+        else { if (bf) GQLA_COMBINE(__nv_bfloat16, 4); else GQLA_COMBINE(float, 4); }
+#undef GQLA_COMBINE
         return e == cudaSuccess ? GQLA_OK : GQLA_ERR_CUDA;
     }
     const size_t smem = (size_t)num_splits * sizeof(float);
